@@ -1,0 +1,153 @@
+/* gnn.h -- C ABI of libgnn_b200: graph message passing on one NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the message-passing primitives of Sec. 3 ("Message Passing") of
+ * "GraphNeuralNetworks.jl: Deep Learning on Graphs with Julia" (arXiv 2412.06354):
+ * gather / scatter, apply_edges, aggregate_neighbors, and propagate, which fuses the two
+ * into a generalised sparse x dense product; plus the pieces of Sec. 3 "Graph Data
+ * Structures" (COO -> sparse form, batching) and "Graph Convolutional Layers" (GCN
+ * normalisation, GAT edge softmax) that the hot path needs, each with its backward pass.
+ *
+ * Conventions (all calls)
+ *  - Edge k runs from source src[k] = j to target dst[k] = i.  Messages flow j -> i and are
+ *    reduced at i over its incoming edges.  Indices are 0-based.  Node ids and edge ids are
+ *    int32 (E < 2^31), row pointers int64.
+ *  - Every pointer is a DEVICE pointer unless its name starts with h_ or the comment says
+ *    host.  gnn_csr itself is a host struct holding device pointers.
+ *  - The caller owns every buffer, including workspaces; the library never allocates or
+ *    frees device memory.  Calls enqueue work on the given stream and return without
+ *    synchronising, except gnn_coo_to_csr, which synchronises the stream once to read its
+ *    4-byte validation word, and the *_host calls, which are documented where declared.
+ *  - Feature matrices are row-major with the feature index contiguous ([N,F], [E,F], [G,F]),
+ *    base address 16-byte aligned, and F*sizeof(element) a multiple of 16 bytes and at most
+ *    2048 bytes for the row-gathering calls (GNN_ERR_UNSUPPORTED otherwise).
+ *  - Edge-aligned arrays passed to calls that take a gnn_csr are in CSR order (position p of
+ *    the by-target form) unless stated; use gnn_permute_edge_data(eid, ...) once to reorder
+ *    COO-ordered data.  Backward calls take weights in transposed-CSR order.
+ *  - Sums accumulate in fp32 in a fixed order: results are bit-identical from run to run.
+ *    No floating-point atomics are used anywhere.
+ *  - Errors: argument errors are detected on the host before any launch and returned as a
+ *    gnn_status; nothing traps.  Outputs are unspecified after an error.
+ */
+#ifndef GNN_B200_H
+#define GNN_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* opaque stream handle: a cudaStream_t (0 = default stream) */
+typedef void* gnn_stream;
+
+typedef enum {
+    GNN_OK = 0,
+    GNN_ERR_INVALID_ARG = 1,
+    GNN_ERR_INDEX_OUT_OF_RANGE = 2,
+    GNN_ERR_NOT_SORTED = 3,
+    GNN_ERR_WORKSPACE_TOO_SMALL = 4,
+    GNN_ERR_UNSUPPORTED = 5,
+    GNN_ERR_CUDA = 6,
+    GNN_ERR_TIMEOUT = 7
+} gnn_status;
+
+typedef enum { GNN_F32 = 0, GNN_BF16 = 1 } gnn_dtype;
+typedef enum { GNN_SUM = 0, GNN_MEAN = 1, GNN_MAX = 2, GNN_MIN = 3 } gnn_op;
+typedef enum { GNN_MSG_COPY_XJ = 0, GNN_MSG_E_MUL_XJ = 1, GNN_MSG_GAT_LOGIT = 2 } gnn_msg;
+
+/* Sparse form of a graph (Sec. 3 "Graph Data Structures": the sparse adjacency encoding the
+ * fused operations run on).  Host struct, device arrays, all caller-owned.
+ *   by target:  rows = targets; rowptr[N+1]; col[p] = source of the edge at position p;
+ *               eid[p] = index of that edge in the original COO list.  Within a row, positions
+ *               are in ascending eid (stable), which makes the form unique.
+ *   transposed: rows = sources; rowptrT[N+1]; colT[q] = target; eidT[q] likewise.
+ *   t2f[q]    = position p in the by-target form of the edge at transposed position q. */
+typedef struct {
+    int32_t N;
+    int64_t E;
+    int64_t* rowptr;
+    int32_t* col;
+    int32_t* eid;
+    int64_t* rowptrT;
+    int32_t* colT;
+    int32_t* eidT;
+    int32_t* t2f;
+} gnn_csr;
+
+const char* gnn_status_string(gnn_status s);
+/* text of the most recent error on the calling thread ("" if none); host string */
+const char* gnn_last_error_string(void);
+int gnn_version(void);
+
+/* ------------------------------------------------------------------ graph set-up ---------- */
+
+/* COO (the default topology format, Sec. 3 "Graph Data Structures") -> both sparse forms.
+ * src, dst: int32 [E].  out: host struct whose seven array pointers the caller has set to
+ * device buffers of sizes rowptr,rowptrT [N+1] int64 and col,eid,colT,eidT,t2f [E] int32; N and
+ * E are filled in.  Validates 0 <= src,dst < N first (GNN_ERR_INDEX_OUT_OF_RANGE; one stream
+ * synchronisation to read the flag).  ws: scratch of at least gnn_coo_to_csr_workspace bytes.
+ * The result is unique, so it can be compared bit for bit. */
+size_t gnn_coo_to_csr_workspace(int32_t N, int64_t E);
+gnn_status gnn_coo_to_csr(int32_t N, int64_t E, const int32_t* src, const int32_t* dst,
+                          gnn_csr* out, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Degrees (graph utility of Sec. 3 "Graph Data Structures").  transposed == 0: incoming edges
+ * per node; != 0: outgoing.  w == NULL: deg_out is int32 [N] (edge counts, duplicates and
+ * loops included).  w != NULL: float [N], the sum of w over the row, w in the order of the
+ * chosen form (CSR order, or transposed-CSR order when transposed != 0). */
+gnn_status gnn_degree(const gnn_csr* g, int transposed, const float* w, void* deg_out,
+                      gnn_stream stream);
+
+/* Append one self-loop per node after the original edges, in node order (A^ = A + I of the GCN
+ * layer named in Sec. 3 "Graph Convolutional Layers").  src_out, dst_out: int32 [E+N]. */
+gnn_status gnn_add_self_loops(int32_t N, int64_t E, const int32_t* src, const int32_t* dst,
+                              int32_t* src_out, int32_t* dst_out, gnn_stream stream);
+
+/* Symmetric GCN normalisation for a graph that already contains its self-loops:
+ * d_i = sum of w over the edges into i (w == NULL: every edge counts 1);
+ * coefficient of edge j->i = w / sqrt(d_i * d_j), or 0 if either degree is 0.
+ * w_csr: NULL or float [E] in CSR order.  Outputs: deg_out float [N] (d), coef_csr float [E] in
+ * CSR order, coef_csrT float [E] in transposed-CSR order (either coef pointer may be NULL). */
+gnn_status gnn_gcn_norm(const gnn_csr* g, const float* w_csr, float* deg_out, float* coef_csr,
+                        float* coef_csrT, gnn_stream stream);
+
+/* out[p, 0..width) = in[perm[p], 0..width) for p < E: reorders edge data, e.g. perm = eid turns
+ * COO order into CSR order, perm = t2f turns CSR order into transposed-CSR order.
+ * elem_bytes is the size of one element (1, 2, 4 or 8).  in and out must not overlap. */
+gnn_status gnn_permute_edge_data(const int32_t* perm, int64_t E, int width, int elem_bytes,
+                                 const void* in, void* out, gnn_stream stream);
+
+/* ------------------------------------------------------------------ fused propagate -------- */
+
+/* propagate (Sec. 3 "Message Passing": apply_edges and aggregate_neighbors combined, the
+ * generalised matrix product), never materialising the E x F message tensor:
+ *   out[i,:] = op over positions p in [rowptr[i], rowptr[i+1]) of  w[p] * X[col[p],:]
+ * msg = GNN_MSG_COPY_XJ (w_csr ignored, may be NULL) or GNN_MSG_E_MUL_XJ (w_csr float [E], one
+ * scalar per edge, CSR order).  op: SUM; MEAN (sum divided by the number of incoming edges);
+ * MAX / MIN (element-wise; argmax int32 [N,F] receives the CSR position of the winner, the
+ * smallest position among equal values; may be NULL).  A node with no incoming edge gets 0 and
+ * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes.
+ * Bytes moved per call: at least 4E (+4E with weights) + 8N + 2*N*F*s, at most
+ * 4E (+4E) + 8N + (E+N)*F*s when no source row is found in L2. */
+size_t gnn_propagate_fused_workspace(int64_t E, int F, gnn_op op);
+gnn_status gnn_propagate_fused(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* X,
+                               const float* w_csr, int F, gnn_dtype dtype, void* out,
+                               int32_t* argmax, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Backward of gnn_propagate_fused for dL/dout = dOut [N,F]:
+ *   SUM/MEAN: dX[j,:] = sum over transposed positions q of row j of
+ *                       wT[q] * scale(colT[q]) * dOut[colT[q],:],  scale = 1 or 1/indegree
+ *             dW[p]   = scale(i) * <X[col[p],:], dOut[i,:]>  for p in row i (CSR order)
+ *   MAX/MIN : dX[j,f] = sum over q in row j of [argmax[colT[q],f] == t2f[q]] * wT[q]*dOut[colT[q],f]
+ * w_csrT: float [E] in transposed-CSR order (E_MUL_XJ) or NULL.  X is needed only for dW.
+ * dX [N,F] and dW float [E] may each be NULL (skipped).  ws as for the forward call. */
+gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op,
+                                        const void* dOut, const void* X, const float* w_csrT,
+                                        const int32_t* argmax, int F, gnn_dtype dtype, void* dX,
+                                        float* dW, void* ws, size_t ws_bytes, gnn_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GNN_B200_H */
