@@ -48,31 +48,34 @@ static inline int grid_for(int64_t n, int threads) {
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 
-// 16-byte global loads/stores with cache hints.
+// 16-byte global loads/stores with L2 cache policies (createpolicy + .L2::cache_hint).
 //   feature rows that are gathered many times: keep in L2 (evict_last)
 //   index / weight / output streams touched once: evict_first, no L1 allocation
-__device__ __forceinline__ uint4 ld_row16(const void* p) {
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ld_hint16(const void* p, uint64_t pol) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_last.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
+                 : "l"(p), "l"(pol));
     return v;
 }
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-__device__ __forceinline__ int ld_stream_i32(const int* p) {
+__device__ __forceinline__ int ld_hint_i32(const int* p, uint64_t pol) {
     int v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.s32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol));
     return v;
 }
-__device__ __forceinline__ float ld_stream_f32(const float* p) {
+__device__ __forceinline__ float ld_hint_f32(const float* p, uint64_t pol) {
     float v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(pol));
     return v;
 }
 __device__ __forceinline__ void st_stream16(void* p, uint4 v) {

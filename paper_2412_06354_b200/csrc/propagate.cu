@@ -1,0 +1,599 @@
+// Fused propagate (Sec. 3 "Message Passing": apply_edges + aggregate_neighbors combined into a
+// generalised sparse x dense product) and its backward passes.
+//
+// Work decomposition: the E positions of the sparse form are cut into fixed chunks of PF_CHUNK
+// consecutive edges, one warp per chunk (merge-path style: perfect balance on power-law rows
+// without any per-graph schedule).  A warp finds its first row by binary search in rowptr and
+// walks the rows that start inside its chunk.  Rows lying wholly inside the chunk are reduced
+// and written directly.  A row cut by a chunk boundary leaves fp32 partials (one "head" slot and
+// one "tail" slot per chunk) that a second kernel combines in ascending chunk order.  Every
+// accumulation order is a fixed function of (E, F, dtype), so results are bit-reproducible and
+// no floating-point atomics are needed.
+//
+// Inside a warp, a feature row of F*s bytes is covered by LPR lanes holding one 16-byte chunk
+// each (times VPL when a row is wider than 512 bytes); the 32/LPR lane groups take alternating
+// edges, and are combined by an xor-shuffle tree at the end of each row.
+#include "propagate.cuh"
+
+namespace gnn {
+
+struct PropParams {
+    const int64_t* rowptr;  // rows of the output
+    const int32_t* col;     // gathered row of X per position
+    const float* w;         // per-position multiplier or nullptr
+    const void* X;          // gathered matrix [N,F]
+    void* out;              // [N,F]
+    int32_t* argmax;        // MODE_MAX/MIN: winner positions [N,F] or nullptr
+    const int64_t* gscale_rowptr;  // if set: each gathered row c is divided by max(1, length of
+                                   // row c in this other sparse form) -- backward of MEAN
+    const int32_t* route_arg;  // MODE_ROUTE: forward argmax [N,F]
+    const int32_t* route_pos;  // MODE_ROUTE: forward position of each transposed position
+    int32_t N;
+    int64_t E;
+    int nvec;  // 16-byte chunks per feature row
+    int F;
+    int mean;  // divide the finished row by max(1, row length)
+    int64_t nchunks;
+    int32_t* tail_row;  // [nchunks] row whose tail partial lives in slot 1, or -1
+    float* part_val;    // [nchunks][2][F]
+    int32_t* part_arg;  // [nchunks][2][F] (MODE_MAX/MIN)
+    uint64_t pol_keep, pol_stream;  // L2 policies, filled in on the device
+};
+
+template <typename T, int VPL, int MODE>
+struct Acc {
+    static constexpr int EPC = Chunk<T>::N;
+    static constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
+    float v[VPL][EPC];
+    int32_t a[ARG ? VPL : 1][EPC];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i)
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) {
+                v[i][j] = 0.f;
+                if (ARG) a[i][j] = -1;
+            }
+    }
+};
+
+// does candidate (cv, ca) beat the incumbent (v, a)?  ties go to the smaller position
+template <int MODE>
+__device__ __forceinline__ bool beats(float cv, int32_t ca, float v, int32_t a) {
+    if (ca < 0) return false;
+    if (a < 0) return true;
+    bool better = (MODE == MODE_MAX) ? (cv > v) : (cv < v);
+    return better || (cv == v && ca < a);
+}
+
+template <typename T, int LPR, int VPL, int MODE>
+struct Walker {
+    static constexpr int EPC = Chunk<T>::N;
+    static constexpr int NG = 32 / LPR;
+    static constexpr int U = (LPR >= 16) ? (8 / VPL) : 4;
+    static constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
+    using A = Acc<T, VPL, MODE>;
+
+    // accumulate positions [a, b) of one row into acc (this lane group's share)
+    __device__ __forceinline__ static void segment(const PropParams& P, int64_t a, int64_t b,
+                                                   int lane, A& acc) {
+        const int g = lane / LPR, li = lane % LPR;
+        const char* Xb = reinterpret_cast<const char*>(P.X);
+        const size_t row_bytes = (size_t)P.nvec * 16;
+        for (int64_t base = a; base < b; base += 32) {
+            const int n = (int)((b - base) < 32 ? (b - base) : 32);
+            int myc = 0;
+            float myw = 1.f;
+            int myt = 0;
+            if (lane < n) {
+                myc = ld_hint_i32(P.col + base + lane, P.pol_stream);
+                if (P.w) myw = ld_hint_f32(P.w + base + lane, P.pol_stream);
+                if (P.gscale_rowptr) {
+                    int64_t d = P.gscale_rowptr[myc + 1] - P.gscale_rowptr[myc];
+                    myw = myw / (float)(d > 1 ? d : 1);
+                }
+                if (MODE == MODE_ROUTE) myt = ld_hint_i32(P.route_pos + base + lane, P.pol_stream);
+            }
+            const int rounds = (n + NG - 1) / NG;
+            for (int r0 = 0; r0 < rounds; r0 += U) {
+                uint4 buf[U][VPL];
+                float wv[U];
+                int tv[U];
+                int cv[U];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int e = (r0 + u) * NG + g;
+                    ok[u] = e < n;
+                    cv[u] = __shfl_sync(0xffffffffu, myc, e & 31);
+                    wv[u] = __shfl_sync(0xffffffffu, myw, e & 31);
+                    tv[u] = (MODE == MODE_ROUTE) ? __shfl_sync(0xffffffffu, myt, e & 31) : 0;
+                    if (ok[u]) {
+                        const char* rp = Xb + (size_t)cv[u] * row_bytes;
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            const int ci = v * LPR + li;
+                            if (ci < P.nvec) buf[u][v] = ld_hint16(rp + (size_t)ci * 16, P.pol_keep);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (!ok[u]) continue;
+                    const int32_t pos = (int32_t)(base + (r0 + u) * NG + g);
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) {
+                        const int ci = v * LPR + li;
+                        if (ci >= P.nvec) continue;
+                        float x[EPC];
+                        Chunk<T>::unpack(buf[u][v], x);
+                        if (MODE == MODE_SUM) {
+#pragma unroll
+                            for (int j = 0; j < EPC; ++j) acc.v[v][j] = fmaf(wv[u], x[j], acc.v[v][j]);
+                        } else if (ARG) {
+#pragma unroll
+                            for (int j = 0; j < EPC; ++j) {
+                                float m = P.w ? wv[u] * x[j] : x[j];
+                                // positions arrive in ascending order within a group: strict
+                                // comparison keeps the first of equal values
+                                bool take = acc.a[ARG ? v : 0][j] < 0 ||
+                                            (MODE == MODE_MAX ? m > acc.v[v][j] : m < acc.v[v][j]);
+                                if (take) { acc.v[v][j] = m; acc.a[ARG ? v : 0][j] = pos; }
+                            }
+                        } else {  // MODE_ROUTE: keep dOut only where this edge was the winner
+                            const int32_t* ap = P.route_arg + (size_t)cv[u] * P.F + (size_t)ci * EPC;
+                            int32_t win[EPC];
+#pragma unroll
+                            for (int j = 0; j < EPC; j += 4) {
+                                int4 t = *reinterpret_cast<const int4*>(ap + j);
+                                win[j] = t.x; win[j + 1] = t.y; win[j + 2] = t.z; win[j + 3] = t.w;
+                            }
+#pragma unroll
+                            for (int j = 0; j < EPC; ++j)
+                                if (win[j] == tv[u]) acc.v[v][j] = fmaf(wv[u], x[j], acc.v[v][j]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // combine the lane groups; afterwards every lane holds the result for its chunk index
+    __device__ __forceinline__ static void combine_groups(A& acc, int lane) {
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            const bool low = (lane & o) == 0;
+#pragma unroll
+            for (int v = 0; v < VPL; ++v)
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) {
+                    float mine = acc.v[v][j];
+                    float ov = __shfl_xor_sync(0xffffffffu, mine, o);
+                    if (ARG) {
+                        int32_t ma = acc.a[ARG ? v : 0][j];
+                        int32_t oa = __shfl_xor_sync(0xffffffffu, ma, o);
+                        if (beats<MODE>(ov, oa, mine, ma)) { acc.v[v][j] = ov; acc.a[ARG ? v : 0][j] = oa; }
+                    } else {
+                        // both partners add in the same operand order -> identical bits
+                        acc.v[v][j] = low ? (mine + ov) : (ov + mine);
+                    }
+                }
+        }
+    }
+
+    __device__ __forceinline__ static void write_final(const PropParams& P, int64_t row,
+                                                       int64_t deg, int lane, A& acc) {
+        if (lane >= LPR) return;
+        char* ob = reinterpret_cast<char*>(P.out) + (size_t)row * P.nvec * 16;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int ci = v * LPR + lane;
+            if (ci >= P.nvec) continue;
+            if (P.mean) {
+                float d = (float)(deg > 1 ? deg : 1);
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) acc.v[v][j] = acc.v[v][j] / d;
+            }
+            st_stream16(ob + (size_t)ci * 16, Chunk<T>::pack(acc.v[v]));
+            if (ARG && P.argmax) {
+                int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
+#pragma unroll
+                for (int j = 0; j < EPC; j += 4)
+                    *reinterpret_cast<int4*>(ap + j) =
+                        make_int4(acc.a[ARG ? v : 0][j], acc.a[ARG ? v : 0][j + 1],
+                                  acc.a[ARG ? v : 0][j + 2], acc.a[ARG ? v : 0][j + 3]);
+            }
+        }
+    }
+
+    __device__ __forceinline__ static void write_partial(const PropParams& P, int64_t chunk,
+                                                         int which, int lane, const A& acc) {
+        if (lane >= LPR) return;
+        size_t off = ((size_t)chunk * 2 + which) * P.F;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int ci = v * LPR + lane;
+            if (ci >= P.nvec) continue;
+            float* pv = P.part_val + off + (size_t)ci * EPC;
+#pragma unroll
+            for (int j = 0; j < EPC; j += 4)
+                *reinterpret_cast<float4*>(pv + j) =
+                    make_float4(acc.v[v][j], acc.v[v][j + 1], acc.v[v][j + 2], acc.v[v][j + 3]);
+            if (ARG) {
+                int32_t* pa = P.part_arg + off + (size_t)ci * EPC;
+#pragma unroll
+                for (int j = 0; j < EPC; j += 4)
+                    *reinterpret_cast<int4*>(pa + j) =
+                        make_int4(acc.a[ARG ? v : 0][j], acc.a[ARG ? v : 0][j + 1],
+                                  acc.a[ARG ? v : 0][j + 2], acc.a[ARG ? v : 0][j + 3]);
+            }
+        }
+    }
+};
+
+template <typename T, int LPR, int VPL, int MODE>
+__global__ void __launch_bounds__(PF_WARPS * 32)
+propagate_chunk_kernel(const PropParams P0) {
+    PropParams P = P0;
+    P.pol_keep = policy_evict_last();
+    P.pol_stream = policy_evict_first();
+    using W = Walker<T, LPR, VPL, MODE>;
+    const int lane = threadIdx.x & 31;
+    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + (threadIdx.x >> 5);
+    if (c >= P.nchunks) return;
+    const int64_t cs = c * PF_CHUNK;
+    const int64_t ce = (cs + PF_CHUNK < P.E) ? cs + PF_CHUNK : P.E;
+    const bool last = (c == P.nchunks - 1);
+    typename W::A acc;
+
+    int r = lower_bound_i64(P.rowptr, P.N + 1, cs);  // first row starting at or after cs
+    int64_t rs = P.rowptr[r];
+    if (rs > cs) {  // the row before it started earlier and reaches into this chunk: head partial
+        acc.clear();
+        W::segment(P, cs, rs < ce ? rs : ce, lane, acc);
+        W::combine_groups(acc, lane);
+        W::write_partial(P, c, 0, lane, acc);
+    }
+    int32_t tail = -1;
+    for (; r < P.N; ++r) {
+        if (!(rs < ce || last)) break;
+        const int64_t re = P.rowptr[r + 1];
+        acc.clear();
+        W::segment(P, rs, re < ce ? re : ce, lane, acc);
+        W::combine_groups(acc, lane);
+        if (re <= ce) {
+            W::write_final(P, r, re - rs, lane, acc);
+        } else {
+            W::write_partial(P, c, 1, lane, acc);
+            tail = r;
+            break;
+        }
+        rs = re;
+    }
+    if (lane == 0) P.tail_row[c] = tail;
+}
+
+// second pass: finish the rows that were cut by chunk boundaries, in ascending chunk order
+template <typename T, int MODE>
+__global__ void propagate_fixup_kernel(const PropParams P) {
+    constexpr int EPC = Chunk<T>::N;
+    constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t c = t / P.nvec;
+    const int ci = (int)(t - c * P.nvec);
+    if (c >= P.nchunks) return;
+    const int32_t r = P.tail_row[c];
+    if (r < 0) return;
+    const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
+    const int64_t c_end = (re - 1) / PF_CHUNK;
+    float v[EPC];
+    int32_t a[EPC];
+    const size_t F = P.F;
+    {
+        const float* pv = P.part_val + ((size_t)c * 2 + 1) * F + (size_t)ci * EPC;
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] = pv[j];
+        if (ARG) {
+            const int32_t* pa = P.part_arg + ((size_t)c * 2 + 1) * F + (size_t)ci * EPC;
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) a[j] = pa[j];
+        }
+    }
+    for (int64_t cc = c + 1; cc <= c_end; ++cc) {
+        const float* pv = P.part_val + ((size_t)cc * 2) * F + (size_t)ci * EPC;
+        if (ARG) {
+            const int32_t* pa = P.part_arg + ((size_t)cc * 2) * F + (size_t)ci * EPC;
+#pragma unroll
+            for (int j = 0; j < EPC; ++j)
+                if (beats<MODE>(pv[j], pa[j], v[j], a[j])) { v[j] = pv[j]; a[j] = pa[j]; }
+        } else {
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) v[j] += pv[j];
+        }
+    }
+    if (P.mean) {
+        float d = (float)(re - rs);
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] = v[j] / d;
+    }
+    char* ob = reinterpret_cast<char*>(P.out) + ((size_t)r * P.nvec + ci) * 16;
+    *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
+    if (ARG && P.argmax) {
+        int32_t* ap = P.argmax + (size_t)r * F + (size_t)ci * EPC;
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) ap[j] = a[j];
+    }
+}
+
+// ------------------------------------------------------------------ edge-weight gradient (SDDMM)
+// dW[p] = scale(i) * <X[col[p],:], dOut[i,:]> for p in row i.  Same chunking; every edge is
+// independent, so no partials.  The dOut row stays in registers along the row.
+struct SddmmParams {
+    const int64_t* rowptr;
+    const int32_t* col;
+    const void* X;
+    const void* dOut;
+    float* dW;
+    int32_t N;
+    int64_t E;
+    int nvec;
+    int mean;
+    int64_t nchunks;
+};
+
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(PF_WARPS * 32)
+sddmm_chunk_kernel(const SddmmParams P) {
+    constexpr int EPC = Chunk<T>::N;
+    constexpr int NG = 32 / LPR;
+    constexpr int U = (LPR >= 16) ? (8 / VPL) : 4;
+    const int lane = threadIdx.x & 31, g = lane / LPR, li = lane % LPR;
+    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + (threadIdx.x >> 5);
+    if (c >= P.nchunks) return;
+    const int64_t cs = c * PF_CHUNK;
+    const int64_t ce = (cs + PF_CHUNK < P.E) ? cs + PF_CHUNK : P.E;
+    if (cs >= ce) return;
+    const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
+    const size_t row_bytes = (size_t)P.nvec * 16;
+    const char* Xb = reinterpret_cast<const char*>(P.X);
+    const char* Db = reinterpret_cast<const char*>(P.dOut);
+    // row containing position cs: last row with rowptr[r] <= cs
+    int r = lower_bound_i64(P.rowptr, P.N + 1, cs + 1) - 1;
+    int64_t pos = cs;
+    while (pos < ce) {
+        while (P.rowptr[r + 1] <= pos) ++r;  // skip rows that end at or before pos
+        const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
+        const int64_t b = re < ce ? re : ce;
+        float d[VPL][EPC];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int ci = v * LPR + li;
+            if (ci < P.nvec) {
+                Chunk<T>::unpack(ld_hint16(Db + (size_t)r * row_bytes + (size_t)ci * 16, pol_stream), d[v]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) d[v][j] = 0.f;
+            }
+        }
+        const float scale = P.mean ? 1.0f / (float)(re - rs) : 1.0f;
+        for (int64_t base = pos; base < b; base += 32) {
+            const int n = (int)((b - base) < 32 ? (b - base) : 32);
+            int myc = lane < n ? ld_hint_i32(P.col + base + lane, pol_stream) : 0;
+            const int rounds = (n + NG - 1) / NG;
+            for (int r0 = 0; r0 < rounds; r0 += U) {
+                uint4 buf[U][VPL];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int e = (r0 + u) * NG + g;
+                    ok[u] = e < n;
+                    int cv = __shfl_sync(0xffffffffu, myc, e & 31);
+                    if (ok[u]) {
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            const int ci = v * LPR + li;
+                            if (ci < P.nvec) buf[u][v] = ld_hint16(Xb + (size_t)cv * row_bytes + (size_t)ci * 16, pol_keep);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    float dot = 0.f;
+                    if (ok[u]) {
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            const int ci = v * LPR + li;
+                            if (ci >= P.nvec) continue;
+                            float x[EPC];
+                            Chunk<T>::unpack(buf[u][v], x);
+#pragma unroll
+                            for (int j = 0; j < EPC; ++j) dot = fmaf(x[j], d[v][j], dot);
+                        }
+                    }
+#pragma unroll
+                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    if (ok[u] && li == 0) P.dW[base + (r0 + u) * NG + g] = scale * dot;
+                }
+            }
+        }
+        pos = b;
+    }
+}
+
+// ------------------------------------------------------------------ host dispatch
+bool pick_shape(int nvec, int* lpr, int* vpl) {
+    if (nvec < 1 || nvec > 128) return false;
+    if (nvec <= 4) { *lpr = 4; *vpl = 1; }
+    else if (nvec <= 8) { *lpr = 8; *vpl = 1; }
+    else if (nvec <= 16) { *lpr = 16; *vpl = 1; }
+    else if (nvec <= 32) { *lpr = 32; *vpl = 1; }
+    else if (nvec <= 64) { *lpr = 32; *vpl = 2; }
+    else { *lpr = 32; *vpl = 4; }
+    return true;
+}
+
+template <typename T, int MODE>
+static void launch_chunks(const PropParams& P, int lpr, int vpl, cudaStream_t st) {
+    const int grid = (int)ceil_div(P.nchunks, PF_WARPS);
+    const int thr = PF_WARPS * 32;
+#define GNN_PF_CASE(L, V) \
+    if (lpr == L && vpl == V) { propagate_chunk_kernel<T, L, V, MODE><<<grid, thr, 0, st>>>(P); }
+    GNN_PF_CASE(4, 1) GNN_PF_CASE(8, 1) GNN_PF_CASE(16, 1) GNN_PF_CASE(32, 1) GNN_PF_CASE(32, 2) GNN_PF_CASE(32, 4)
+#undef GNN_PF_CASE
+    const int64_t threads = P.nchunks * P.nvec;
+    propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
+}
+
+template <typename T>
+static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
+    switch (mode) {
+        case MODE_SUM: launch_chunks<T, MODE_SUM>(P, lpr, vpl, st); break;
+        case MODE_MAX: launch_chunks<T, MODE_MAX>(P, lpr, vpl, st); break;
+        case MODE_MIN: launch_chunks<T, MODE_MIN>(P, lpr, vpl, st); break;
+        default: launch_chunks<T, MODE_ROUTE>(P, lpr, vpl, st); break;
+    }
+}
+
+template <typename T>
+static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st) {
+    const int grid = (int)ceil_div(P.nchunks, PF_WARPS);
+    const int thr = PF_WARPS * 32;
+#define GNN_SD_CASE(L, V) \
+    if (lpr == L && vpl == V) { sddmm_chunk_kernel<T, L, V><<<grid, thr, 0, st>>>(P); }
+    GNN_SD_CASE(4, 1) GNN_SD_CASE(8, 1) GNN_SD_CASE(16, 1) GNN_SD_CASE(32, 1) GNN_SD_CASE(32, 2) GNN_SD_CASE(32, 4)
+#undef GNN_SD_CASE
+}
+
+static int64_t num_chunks(int64_t E) { return E > 0 ? ceil_div(E, PF_CHUNK) : 1; }
+
+struct PfWs {
+    int32_t* tail_row;
+    float* part_val;
+    int32_t* part_arg;
+    size_t bytes;
+};
+static PfWs pf_carve(void* ws, int64_t E, int F, bool with_arg) {
+    PfWs w;
+    int64_t nc = num_chunks(E);
+    char* p = (char*)ws;
+    size_t off = 0;
+    w.tail_row = (int32_t*)(p + off); off += up256((size_t)nc * 4);
+    w.part_val = (float*)(p + off); off += up256((size_t)nc * 2 * F * 4);
+    w.part_arg = (int32_t*)(p + off); if (with_arg) off += up256((size_t)nc * 2 * F * 4);
+    w.bytes = off;
+    return w;
+}
+
+size_t chunked_workspace(int64_t E, int F, bool with_arg) { return pf_carve(nullptr, E, F, with_arg).bytes; }
+
+gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const int64_t* rowptr,
+                       const int32_t* col, const float* w, const void* X, void* out,
+                       int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
+                       const int32_t* route_pos, int mean, int F, gnn_dtype dtype, void* ws,
+                       size_t ws_bytes, cudaStream_t st) {
+    const int s = elem_size(dtype);
+    GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED,
+                "%s: F*sizeof(element) = %d must be a multiple of 16 bytes", who, F * s);
+    const int nvec = F * s / 16;
+    int lpr, vpl;
+    GNN_REQUIRE(pick_shape(nvec, &lpr, &vpl), GNN_ERR_UNSUPPORTED,
+                "%s: feature rows wider than 2048 bytes are not supported (F=%d)", who, F);
+    GNN_REQUIRE(aligned16(X) && aligned16(out), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
+    const bool with_arg = (mode == MODE_MAX || mode == MODE_MIN);
+    PfWs wsv = pf_carve(ws, E, F, with_arg);
+    GNN_REQUIRE(ws && ws_bytes >= wsv.bytes && aligned16(ws), GNN_ERR_WORKSPACE_TOO_SMALL,
+                "%s: workspace of %zu bytes (16-byte aligned) needed, %zu given", who, wsv.bytes, ws_bytes);
+    if (N == 0) return GNN_OK;
+    PropParams P;
+    P.rowptr = rowptr; P.col = col; P.w = w; P.X = X; P.out = out; P.argmax = argmax;
+    P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
+    P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.nchunks = num_chunks(E);
+    P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
+    P.pol_keep = 0; P.pol_stream = 0;
+    if (dtype == GNN_F32) launch_mode<float>(P, mode, lpr, vpl, st);
+    else launch_mode<__nv_bfloat16>(P, mode, lpr, vpl, st);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+}  // namespace gnn
+
+using namespace gnn;
+
+extern "C" {
+
+size_t gnn_propagate_fused_workspace(int64_t E, int F, gnn_op op) {
+    if (E < 0 || F <= 0) return 0;
+    // MAX/MIN keep winner positions beside the partial values; their backward needs values
+    // only, so the forward size always suffices for the backward call
+    return chunked_workspace(E, F, op == GNN_MAX || op == GNN_MIN);
+}
+
+gnn_status gnn_propagate_fused(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* X,
+                               const float* w_csr, int F, gnn_dtype dtype, void* out,
+                               int32_t* argmax, void* ws, size_t ws_bytes, gnn_stream stream) {
+    GNN_REQUIRE(g && g->rowptr && X && out, GNN_ERR_INVALID_ARG, "gnn_propagate_fused: null argument");
+    GNN_REQUIRE(g->E == 0 || g->col, GNN_ERR_INVALID_ARG, "gnn_propagate_fused: null col");
+    GNN_REQUIRE(msg == GNN_MSG_COPY_XJ || msg == GNN_MSG_E_MUL_XJ, GNN_ERR_UNSUPPORTED,
+                "gnn_propagate_fused: message must be COPY_XJ or E_MUL_XJ");
+    GNN_REQUIRE(msg == GNN_MSG_COPY_XJ || w_csr, GNN_ERR_INVALID_ARG, "gnn_propagate_fused: E_MUL_XJ needs w_csr");
+    GNN_REQUIRE(dtype == GNN_F32 || dtype == GNN_BF16, GNN_ERR_INVALID_ARG, "gnn_propagate_fused: bad dtype");
+    GNN_REQUIRE(op >= GNN_SUM && op <= GNN_MIN, GNN_ERR_INVALID_ARG, "gnn_propagate_fused: bad op");
+    GNN_REQUIRE(!argmax || aligned16(argmax), GNN_ERR_INVALID_ARG, "gnn_propagate_fused: argmax must be 16-byte aligned");
+    const float* w = (msg == GNN_MSG_E_MUL_XJ) ? w_csr : nullptr;
+    const int mode = op == GNN_MAX ? MODE_MAX : op == GNN_MIN ? MODE_MIN : MODE_SUM;
+    return run_chunked("gnn_propagate_fused", mode, g->N, g->E, g->rowptr, g->col, w, X, out,
+                       argmax, nullptr, nullptr, nullptr, op == GNN_MEAN, F, dtype, ws, ws_bytes,
+                       as_stream(stream));
+}
+
+gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op,
+                                        const void* dOut, const void* X, const float* w_csrT,
+                                        const int32_t* argmax, int F, gnn_dtype dtype, void* dX,
+                                        float* dW, void* ws, size_t ws_bytes, gnn_stream stream) {
+    const char* who = "gnn_propagate_fused_backward";
+    GNN_REQUIRE(g && g->rowptr && g->rowptrT && dOut, GNN_ERR_INVALID_ARG, "%s: null argument", who);
+    GNN_REQUIRE(g->E == 0 || (g->col && g->colT), GNN_ERR_INVALID_ARG, "%s: null col", who);
+    GNN_REQUIRE(msg == GNN_MSG_COPY_XJ || msg == GNN_MSG_E_MUL_XJ, GNN_ERR_UNSUPPORTED,
+                "%s: message must be COPY_XJ or E_MUL_XJ", who);
+    GNN_REQUIRE(dtype == GNN_F32 || dtype == GNN_BF16, GNN_ERR_INVALID_ARG, "%s: bad dtype", who);
+    GNN_REQUIRE(op >= GNN_SUM && op <= GNN_MIN, GNN_ERR_INVALID_ARG, "%s: bad op", who);
+    const bool mm = (op == GNN_MAX || op == GNN_MIN);
+    cudaStream_t st = as_stream(stream);
+    if (dX) {
+        GNN_REQUIRE(msg == GNN_MSG_COPY_XJ || w_csrT, GNN_ERR_INVALID_ARG, "%s: E_MUL_XJ needs w_csrT for dX", who);
+        const float* w = (msg == GNN_MSG_E_MUL_XJ) ? w_csrT : nullptr;
+        gnn_status rc;
+        if (mm) {
+            GNN_REQUIRE(argmax && (g->E == 0 || g->t2f) && aligned16(argmax), GNN_ERR_INVALID_ARG,
+                        "%s: MAX/MIN need the forward argmax (16-byte aligned) and t2f", who);
+            rc = run_chunked(who, MODE_ROUTE, g->N, g->E, g->rowptrT, g->colT, w, dOut, dX, nullptr,
+                             nullptr, argmax, g->t2f, 0, F, dtype, ws, ws_bytes, st);
+        } else {
+            rc = run_chunked(who, MODE_SUM, g->N, g->E, g->rowptrT, g->colT, w, dOut, dX, nullptr,
+                             op == GNN_MEAN ? g->rowptr : nullptr, nullptr, nullptr, 0, F, dtype, ws,
+                             ws_bytes, st);
+        }
+        if (rc != GNN_OK) return rc;
+    }
+    if (dW) {
+        GNN_REQUIRE(!mm, GNN_ERR_UNSUPPORTED, "%s: dW is defined for SUM/MEAN only", who);
+        GNN_REQUIRE(X, GNN_ERR_INVALID_ARG, "%s: dW needs X", who);
+        const int s = elem_size(dtype);
+        GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED, "%s: F*sizeof(element) must be a multiple of 16 bytes", who);
+        int lpr, vpl;
+        GNN_REQUIRE(pick_shape(F * s / 16, &lpr, &vpl), GNN_ERR_UNSUPPORTED, "%s: feature rows wider than 2048 bytes", who);
+        GNN_REQUIRE(aligned16(X) && aligned16(dOut), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
+        if (g->E > 0) {
+            SddmmParams S;
+            S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW;
+            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_chunks(g->E);
+            if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
+            else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
+            GNN_CHECK_LAUNCH(who);
+        }
+    }
+    return GNN_OK;
+}
+
+}  // extern "C"

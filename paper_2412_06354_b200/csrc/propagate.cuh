@@ -1,0 +1,24 @@
+// Declarations shared by the kernels that reduce gathered rows over fixed edge chunks.
+#pragma once
+#include "common.cuh"
+
+namespace gnn {
+
+constexpr int PF_CHUNK = 256;  // edges per warp
+constexpr int PF_WARPS = 8;    // warps per block
+
+enum { MODE_SUM = 0, MODE_MAX = 1, MODE_MIN = 2, MODE_ROUTE = 3 };
+
+// lanes per row (4..32) and 16-byte vectors per lane (1, 2, 4) for rows of nvec 16-byte chunks
+bool pick_shape(int nvec, int* lpr, int* vpl);
+
+size_t chunked_workspace(int64_t E, int F, bool with_arg);
+
+// out[r,:] = reduce over positions p of row r of  w[p] * X[col[p],:]   (see propagate.cu)
+gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const int64_t* rowptr,
+                       const int32_t* col, const float* w, const void* X, void* out,
+                       int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
+                       const int32_t* route_pos, int mean, int F, gnn_dtype dtype, void* ws,
+                       size_t ws_bytes, cudaStream_t st);
+
+}  // namespace gnn
