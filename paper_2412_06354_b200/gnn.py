@@ -1,0 +1,205 @@
+"""ctypes binding of libgnn_b200.so: argument marshalling only.
+
+Every function here has the name of the C entry point without the ``gnn_`` prefix, takes torch
+CUDA tensors (torch is used for device memory and streams, nothing else), allocates outputs and
+workspaces when they are not passed in, and raises ``GnnError`` on a non-zero status.  There is no
+CPU path: loading fails if the CUDA library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgnn_b200.so")
+_lib = None
+
+SUM, MEAN, MAX, MIN = 0, 1, 2, 3
+COPY_XJ, E_MUL_XJ, GAT_LOGIT = 0, 1, 2
+F32, BF16 = 0, 1
+OPS = {"sum": SUM, "mean": MEAN, "max": MAX, "min": MIN}
+STATUS_NAMES = ["OK", "INVALID_ARG", "INDEX_OUT_OF_RANGE", "NOT_SORTED", "WORKSPACE_TOO_SMALL", "UNSUPPORTED", "CUDA", "TIMEOUT"]
+
+
+class GnnError(RuntimeError):
+    def __init__(self, status, msg):
+        super().__init__(f"gnn status {status} ({STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else '?'}): {msg}")
+        self.status = status
+
+
+class CsrStruct(C.Structure):
+    _fields_ = [("N", C.c_int32), ("E", C.c_int64), ("rowptr", C.c_void_p), ("col", C.c_void_p), ("eid", C.c_void_p),
+                ("rowptrT", C.c_void_p), ("colT", C.c_void_p), ("eidT", C.c_void_p), ("t2f", C.c_void_p)]
+
+
+_VP, _I32, _I64, _INT, _SZ, _F = C.c_void_p, C.c_int32, C.c_int64, C.c_int, C.c_size_t, C.c_float
+_CSR = C.POINTER(CsrStruct)
+
+# name -> (restype, argtypes); mirrors include/gnn.h
+SIGNATURES = {
+    "gnn_status_string": (C.c_char_p, [_INT]),
+    "gnn_last_error_string": (C.c_char_p, []),
+    "gnn_version": (_INT, []),
+    "gnn_coo_to_csr_workspace": (_SZ, [_I32, _I64]),
+    "gnn_coo_to_csr": (_INT, [_I32, _I64, _VP, _VP, _CSR, _VP, _SZ, _VP]),
+    "gnn_degree": (_INT, [_CSR, _INT, _VP, _VP, _VP]),
+    "gnn_add_self_loops": (_INT, [_I32, _I64, _VP, _VP, _VP, _VP, _VP]),
+    "gnn_gcn_norm": (_INT, [_CSR, _VP, _VP, _VP, _VP, _VP]),
+    "gnn_permute_edge_data": (_INT, [_VP, _I64, _INT, _INT, _VP, _VP, _VP]),
+    "gnn_propagate_fused_workspace": (_SZ, [_I64, _INT, _INT]),
+    "gnn_propagate_fused": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_fused_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+}
+
+
+def load(path: str = LIB_PATH):
+    """Load the CUDA library (no GPU needed to load it) and set the prototypes."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with `python -m paper_2412_06354_b200.build` "
+                              "(there is no CPU fallback)")
+        lib = C.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _check(rc):
+    if rc != 0:
+        raise GnnError(rc, load().gnn_last_error_string().decode())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _p(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _dtype(t):
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported feature dtype {t.dtype}")
+
+
+def _op(op):
+    return OPS[op] if isinstance(op, str) else int(op)
+
+
+def _dev(t):
+    assert t.is_cuda and t.is_contiguous(), "CUDA contiguous tensor expected"
+    return t
+
+
+class Graph:
+    """Both sparse forms of a graph on the device (see gnn_csr in gnn.h)."""
+
+    def __init__(self, N, E, device):
+        i64 = dict(dtype=torch.int64, device=device)
+        i32 = dict(dtype=torch.int32, device=device)
+        self.N, self.E = int(N), int(E)
+        self.rowptr = torch.empty(N + 1, **i64)
+        self.rowptrT = torch.empty(N + 1, **i64)
+        n = max(self.E, 1)
+        self.col, self.eid, self.colT, self.eidT, self.t2f = (torch.empty(n, **i32) for _ in range(5))
+        self.c = CsrStruct(self.N, self.E, *(t.data_ptr() for t in (self.rowptr, self.col, self.eid, self.rowptrT, self.colT, self.eidT, self.t2f)))
+
+    @property
+    def ref(self):
+        return C.byref(self.c)
+
+    def nbytes(self):
+        return sum(t.numel() * t.element_size() for t in (self.rowptr, self.col, self.eid, self.rowptrT, self.colT, self.eidT, self.t2f))
+
+
+# ------------------------------------------------------------------ graph set-up
+def coo_to_csr(N, src, dst, ws=None) -> Graph:
+    src, dst = _dev(src), _dev(dst)
+    E = src.numel()
+    g = Graph(N, E, src.device)
+    need = load().gnn_coo_to_csr_workspace(N, E)
+    if ws is None:
+        ws = torch.empty(need, dtype=torch.uint8, device=src.device)
+    _check(load().gnn_coo_to_csr(N, E, _p(src), _p(dst), g.ref, _p(ws), ws.numel(), _stream()))
+    return g
+
+
+def degree(g: Graph, transposed=False, w=None):
+    out = torch.empty(g.N, dtype=torch.int32 if w is None else torch.float32, device=g.rowptr.device)
+    _check(load().gnn_degree(g.ref, int(transposed), _p(w), _p(out), _stream()))
+    return out
+
+
+def add_self_loops(N, src, dst):
+    E = src.numel()
+    so = torch.empty(E + N, dtype=torch.int32, device=src.device)
+    do = torch.empty(E + N, dtype=torch.int32, device=src.device)
+    _check(load().gnn_add_self_loops(N, E, _p(src), _p(dst), _p(so), _p(do), _stream()))
+    return so, do
+
+
+def gcn_norm(g: Graph, w_csr=None, want_T=True):
+    dev = g.rowptr.device
+    deg = torch.empty(g.N, dtype=torch.float32, device=dev)
+    coef = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev)
+    coefT = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev) if want_T else None
+    _check(load().gnn_gcn_norm(g.ref, _p(w_csr), _p(deg), _p(coef), _p(coefT), _stream()))
+    return deg, coef[:g.E], (coefT[:g.E] if want_T else None)
+
+
+def permute_edge_data(perm, x, out=None):
+    x = _dev(x)
+    E = perm.numel()
+    width = x.numel() // max(E, 1) if E else 1
+    if out is None:
+        out = torch.empty_like(x)
+    _check(load().gnn_permute_edge_data(_p(perm), E, max(width, 1), x.element_size(), _p(x), _p(out), _stream()))
+    return out
+
+
+# ------------------------------------------------------------------ fused propagate
+def propagate_fused_workspace(E, F, op="sum"):
+    return load().gnn_propagate_fused_workspace(E, F, _op(op))
+
+
+def propagate_fused(g: Graph, X, w_csr=None, op="sum", out=None, argmax=None, ws=None):
+    """-> out, or (out, argmax) for max/min."""
+    X = _dev(X)
+    F = X.shape[1]
+    opc = _op(op)
+    if out is None:
+        out = torch.empty((g.N, F), dtype=X.dtype, device=X.device)
+    if opc in (MAX, MIN) and argmax is None:
+        argmax = torch.empty((g.N, F), dtype=torch.int32, device=X.device)
+    if ws is None:
+        ws = torch.empty(propagate_fused_workspace(g.E, F, opc), dtype=torch.uint8, device=X.device)
+    msg = COPY_XJ if w_csr is None else E_MUL_XJ
+    _check(load().gnn_propagate_fused(g.ref, msg, opc, _p(X), _p(w_csr), F, _dtype(X), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    return (out, argmax) if opc in (MAX, MIN) else out
+
+
+def propagate_fused_backward(g: Graph, dOut, op="sum", X=None, w_csrT=None, argmax=None, want_dX=True, want_dW=False,
+                             dX=None, dW=None, ws=None):
+    """-> (dX or None, dW or None)."""
+    dOut = _dev(dOut)
+    F = dOut.shape[1]
+    opc = _op(op)
+    if want_dX and dX is None:
+        dX = torch.empty((g.N, F), dtype=dOut.dtype, device=dOut.device)
+    if want_dW and dW is None:
+        dW = torch.empty(max(g.E, 1), dtype=torch.float32, device=dOut.device)
+    if ws is None:
+        ws = torch.empty(propagate_fused_workspace(g.E, F, opc), dtype=torch.uint8, device=dOut.device)
+    msg = COPY_XJ if (w_csrT is None) else E_MUL_XJ
+    _check(load().gnn_propagate_fused_backward(g.ref, msg, opc, _p(dOut), _p(X), _p(w_csrT), _p(argmax), F, _dtype(dOut),
+                                               _p(dX if want_dX else None), _p(dW if want_dW else None), _p(ws), ws.numel(), _stream()))
+    return (dX if want_dX else None), (dW[:g.E] if want_dW else None)
