@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark: fused propagate forward + backward on the large power-law graph.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--cases 128:bf16,...] [--impl reference]
+
+One step = the whole aggregation sweep on a seeded R-MAT graph (N = 2.4 M nodes, E = 123 M
+directed edges, randomly relabelled, sorted by target): for every feature width F in
+{32, 64, 128, 256, 512} x {bf16, f32} and for both fused messages (copy_xj+sum, e_mul_xj+sum),
+one gnn_propagate_fused and one gnn_propagate_fused_backward (dX).  The metric is
+edges*features per second: sum over the cases of E*F, divided by the time of the step.
+
+Prints ONE JSON line (rank 0).  `value` is measured with every input resident in HBM; `e2e`
+repeats the step through the *_host entry points with pinned host buffers, copying the features
+and the incoming gradient to the device and the two results back inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "propagate fwd+bwd edges*feat/s"
+UNIT = "edges*feat/s"
+ALL_CASES = [(F, dt) for dt in ("bf16", "f32") for F in (32, 64, 128, 256, 512)]
+FMAX = 512
+
+
+def parse_cases(s):
+    if not s or s == "sweep":
+        return ALL_CASES
+    out = []
+    for tok in s.split(","):
+        f, dt = tok.split(":")
+        out.append((int(f), dt))
+    return out
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier pool measurement, MEASURED_PEAKS.json absent)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def compulsory_bytes(N, E, F, s, weighted):
+    """Every array touched once: index (+weight) stream, row pointers, X read once, out written once."""
+    return 4 * E + (4 * E if weighted else 0) + 8 * N + 2 * N * F * s
+
+
+def gather_bytes(N, E, F, s, weighted):
+    """No reuse at all: every edge fetches its source row."""
+    return 4 * E + (4 * E if weighted else 0) + 8 * N + (E + N) * F * s
+
+
+# ----------------------------------------------------------------------------- reference arm
+def run_reference(args, rank):
+    """The CPU checker, as it stands, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2412_06354_b200 import synth
+    cores = len(os.sched_getaffinity(0))
+    oracle.set_threads(cores)
+    sample = cpu_sample(synth)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t = cpu_step(oracle, sample)
+        if i >= args.warmup:
+            times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    val = sample["E"] * sample["F"] / (ms * 1e-3)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD_NAME},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample["desc"]},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+WORKLOAD_NAME = "large sparse aggregation sweep: R-MAT N=2.4M E=123M (a=.57 b=.19 c=.19, symmetrised, relabelled, sorted by dst), F in {32,64,128,256,512} x {bf16,f32}, copy_xj+sum and e_mul_xj+sum, fwd + bwd dX"
+
+
+def cpu_sample(synth, pairs=1_000_000, F=128):
+    """A smaller graph of the same family for the CPU checker: R-MAT with the same parameters and
+    the same mean degree (N=39,024, 2,000,000 directed edges), bf16 features of width 128."""
+    n = 2_400_000 * (2 * pairs) // 123_000_000
+    src, dst = synth.rmat(16, n, pairs, synth.BASE_SEED + 5, symmetric=True, relabel=True, sort_by_dst=True)
+    return dict(N=n, E=len(src), F=F, src=src, dst=dst, X=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 20),
+                R=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 21), w=synth.uniform_f32((len(src),), 0, 1, synth.BASE_SEED + 5, 13),
+                desc=f"same generator at N={n}, E={2 * pairs} (same mean degree), F={F} bf16, e_mul_xj+sum fwd + bwd dX, fp64")
+
+
+def cpu_step(oracle, s):
+    t0 = time.perf_counter()
+    oracle.propagate("sum", s["N"], s["src"], s["dst"], s["X"], s["w"])
+    oracle.propagate_backward("sum", s["N"], s["src"], s["dst"], s["X"], s["w"], s["R"])
+    return time.perf_counter() - t0
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200")
+    ap.add_argument("--cases", default="sweep")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        return run_reference(args, rank)
+    assert args.warmup >= 3 or os.environ.get("GNN_BENCH_ALLOW_SHORT"), "use at least 3 warm-up steps"
+
+    import torch
+    from paper_2412_06354_b200 import build, gnn, synth
+    build.build()
+    gnn.load()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cases = parse_cases(args.cases)
+    fmax = max(F for F, _ in cases)
+    # ---- inputs (host, seeded) -> device
+    wl = synth.workload_large_graph()
+    N, E, seed = wl["N"], len(wl["src"]), wl["seed"]
+    src_d, dst_d = torch.from_numpy(wl["src"]).to(dev), torch.from_numpy(wl["dst"]).to(dev)
+    g = gnn.coo_to_csr(N, src_d, dst_d)
+    del src_d, dst_d
+    w_csr = gnn.permute_edge_data(g.eid, torch.from_numpy(wl["w"]).to(dev))
+    w_csrT = gnn.permute_edge_data(g.t2f, w_csr)
+    hX = torch.from_numpy(synth.normal_f32((N * fmax,), seed, 20))
+    hR = torch.from_numpy(synth.normal_f32((N * fmax,), seed, 21))
+    X32, R32 = hX.to(dev), hR.to(dev)
+    Xb, Rb = X32.to(torch.bfloat16), R32.to(torch.bfloat16)  # RNE, same bits as the host bf16 generator
+    out32 = torch.empty(N * fmax, dtype=torch.float32, device=dev)
+    dX32 = torch.empty(N * fmax, dtype=torch.float32, device=dev)
+    ws = torch.empty(gnn.propagate_fused_workspace(E, fmax, "sum"), dtype=torch.uint8, device=dev)
+    torch.cuda.empty_cache()
+
+    def views(F, dt):
+        n = N * F
+        if dt == "f32":
+            return X32[:n].view(N, F), R32[:n].view(N, F), out32[:n].view(N, F), dX32[:n].view(N, F)
+        return (Xb[:n].view(N, F), Rb[:n].view(N, F), out32.view(torch.bfloat16)[:n].view(N, F),
+                dX32.view(torch.bfloat16)[:n].view(N, F))
+
+    plan = []  # (F, dt, weighted, tensors)
+    for F, dt in cases:
+        for weighted in (False, True):
+            plan.append((F, dt, weighted, views(F, dt)))
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        for i, (F, dt, weighted, (X, R, out, dX)) in enumerate(plan):
+            if events is not None:
+                events[i][0].record(stream)
+            gnn.propagate_fused(g, X, w_csr if weighted else None, "sum", out=out, ws=ws)
+            if events is not None:
+                events[i][1].record(stream)
+            gnn.propagate_fused_backward(g, R, "sum", w_csrT=w_csrT if weighted else None, dX=dX, ws=ws)
+            if events is not None:
+                events[i][2].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in plan] for _ in range(args.steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    t0.record(stream)
+    for k in range(args.steps):
+        step(ev[k])
+    t1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    work = sum(E * F for F, _, _, _ in plan)  # edges*features per step (each fwd+bwd pair counted once)
+    value = world * work / (ms_per_step * 1e-3)
+
+    # ---- per-case breakdown and the roofline of the chunked propagate kernel
+    peak, peak_src = measured_peak()
+    per_case, tot_ms, tot_comp, tot_gath = [], 0.0, 0.0, 0.0
+    for i, (F, dt, weighted, _) in enumerate(plan):
+        s = 2 if dt == "bf16" else 4
+        f_ms = statistics.mean(ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps))
+        b_ms = statistics.mean(ev[k][i][1].elapsed_time(ev[k][i][2]) for k in range(args.steps))
+        comp, gath = compulsory_bytes(N, E, F, s, weighted), gather_bytes(N, E, F, s, weighted)
+        tot_ms += f_ms + b_ms
+        tot_comp += 2 * comp
+        tot_gath += 2 * gath
+        per_case.append({"F": F, "dtype": dt, "msg": "e_mul_xj" if weighted else "copy_xj", "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
+                         "edges_feat_per_s": E * F / ((f_ms + b_ms) * 1e-3), "compulsory_GBs_fwd": comp / f_ms / 1e6,
+                         "gather_GBs_fwd": gath / f_ms / 1e6, "compulsory_frac_fwd": comp / f_ms / 1e6 / peak})
+    launches = 2 * len(plan)  # gnn_propagate_fused + _backward calls per step; each is 2 kernels
+    achieved = tot_comp / tot_ms / 1e6
+    roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel (+ fixup), all launches of the step",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "peak_source": peak_src, "bytes_model": "compulsory: 4E(+4E weights)+8N+2*N*F*s per launch",
+                "bytes_per_launch_avg": tot_comp / (2 * len(plan)), "ms_per_launch_avg": tot_ms / (2 * len(plan)),
+                "gather_upper_bound_GBs": tot_gath / tot_ms / 1e6}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32 accumulate (bf16 and f32 storage)", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAME, "N": N, "E": E, "cases": [f"{F}:{dt}" for F, dt in cases],
+                       "l2": "inputs larger than L2: every launch streams >= 0.5 GB of indices and a feature matrix of 154 MB to 4.9 GB",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "gpu_launches": 4 * len(plan) * args.steps, "roofline": roofline, "per_case": per_case}
+
+    # ---- end to end through the host-buffer entry points
+    if not args.no_e2e and hasattr(gnn, "propagate_fused_host"):
+        line["e2e"] = run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, dev, world, barrier)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        cores = len(os.sched_getaffinity(0))
+        oracle.set_threads(cores)
+        sample = cpu_sample(synth)
+        cpu_step(oracle, sample)
+        t = min(cpu_step(oracle, sample) for _ in range(2))
+        line["cpu_baseline"] = {"value": sample["E"] * sample["F"] / t, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample["desc"]}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, dev, world, barrier):
+    """Same step, but features and incoming gradients start in pinned host memory and both results
+    end in pinned host memory, every case, inside the timed region.  The graph and the edge
+    weights stay resident (they do not change from step to step in full-graph training)."""
+    pin = dict(pin_memory=True)
+    hXp, hRp = hX.pin_memory(), hR.pin_memory()
+    hXb, hRb = hX.to(torch.bfloat16).pin_memory(), hR.to(torch.bfloat16).pin_memory()
+    hout = torch.empty(N * fmax, dtype=torch.float32, **pin)
+    hdX = torch.empty(N * fmax, dtype=torch.float32, **pin)
+    stage = [torch.empty(N * fmax, dtype=torch.float32, device=dev) for _ in range(2)]
+    h2d = d2h = 0
+    calls = []
+    for F, dt, weighted, _ in plan:
+        n = N * F
+        if dt == "f32":
+            hx, hr, ho, hd = hXp[:n].view(N, F), hRp[:n].view(N, F), hout[:n].view(N, F), hdX[:n].view(N, F)
+            sx, so = stage[0][:n].view(N, F), stage[1][:n].view(N, F)
+        else:
+            hx, hr = hXb[:n].view(N, F), hRb[:n].view(N, F)
+            ho, hd = hout.view(torch.bfloat16)[:n].view(N, F), hdX.view(torch.bfloat16)[:n].view(N, F)
+            sx, so = stage[0].view(torch.bfloat16)[:n].view(N, F), stage[1].view(torch.bfloat16)[:n].view(N, F)
+        calls.append((hx, hr, ho, hd, sx, so, weighted))
+        h2d += 2 * hx.numel() * hx.element_size()
+        d2h += 2 * ho.numel() * ho.element_size()
+
+    def step():
+        for hx, hr, ho, hd, sx, so, weighted in calls:
+            gnn.propagate_fused_host(g, hx, w_csr if weighted else None, "sum", ho, sx, so, ws)
+            gnn.propagate_fused_backward_host(g, hr, "sum", w_csrT if weighted else None, hd, sx, so, ws)
+
+    step()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record(torch.cuda.current_stream())
+    for _ in range(args.e2e_steps):
+        step()
+    t1.record(torch.cuda.current_stream())
+    barrier()
+    ms = t0.elapsed_time(t1) / args.e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    work = sum(E * F for F, _, _, _ in plan)
+    return {"value": world * work / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": args.e2e_steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "note": "features and gradients copied from pinned host memory, results copied back, per case; graph and edge weights resident"}
+
+
+if __name__ == "__main__":
+    main()

@@ -147,6 +147,24 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
                                         const int32_t* argmax, int F, gnn_dtype dtype, void* dX,
                                         float* dW, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* Host-buffer variants for callers whose features live in host memory (one call = copy in,
+ * compute, copy out; no counterpart in the paper beyond its "transfer the batch to the gpu"
+ * step in the training example).  h_X / h_dOut and h_out / h_dX are HOST arrays [N,F] (pinned
+ * memory makes the copies asynchronous); d_in and d_out are device staging buffers of N*F*s
+ * bytes each; the graph, the weights, argmax and ws are device memory as above.  The calls
+ * enqueue host->device copy, kernels and device->host copy on the stream and return without
+ * synchronising: the host arrays must stay valid, and h_out / h_dX are complete, only once the
+ * stream has been synchronised.  The backward variant computes dX only. */
+gnn_status gnn_propagate_fused_host(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* h_X,
+                                    const float* w_csr, int F, gnn_dtype dtype, void* h_out,
+                                    int32_t* argmax, void* d_in, void* d_out, void* ws,
+                                    size_t ws_bytes, gnn_stream stream);
+gnn_status gnn_propagate_fused_backward_host(const gnn_csr* g, gnn_msg msg, gnn_op op,
+                                             const void* h_dOut, const float* w_csrT,
+                                             const int32_t* argmax, int F, gnn_dtype dtype,
+                                             void* h_dX, void* d_in, void* d_out, void* ws,
+                                             size_t ws_bytes, gnn_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

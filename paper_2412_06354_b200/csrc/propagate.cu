@@ -596,4 +596,45 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
     return GNN_OK;
 }
 
+static gnn_status copy_async(const char* who, void* dst, const void* src, size_t bytes,
+                             cudaMemcpyKind kind, cudaStream_t st) {
+    if (bytes == 0) return GNN_OK;
+    cudaError_t e = cudaMemcpyAsync(dst, src, bytes, kind, st);
+    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: copy failed: %s", who, cudaGetErrorString(e));
+    return GNN_OK;
+}
+
+gnn_status gnn_propagate_fused_host(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* h_X,
+                                    const float* w_csr, int F, gnn_dtype dtype, void* h_out,
+                                    int32_t* argmax, void* d_in, void* d_out, void* ws,
+                                    size_t ws_bytes, gnn_stream stream) {
+    const char* who = "gnn_propagate_fused_host";
+    GNN_REQUIRE(g && h_X && h_out && d_in && d_out, GNN_ERR_INVALID_ARG, "%s: null argument", who);
+    GNN_REQUIRE(F > 0 && (dtype == GNN_F32 || dtype == GNN_BF16), GNN_ERR_INVALID_ARG, "%s: bad F or dtype", who);
+    const size_t bytes = (size_t)g->N * F * elem_size(dtype);
+    cudaStream_t st = as_stream(stream);
+    gnn_status rc = copy_async(who, d_in, h_X, bytes, cudaMemcpyHostToDevice, st);
+    if (rc != GNN_OK) return rc;
+    rc = gnn_propagate_fused(g, msg, op, d_in, w_csr, F, dtype, d_out, argmax, ws, ws_bytes, stream);
+    if (rc != GNN_OK) return rc;
+    return copy_async(who, h_out, d_out, bytes, cudaMemcpyDeviceToHost, st);
+}
+
+gnn_status gnn_propagate_fused_backward_host(const gnn_csr* g, gnn_msg msg, gnn_op op,
+                                             const void* h_dOut, const float* w_csrT,
+                                             const int32_t* argmax, int F, gnn_dtype dtype,
+                                             void* h_dX, void* d_in, void* d_out, void* ws,
+                                             size_t ws_bytes, gnn_stream stream) {
+    const char* who = "gnn_propagate_fused_backward_host";
+    GNN_REQUIRE(g && h_dOut && h_dX && d_in && d_out, GNN_ERR_INVALID_ARG, "%s: null argument", who);
+    GNN_REQUIRE(F > 0 && (dtype == GNN_F32 || dtype == GNN_BF16), GNN_ERR_INVALID_ARG, "%s: bad F or dtype", who);
+    const size_t bytes = (size_t)g->N * F * elem_size(dtype);
+    cudaStream_t st = as_stream(stream);
+    gnn_status rc = copy_async(who, d_in, h_dOut, bytes, cudaMemcpyHostToDevice, st);
+    if (rc != GNN_OK) return rc;
+    rc = gnn_propagate_fused_backward(g, msg, op, d_in, nullptr, w_csrT, argmax, F, dtype, d_out, nullptr, ws, ws_bytes, stream);
+    if (rc != GNN_OK) return rc;
+    return copy_async(who, h_dX, d_out, bytes, cudaMemcpyDeviceToHost, st);
+}
+
 }  // extern "C"

@@ -51,6 +51,8 @@ SIGNATURES = {
     "gnn_propagate_fused_workspace": (_SZ, [_I64, _INT, _INT]),
     "gnn_propagate_fused": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_fused_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_fused_backward_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _SZ, _VP]),
 }
 
 
@@ -203,3 +205,20 @@ def propagate_fused_backward(g: Graph, dOut, op="sum", X=None, w_csrT=None, argm
     _check(load().gnn_propagate_fused_backward(g.ref, msg, opc, _p(dOut), _p(X), _p(w_csrT), _p(argmax), F, _dtype(dOut),
                                                _p(dX if want_dX else None), _p(dW if want_dW else None), _p(ws), ws.numel(), _stream()))
     return (dX if want_dX else None), (dW[:g.E] if want_dW else None)
+
+
+def propagate_fused_host(g: Graph, h_X, w_csr, op, h_out, d_in, d_out, ws, argmax=None):
+    """Host-buffer forward: h_X, h_out are (pinned) host tensors; d_in, d_out device staging."""
+    F = h_X.shape[1]
+    msg = COPY_XJ if w_csr is None else E_MUL_XJ
+    _check(load().gnn_propagate_fused_host(g.ref, msg, _op(op), _p(h_X), _p(w_csr), F, _dtype(h_X), _p(h_out), _p(argmax),
+                                           _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
+    return h_out
+
+
+def propagate_fused_backward_host(g: Graph, h_dOut, op, w_csrT, h_dX, d_in, d_out, ws, argmax=None):
+    F = h_dOut.shape[1]
+    msg = COPY_XJ if w_csrT is None else E_MUL_XJ
+    _check(load().gnn_propagate_fused_backward_host(g.ref, msg, _op(op), _p(h_dOut), _p(w_csrT), _p(argmax), F, _dtype(h_dOut),
+                                                    _p(h_dX), _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
+    return h_dX
