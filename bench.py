@@ -159,6 +159,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--graph-scale", type=int, default=22,
+                    help="R-MAT scale; 22 is the full workload, smaller values shrink N and E by powers of two (profiling captures)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -181,7 +183,9 @@ def main():
     cases = parse_cases(args.cases)
     fmax = max(F for F, _ in cases)
     # ---- inputs (host, seeded) -> device
-    wl = synth.workload_large_graph()
+    shrink = 22 - args.graph_scale
+    assert 0 <= shrink <= 10
+    wl = synth.workload_large_graph(n=2_400_000 >> shrink, scale=args.graph_scale, pairs=61_500_000 >> shrink)
     N, E, seed = wl["N"], len(wl["src"]), wl["seed"]
     src_d, dst_d = torch.from_numpy(wl["src"]).to(dev), torch.from_numpy(wl["dst"]).to(dev)
     g = gnn.coo_to_csr(N, src_d, dst_d)
@@ -273,7 +277,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32 accumulate (bf16 and f32 storage)", "data": "synthetic",
-            "config": {"workload": WORKLOAD_NAME, "N": N, "E": E, "cases": [f"{F}:{dt}" for F, dt in cases],
+            "config": {"workload": WORKLOAD_NAME if shrink == 0 else f"REDUCED graph (R-MAT scale {args.graph_scale}) of: " + WORKLOAD_NAME, "N": N, "E": E, "cases": [f"{F}:{dt}" for F, dt in cases],
                        "l2": "inputs larger than L2: every launch streams >= 0.5 GB of indices and a feature matrix of 154 MB to 4.9 GB",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "gpu_launches": 4 * len(plan) * args.steps, "roofline": roofline, "per_case": per_case}

@@ -147,6 +147,80 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
                                         const int32_t* argmax, int F, gnn_dtype dtype, void* dX,
                                         float* dW, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* ------------------------------------------------------------------ unfused primitives ------ */
+
+/* gather (Sec. 3 "Message Passing"): out[k,:] = X[idx[k],:] for k < E; idx = the source vector
+ * gives x_j per edge, the target vector gives x_i.  Indices must lie in [0,N) (the vectors that
+ * gnn_coo_to_csr accepted do).  A bit-exact copy. */
+gnn_status gnn_gather(const int32_t* idx, int64_t E, const void* X, int32_t N, int F,
+                      gnn_dtype dtype, void* out, gnn_stream stream);
+
+/* Backward of gather = scatter-add, run as a segmented sum: dX[n,:] = sum of dOut[k,:] over the
+ * edges k with dst[k] == n (by_src == 0) or src[k] == n (by_src != 0).  dOut_EF is [E,F] in the
+ * ORIGINAL COO edge order (rows are found through eid / eidT).  ws as for gnn_propagate_fused
+ * with op SUM. */
+gnn_status gnn_gather_backward(const gnn_csr* g, int by_src, const void* dOut_EF, int F,
+                               gnn_dtype dtype, void* dX, void* ws, size_t ws_bytes,
+                               gnn_stream stream);
+
+/* apply_edges (Sec. 3 "Message Passing"): one message per edge, written in CSR order.
+ *   COPY_XJ    m[p,:] = X[col[p],:]
+ *   E_MUL_XJ   m[p,f] = e[p, f / (F / e_width)] * X[col[p], f]; e is float [E, e_width] in CSR
+ *              order, e_width = 1 (one scalar per edge), H (one per head) or F (element-wise)
+ *   GAT_LOGIT  m[p,h] = LeakyReLU_slope(al[col[p],h] + ar[i,h]) for p in row i; here
+ *              X_or_al = al and ar are float [N,F] with F = number of heads, dtype must be F32
+ * The message function set is fixed; arbitrary closures cannot cross a C ABI. */
+gnn_status gnn_apply_edges(const gnn_csr* g, gnn_msg msg, const void* X_or_al, const void* ar,
+                           const float* e, int e_width, int F, gnn_dtype dtype, float slope,
+                           void* m_out, gnn_stream stream);
+
+/* aggregate_neighbors (Sec. 3 "Message Passing"): out[i,:] = op over p in row i of m[p,:], with
+ * m [E,F] in CSR order; ops, empty rows, argmax and ws as for gnn_propagate_fused. */
+gnn_status gnn_aggregate(const gnn_csr* g, gnn_op op, const void* m_EF, int F, gnn_dtype dtype,
+                         void* out, int32_t* argmax, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Backward of aggregate w.r.t. the messages (CSR order): SUM dm[p,:] = dOut[i,:]; MEAN divided
+ * by the in-degree of i; MAX/MIN dm[p,f] = dOut[i,f] if argmax[i,f] == p else 0. */
+gnn_status gnn_aggregate_backward(const gnn_csr* g, gnn_op op, const void* dOut_NF,
+                                  const int32_t* argmax, int F, gnn_dtype dtype, void* dm_EF,
+                                  gnn_stream stream);
+
+/* ------------------------------------------------------------------ edge softmax ------------ */
+
+/* Attention normalisation of the GAT layer (Sec. 3 "Graph Convolutional Layers"): for every node
+ * i and head h, over the incoming edges p of i:
+ *   alpha[p,h] = exp(s[p,h] - max_i) / sum_p' exp(s[p',h] - max_i)
+ * logits_EH, alpha_EH: [E,H] of dtype in CSR order; math in fp32.  rowmax, rowsum: optional
+ * float [N,H] (0 for nodes without incoming edges). */
+gnn_status gnn_edge_softmax(const gnn_csr* g, const void* logits_EH, int H, gnn_dtype dtype,
+                            void* alpha_EH, float* rowmax, float* rowsum, gnn_stream stream);
+
+/* dLogits[p,h] = alpha[p,h] * (dAlpha[p,h] - sum over the row of alpha*dAlpha) */
+gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, const void* dAlpha_EH,
+                                     int H, gnn_dtype dtype, void* dLogits_EH, gnn_stream stream);
+
+/* ------------------------------------------------------------------ batched-graph pooling --- */
+
+/* A batch of graphs is one block-diagonal graph whose nodes are numbered graph by graph
+ * (Sec. 3 "Graph Data Structures": batching).  graph_id: int32 [N], non-decreasing, in [0,G).
+ * graph_ptr: int64 [G+1], node range of graph g = graph_ptr[g] .. graph_ptr[g+1]-1.
+ * Returns GNN_ERR_NOT_SORTED if the ids are not sorted or out of range (one stream
+ * synchronisation to read the flag; ws: at least 4 bytes of device scratch). */
+gnn_status gnn_graph_ptr_from_ids(const int32_t* graph_id, int32_t N, int32_t G, int64_t* graph_ptr,
+                                  void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Global pooling (GlobalPool in the training example): out[g,:] = op over the nodes of graph g
+ * of X[n,:]; an empty graph gives 0; MAX/MIN: argmax int32 [G,F] = winning node id (first node
+ * among equals), -1 if none.  ws: gnn_propagate_fused_workspace(N, F, op) bytes. */
+gnn_status gnn_reduce_nodes(const int64_t* graph_ptr, int32_t G, int32_t N, gnn_op op, const void* X,
+                            int F, gnn_dtype dtype, void* out_GF, int32_t* argmax, void* ws,
+                            size_t ws_bytes, gnn_stream stream);
+
+/* dX[n,:] = dOut[g(n),:] (SUM), / n_g (MEAN), or routed to the argmax node only (MAX/MIN) */
+gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_t N, gnn_op op,
+                                     const void* dOut_GF, const int32_t* argmax, int F,
+                                     gnn_dtype dtype, void* dX_NF, gnn_stream stream);
+
 /* Host-buffer variants for callers whose features live in host memory (one call = copy in,
  * compute, copy out; no counterpart in the paper beyond its "transfer the batch to the gpu"
  * step in the training example).  h_X / h_dOut and h_out / h_dX are HOST arrays [N,F] (pinned

@@ -17,7 +17,8 @@ OBJ = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libgnn_b200.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-         "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
+         "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC,
+         *os.environ.get("GNN_NVCC_FLAGS", "").split()]
 
 
 def _newest(paths):
@@ -44,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 if r.returncode != 0:
                     raise RuntimeError("nvcc failed: " + " ".join(r.args))
     if jobs or not os.path.exists(LIB):
-        subprocess.check_call([NVCC, "-shared", "-o", LIB, *objs, "-lcuda"])
+        subprocess.check_call([NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB, *objs])
     from . import synth
     synth.build(force)
     return LIB

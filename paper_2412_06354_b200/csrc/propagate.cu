@@ -2,7 +2,7 @@
 // generalised sparse x dense product) and its backward passes.
 //
 // Work decomposition: the E positions of the sparse form are cut into fixed chunks of PF_CHUNK
-// consecutive edges, one warp per chunk (merge-path style: perfect balance on power-law rows
+// consecutive edges (256 or 1024), one warp per chunk (merge-path style: perfect balance on power-law rows
 // without any per-graph schedule).  A warp finds its first row by binary search in rowptr and
 // walks the rows that start inside its chunk.  Rows lying wholly inside the chunk are reduced
 // and written directly.  A row cut by a chunk boundary leaves fp32 partials (one "head" slot and
@@ -15,11 +15,21 @@
 // edges, and are combined by an xor-shuffle tree at the end of each row.
 #include "propagate.cuh"
 
+#ifndef PF_U_NARROW
+#define PF_U_NARROW 4
+#endif
+#ifndef PF_U_WIDE
+#define PF_U_WIDE 8
+#endif
+#ifndef PF_MIN_BLOCKS
+#define PF_MIN_BLOCKS 3
+#endif
+
 namespace gnn {
 
 struct PropParams {
     const int64_t* rowptr;  // rows of the output
-    const int32_t* col;     // gathered row of X per position
+    const int32_t* col;     // gathered row of X per position (nullptr: position p gathers row p)
     const float* w;         // per-position multiplier or nullptr
     const void* X;          // gathered matrix [N,F]
     void* out;              // [N,F]
@@ -33,12 +43,20 @@ struct PropParams {
     int nvec;  // 16-byte chunks per feature row
     int F;
     int mean;  // divide the finished row by max(1, row length)
+    int chunk;  // edges per warp, a multiple of PF_SLAB
     int64_t nchunks;
     int32_t* tail_row;  // [nchunks] row whose tail partial lives in slot 1, or -1
     float* part_val;    // [nchunks][2][F]
     int32_t* part_arg;  // [nchunks][2][F] (MODE_MAX/MIN)
-    uint64_t pol_keep, pol_stream;  // L2 policies, filled in on the device
 };
+
+// d.xy += w.xy * x.xy as one packed fp32x2 FMA (each half is an IEEE fused multiply-add)
+__device__ __forceinline__ void fma2(float& a0, float& a1, float x0, float x1, float w0, float w1) {
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mov.b64 rc, {%0, %1};\n\tfma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+        : "+f"(a0), "+f"(a1)
+        : "f"(x0), "f"(x1), "f"(w0), "f"(w1));
+}
 
 template <typename T, int VPL, int MODE>
 struct Acc {
@@ -66,95 +84,112 @@ __device__ __forceinline__ bool beats(float cv, int32_t ca, float v, int32_t a) 
     return better || (cv == v && ca < a);
 }
 
+// per-warp staging area for one slab of PF_SLAB consecutive positions:
+// (gathered row, forward position [MODE_ROUTE], multiplier, multiplier) -- the multiplier is
+// stored twice so that one 16-byte shared load yields the register pair the packed FMA wants
+struct SlabSmem {
+    int4 e[PF_SLAB];
+};
+
 template <typename T, int LPR, int VPL, int MODE>
 struct Walker {
     static constexpr int EPC = Chunk<T>::N;
     static constexpr int NG = 32 / LPR;
-    static constexpr int U = (LPR >= 16) ? (8 / VPL) : 4;
+    static constexpr int U = (LPR >= 16) ? (PF_U_WIDE / VPL) : PF_U_NARROW;
     static constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
     using A = Acc<T, VPL, MODE>;
 
-    // accumulate positions [a, b) of one row into acc (this lane group's share)
-    __device__ __forceinline__ static void segment(const PropParams& P, int64_t a, int64_t b,
-                                                   int lane, A& acc) {
+    // copy indices and multipliers of positions [sb, se) into shared memory (one round trip)
+    __device__ __forceinline__ static void stage(const PropParams& P, int64_t sb, int64_t se, int lane,
+                                                 SlabSmem& S, uint64_t pol_stream) {
+        __syncwarp();
+        for (int i = lane; i < (int)(se - sb); i += 32) {
+            int c = P.col ? ld_hint_i32(P.col + sb + i, pol_stream) : (int)(sb + i);  // no col: row p of X
+            float w = P.w ? ld_hint_f32(P.w + sb + i, pol_stream) : 1.0f;
+            if (P.gscale_rowptr) {
+                int64_t d = P.gscale_rowptr[c + 1] - P.gscale_rowptr[c];
+                w = w / (float)(d > 1 ? d : 1);
+            }
+            int t = (MODE == MODE_ROUTE) ? ld_hint_i32(P.route_pos + sb + i, pol_stream) : 0;
+            S.e[i] = make_int4(c, t, __float_as_int(w), __float_as_int(w));
+        }
+        __syncwarp();
+    }
+
+    // one gathered row chunk -> accumulator
+    __device__ __forceinline__ static void consume(const PropParams& P, const int4& e, const uint4* buf,
+                                                   int32_t pos, int lane_chunk0, A& acc) {
+        const float w0 = __int_as_float(e.z), w1 = __int_as_float(e.w);
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            float x[EPC];
+            Chunk<T>::unpack(buf[v], x);
+            if (MODE == MODE_SUM) {
+#pragma unroll
+                for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], w0, w1);
+            } else if (ARG) {
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) {
+                    float m = P.w ? w0 * x[j] : x[j];
+                    // positions arrive in ascending order within a group: strict comparison
+                    // keeps the first of equal values
+                    bool take = acc.a[ARG ? v : 0][j] < 0 ||
+                                (MODE == MODE_MAX ? m > acc.v[v][j] : m < acc.v[v][j]);
+                    if (take) { acc.v[v][j] = m; acc.a[ARG ? v : 0][j] = pos; }
+                }
+            } else {  // MODE_ROUTE: keep dOut only where this edge was the winner
+                const int32_t* ap = P.route_arg + (size_t)e.x * P.F + (size_t)(v * LPR + lane_chunk0) * EPC;
+                int32_t win[EPC];
+#pragma unroll
+                for (int j = 0; j < EPC; j += 4) {
+                    int4 t = *reinterpret_cast<const int4*>(ap + j);
+                    win[j] = t.x; win[j + 1] = t.y; win[j + 2] = t.z; win[j + 3] = t.w;
+                }
+#pragma unroll
+                for (int j = 0; j < EPC; ++j)
+                    if (win[j] == e.y) acc.v[v][j] = fmaf(w0, x[j], acc.v[v][j]);
+            }
+        }
+    }
+
+    // accumulate staged positions [p0, e1) (all inside the slab starting at sb) into acc.
+    // Lanes beyond the row width (rows that do not fill LPR*VPL chunks) read chunk 0 instead:
+    // always in bounds, never written back, so the loop needs no lane masking.
+    __device__ __forceinline__ static void slab_segment(const PropParams& P, int64_t sb, int64_t p0, int64_t e1,
+                                                        int lane, const SlabSmem& S, uint64_t pol_keep, A& acc) {
         const int g = lane / LPR, li = lane % LPR;
-        const char* Xb = reinterpret_cast<const char*>(P.X);
-        const size_t row_bytes = (size_t)P.nvec * 16;
-        for (int64_t base = a; base < b; base += 32) {
-            const int n = (int)((b - base) < 32 ? (b - base) : 32);
-            int myc = 0;
-            float myw = 1.f;
-            int myt = 0;
-            if (lane < n) {
-                myc = ld_hint_i32(P.col + base + lane, P.pol_stream);
-                if (P.w) myw = ld_hint_f32(P.w + base + lane, P.pol_stream);
-                if (P.gscale_rowptr) {
-                    int64_t d = P.gscale_rowptr[myc + 1] - P.gscale_rowptr[myc];
-                    myw = myw / (float)(d > 1 ? d : 1);
-                }
-                if (MODE == MODE_ROUTE) myt = ld_hint_i32(P.route_pos + base + lane, P.pol_stream);
-            }
-            const int rounds = (n + NG - 1) / NG;
-            for (int r0 = 0; r0 < rounds; r0 += U) {
-                uint4 buf[U][VPL];
-                float wv[U];
-                int tv[U];
-                int cv[U];
-                bool ok[U];
+        const uint32_t row_bytes = (uint32_t)P.nvec * 16;
+        const char* Xl[VPL];
+        int c0[VPL];
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int e = (r0 + u) * NG + g;
-                    ok[u] = e < n;
-                    cv[u] = __shfl_sync(0xffffffffu, myc, e & 31);
-                    wv[u] = __shfl_sync(0xffffffffu, myw, e & 31);
-                    tv[u] = (MODE == MODE_ROUTE) ? __shfl_sync(0xffffffffu, myt, e & 31) : 0;
-                    if (ok[u]) {
-                        const char* rp = Xb + (size_t)cv[u] * row_bytes;
+        for (int v = 0; v < VPL; ++v) {
+            c0[v] = (v * LPR + li < P.nvec) ? v * LPR + li : 0;
+            Xl[v] = reinterpret_cast<const char*>(P.X) + (size_t)c0[v] * 16;
+        }
+        const int lane_chunk0 = (li < P.nvec) ? li : 0;  // VPL > 1 only with full rows of 32 lanes
+        const int i1 = (int)(e1 - sb);
+        int i = (int)(p0 - sb) + g;
+        // full groups of U positions per lane group: no predicates
+        for (; i + (U - 1) * NG < i1; i += NG * U) {
+            int4 e[U];
+            uint4 buf[U][VPL];
 #pragma unroll
-                        for (int v = 0; v < VPL; ++v) {
-                            const int ci = v * LPR + li;
-                            if (ci < P.nvec) buf[u][v] = ld_hint16(rp + (size_t)ci * 16, P.pol_keep);
-                        }
-                    }
-                }
+            for (int u = 0; u < U; ++u) e[u] = S.e[i + u * NG];
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (!ok[u]) continue;
-                    const int32_t pos = (int32_t)(base + (r0 + u) * NG + g);
+            for (int u = 0; u < U; ++u)
 #pragma unroll
-                    for (int v = 0; v < VPL; ++v) {
-                        const int ci = v * LPR + li;
-                        if (ci >= P.nvec) continue;
-                        float x[EPC];
-                        Chunk<T>::unpack(buf[u][v], x);
-                        if (MODE == MODE_SUM) {
+                for (int v = 0; v < VPL; ++v)
+                    buf[u][v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e[u].x * row_bytes, pol_keep);
 #pragma unroll
-                            for (int j = 0; j < EPC; ++j) acc.v[v][j] = fmaf(wv[u], x[j], acc.v[v][j]);
-                        } else if (ARG) {
+            for (int u = 0; u < U; ++u) consume(P, e[u], buf[u], (int32_t)(sb + i + u * NG), lane_chunk0, acc);
+        }
+        // remainder: fewer than U positions for this lane group
+        for (; i < i1; i += NG) {
+            const int4 e = S.e[i];
+            uint4 buf[VPL];
 #pragma unroll
-                            for (int j = 0; j < EPC; ++j) {
-                                float m = P.w ? wv[u] * x[j] : x[j];
-                                // positions arrive in ascending order within a group: strict
-                                // comparison keeps the first of equal values
-                                bool take = acc.a[ARG ? v : 0][j] < 0 ||
-                                            (MODE == MODE_MAX ? m > acc.v[v][j] : m < acc.v[v][j]);
-                                if (take) { acc.v[v][j] = m; acc.a[ARG ? v : 0][j] = pos; }
-                            }
-                        } else {  // MODE_ROUTE: keep dOut only where this edge was the winner
-                            const int32_t* ap = P.route_arg + (size_t)cv[u] * P.F + (size_t)ci * EPC;
-                            int32_t win[EPC];
-#pragma unroll
-                            for (int j = 0; j < EPC; j += 4) {
-                                int4 t = *reinterpret_cast<const int4*>(ap + j);
-                                win[j] = t.x; win[j + 1] = t.y; win[j + 2] = t.z; win[j + 3] = t.w;
-                            }
-#pragma unroll
-                            for (int j = 0; j < EPC; ++j)
-                                if (win[j] == tv[u]) acc.v[v][j] = fmaf(wv[u], x[j], acc.v[v][j]);
-                        }
-                    }
-                }
-            }
+            for (int v = 0; v < VPL; ++v) buf[v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e.x * row_bytes, pol_keep);
+            consume(P, e, buf, (int32_t)(sb + i), lane_chunk0, acc);
         }
     }
 
@@ -232,43 +267,53 @@ struct Walker {
 };
 
 template <typename T, int LPR, int VPL, int MODE>
-__global__ void __launch_bounds__(PF_WARPS * 32)
-propagate_chunk_kernel(const PropParams P0) {
-    PropParams P = P0;
-    P.pol_keep = policy_evict_last();
-    P.pol_stream = policy_evict_first();
+__global__ void __launch_bounds__(PF_WARPS * 32, (VPL == 1 && MODE == MODE_SUM) ? PF_MIN_BLOCKS : 2)
+propagate_chunk_kernel(const PropParams P) {
     using W = Walker<T, LPR, VPL, MODE>;
-    const int lane = threadIdx.x & 31;
-    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + (threadIdx.x >> 5);
+    __shared__ SlabSmem s_slab[PF_WARPS];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + wib;
     if (c >= P.nchunks) return;
-    const int64_t cs = c * PF_CHUNK;
-    const int64_t ce = (cs + PF_CHUNK < P.E) ? cs + PF_CHUNK : P.E;
+    SlabSmem& S = s_slab[wib];
+    const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
+    const int64_t cs = c * P.chunk;
+    const int64_t ce = (cs + P.chunk < P.E) ? cs + P.chunk : P.E;
     const bool last = (c == P.nchunks - 1);
-    typename W::A acc;
 
-    int r = lower_bound_i64(P.rowptr, P.N + 1, cs);  // first row starting at or after cs
-    int64_t rs = P.rowptr[r];
-    if (rs > cs) {  // the row before it started earlier and reaches into this chunk: head partial
-        acc.clear();
-        W::segment(P, cs, rs < ce ? rs : ce, lane, acc);
-        W::combine_groups(acc, lane);
-        W::write_partial(P, c, 0, lane, acc);
-    }
+    // cur = the row containing position cs, or the first (possibly empty) row starting at cs
+    int cur = lower_bound_i64(P.rowptr, P.N + 1, cs);
+    if (P.rowptr[cur] > cs) --cur;
+    int64_t pos = cs;
+    int64_t sb = cs - PF_SLAB;  // nothing staged yet
     int32_t tail = -1;
-    for (; r < P.N; ++r) {
-        if (!(rs < ce || last)) break;
-        const int64_t re = P.rowptr[r + 1];
+    typename W::A acc;
+    while (cur < P.N) {
+        const int64_t rs = P.rowptr[cur], re = P.rowptr[cur + 1];
+        const int64_t b = re < ce ? re : ce;
         acc.clear();
-        W::segment(P, rs, re < ce ? re : ce, lane, acc);
-        W::combine_groups(acc, lane);
-        if (re <= ce) {
-            W::write_final(P, r, re - rs, lane, acc);
-        } else {
-            W::write_partial(P, c, 1, lane, acc);
-            tail = r;
+        const int64_t pos0 = pos;
+        while (pos < b) {
+            if (pos >= sb + PF_SLAB) {
+                sb = cs + ((pos - cs) / PF_SLAB) * PF_SLAB;
+                W::stage(P, sb, (sb + PF_SLAB < ce) ? sb + PF_SLAB : ce, lane, S, pol_stream);
+            }
+            const int64_t e = (b < sb + PF_SLAB) ? b : sb + PF_SLAB;
+            W::slab_segment(P, sb, pos, e, lane, S, pol_keep, acc);
+            pos = e;
+        }
+        // with at most one position only lane group 0 holds data: nothing to combine
+        if (b - (pos0) > 1) W::combine_groups(acc, lane);
+        const bool started_here = rs >= cs;
+        if (re <= ce) {  // the row ends inside this chunk
+            if (started_here) W::write_final(P, cur, re - rs, lane, acc);
+            else W::write_partial(P, c, 0, lane, acc);
+            ++cur;
+            if (!(re < ce || last)) break;  // the next row starts in the next chunk
+        } else {  // the row continues in the next chunk
+            W::write_partial(P, c, started_here ? 1 : 0, lane, acc);
+            if (started_here) tail = cur;
             break;
         }
-        rs = re;
     }
     if (lane == 0) P.tail_row[c] = tail;
 }
@@ -285,7 +330,7 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
     const int32_t r = P.tail_row[c];
     if (r < 0) return;
     const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
-    const int64_t c_end = (re - 1) / PF_CHUNK;
+    const int64_t c_end = (re - 1) / P.chunk;
     float v[EPC];
     int32_t a[EPC];
     const size_t F = P.F;
@@ -350,8 +395,8 @@ sddmm_chunk_kernel(const SddmmParams P) {
     const int lane = threadIdx.x & 31, g = lane / LPR, li = lane % LPR;
     const int64_t c = (int64_t)blockIdx.x * PF_WARPS + (threadIdx.x >> 5);
     if (c >= P.nchunks) return;
-    const int64_t cs = c * PF_CHUNK;
-    const int64_t ce = (cs + PF_CHUNK < P.E) ? cs + PF_CHUNK : P.E;
+    const int64_t cs = c * PF_SLAB;
+    const int64_t ce = (cs + PF_SLAB < P.E) ? cs + PF_SLAB : P.E;
     if (cs >= ce) return;
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
     const size_t row_bytes = (size_t)P.nvec * 16;
@@ -464,7 +509,11 @@ static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st
 #undef GNN_SD_CASE
 }
 
-static int64_t num_chunks(int64_t E) { return E > 0 ? ceil_div(E, PF_CHUNK) : 1; }
+// edges per warp: one slab on small graphs (more warps), four slabs once there are enough
+// edges to fill the machine many times over (fewer partial rows to write and re-read)
+static int chunk_edges(int64_t E) { return E >= (int64_t)8 * 1024 * 1024 ? 4 * PF_SLAB : PF_SLAB; }
+static int64_t num_chunks(int64_t E) { return E > 0 ? ceil_div(E, chunk_edges(E)) : 1; }
+static int64_t num_slabs(int64_t E) { return E > 0 ? ceil_div(E, PF_SLAB) : 1; }
 
 struct PfWs {
     int32_t* tail_row;
@@ -507,9 +556,8 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     PropParams P;
     P.rowptr = rowptr; P.col = col; P.w = w; P.X = X; P.out = out; P.argmax = argmax;
     P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
-    P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.nchunks = num_chunks(E);
+    P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
-    P.pol_keep = 0; P.pol_stream = 0;
     if (dtype == GNN_F32) launch_mode<float>(P, mode, lpr, vpl, st);
     else launch_mode<__nv_bfloat16>(P, mode, lpr, vpl, st);
     GNN_CHECK_LAUNCH(who);
@@ -587,7 +635,7 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
         if (g->E > 0) {
             SddmmParams S;
             S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW;
-            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_chunks(g->E);
+            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_slabs(g->E);
             if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
             else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
             GNN_CHECK_LAUNCH(who);

@@ -4,7 +4,7 @@
 
 namespace gnn {
 
-constexpr int PF_CHUNK = 256;  // edges per warp
+constexpr int PF_SLAB = 256;   // positions staged in shared memory at a time
 constexpr int PF_WARPS = 8;    // warps per block
 
 enum { MODE_SUM = 0, MODE_MAX = 1, MODE_MIN = 2, MODE_ROUTE = 3 };

@@ -51,6 +51,16 @@ SIGNATURES = {
     "gnn_propagate_fused_workspace": (_SZ, [_I64, _INT, _INT]),
     "gnn_propagate_fused": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_gather": (_INT, [_VP, _I64, _VP, _I32, _INT, _INT, _VP, _VP]),
+    "gnn_gather_backward": (_INT, [_CSR, _INT, _VP, _INT, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_apply_edges": (_INT, [_CSR, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP]),
+    "gnn_aggregate": (_INT, [_CSR, _INT, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_aggregate_backward": (_INT, [_CSR, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
+    "gnn_edge_softmax": (_INT, [_CSR, _VP, _INT, _INT, _VP, _VP, _VP, _VP]),
+    "gnn_edge_softmax_backward": (_INT, [_CSR, _VP, _VP, _INT, _INT, _VP, _VP]),
+    "gnn_graph_ptr_from_ids": (_INT, [_VP, _I32, _I32, _VP, _VP, _SZ, _VP]),
+    "gnn_reduce_nodes": (_INT, [_VP, _I32, _I32, _INT, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_reduce_nodes_backward": (_INT, [_VP, _I32, _I32, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
     "gnn_propagate_fused_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _SZ, _VP]),
 }
@@ -222,3 +232,103 @@ def propagate_fused_backward_host(g: Graph, h_dOut, op, w_csrT, h_dX, d_in, d_ou
     _check(load().gnn_propagate_fused_backward_host(g.ref, msg, _op(op), _p(h_dOut), _p(w_csrT), _p(argmax), F, _dtype(h_dOut),
                                                     _p(h_dX), _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
     return h_dX
+
+
+# ------------------------------------------------------------------ unfused primitives
+def _ws(E, F, op, device, ws):
+    if ws is None:
+        ws = torch.empty(propagate_fused_workspace(E, F, op), dtype=torch.uint8, device=device)
+    return ws
+
+
+def gather(idx, X, out=None):
+    X = _dev(X)
+    E, F = idx.numel(), X.shape[1]
+    if out is None:
+        out = torch.empty((E, F), dtype=X.dtype, device=X.device)
+    _check(load().gnn_gather(_p(idx), E, _p(X), X.shape[0], F, _dtype(X), _p(out), _stream()))
+    return out
+
+
+def gather_backward(g: Graph, dOut_EF, by_src=False, ws=None):
+    dOut_EF = _dev(dOut_EF)
+    F = dOut_EF.shape[1]
+    dX = torch.empty((g.N, F), dtype=dOut_EF.dtype, device=dOut_EF.device)
+    ws = _ws(g.E, F, SUM, dOut_EF.device, ws)
+    _check(load().gnn_gather_backward(g.ref, int(by_src), _p(dOut_EF), F, _dtype(dOut_EF), _p(dX), _p(ws), ws.numel(), _stream()))
+    return dX
+
+
+def apply_edges(g: Graph, msg, X, ar=None, e=None, slope=0.2):
+    """COPY_XJ / E_MUL_XJ: X [N,F], e float32 [E] or [E,w] (CSR order) -> m [E,F] of X.dtype.
+    GAT_LOGIT: X = al, ar float32 [N,H] -> float32 [E,H]."""
+    X = _dev(X)
+    F = X.shape[1]
+    ew = 0 if e is None else (1 if e.dim() == 1 else e.shape[1])
+    m = torch.empty((max(g.E, 1), F), dtype=X.dtype, device=X.device)
+    _check(load().gnn_apply_edges(g.ref, msg, _p(X), _p(ar), _p(e), ew, F, _dtype(X), float(slope), _p(m), _stream()))
+    return m[:g.E]
+
+
+def aggregate(g: Graph, m_EF, op="sum", ws=None):
+    m_EF = _dev(m_EF)
+    F = m_EF.shape[1]
+    opc = _op(op)
+    out = torch.empty((g.N, F), dtype=m_EF.dtype, device=m_EF.device)
+    argmax = torch.empty((g.N, F), dtype=torch.int32, device=m_EF.device) if opc in (MAX, MIN) else None
+    ws = _ws(g.E, F, opc, m_EF.device, ws)
+    _check(load().gnn_aggregate(g.ref, opc, _p(m_EF), F, _dtype(m_EF), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    return (out, argmax) if opc in (MAX, MIN) else out
+
+
+def aggregate_backward(g: Graph, dOut, op="sum", argmax=None):
+    dOut = _dev(dOut)
+    F = dOut.shape[1]
+    dm = torch.empty((max(g.E, 1), F), dtype=dOut.dtype, device=dOut.device)
+    _check(load().gnn_aggregate_backward(g.ref, _op(op), _p(dOut), _p(argmax), F, _dtype(dOut), _p(dm), _stream()))
+    return dm[:g.E]
+
+
+def edge_softmax(g: Graph, logits, want_stats=False):
+    logits = _dev(logits)
+    H = logits.shape[1]
+    alpha = torch.empty_like(logits)
+    rmax = torch.empty((g.N, H), dtype=torch.float32, device=logits.device) if want_stats else None
+    rsum = torch.empty((g.N, H), dtype=torch.float32, device=logits.device) if want_stats else None
+    _check(load().gnn_edge_softmax(g.ref, _p(logits), H, _dtype(logits), _p(alpha), _p(rmax), _p(rsum), _stream()))
+    return (alpha, rmax, rsum) if want_stats else alpha
+
+
+def edge_softmax_backward(g: Graph, alpha, dalpha):
+    alpha, dalpha = _dev(alpha), _dev(dalpha)
+    ds = torch.empty_like(alpha)
+    _check(load().gnn_edge_softmax_backward(g.ref, _p(alpha), _p(dalpha), alpha.shape[1], _dtype(alpha), _p(ds), _stream()))
+    return ds
+
+
+# ------------------------------------------------------------------ pooling
+def graph_ptr_from_ids(graph_id, G):
+    N = graph_id.numel()
+    gptr = torch.empty(G + 1, dtype=torch.int64, device=graph_id.device)
+    ws = torch.empty(256, dtype=torch.uint8, device=graph_id.device)
+    _check(load().gnn_graph_ptr_from_ids(_p(graph_id), N, G, _p(gptr), _p(ws), ws.numel(), _stream()))
+    return gptr
+
+
+def reduce_nodes(graph_ptr, X, op="mean", ws=None):
+    X = _dev(X)
+    G, (N, F) = graph_ptr.numel() - 1, X.shape
+    opc = _op(op)
+    out = torch.empty((G, F), dtype=X.dtype, device=X.device)
+    argmax = torch.empty((G, F), dtype=torch.int32, device=X.device) if opc in (MAX, MIN) else None
+    ws = _ws(N, F, opc, X.device, ws)
+    _check(load().gnn_reduce_nodes(_p(graph_ptr), G, N, opc, _p(X), F, _dtype(X), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    return (out, argmax) if opc in (MAX, MIN) else out
+
+
+def reduce_nodes_backward(graph_ptr, dOut, N, op="mean", argmax=None):
+    dOut = _dev(dOut)
+    G, F = dOut.shape
+    dX = torch.empty((N, F), dtype=dOut.dtype, device=dOut.device)
+    _check(load().gnn_reduce_nodes_backward(_p(graph_ptr), G, N, _op(op), _p(dOut), _p(argmax), F, _dtype(dOut), _p(dX), _stream()))
+    return dX
