@@ -199,6 +199,30 @@ gnn_status gnn_edge_softmax(const gnn_csr* g, const void* logits_EH, int H, gnn_
 gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, const void* dAlpha_EH,
                                      int H, gnn_dtype dtype, void* dLogits_EH, gnn_stream stream);
 
+/* ------------------------------------------------------------------ fused GAT layer core ---- */
+
+/* GAT attention (Sec. 3 "Graph Convolutional Layers" names the layer) on an already transformed
+ * node tensor Wx [N,H,C] of dtype; a_src, a_dst float [H,C]:
+ *   al[n,h] = <a_src[h,:], Wx[n,h,:]>,  ar[n,h] = <a_dst[h,:], Wx[n,h,:]>
+ *   s[p,h]  = LeakyReLU_slope(al[col[p],h] + ar[i,h]),  alpha = edge softmax of s per row and head
+ *   out[i,h,:] = sum over p in row i of alpha[p,h] * Wx[col[p],h,:]      (heads concatenated)
+ * No self-loops are added; a node without incoming edges gets 0.  Saved for the backward call:
+ * alpha_csr float [E,H] (CSR order), al, ar float [N,H].  H must be a power of two <= 32 and
+ * C*sizeof(element) a multiple of 16 bytes.  The E x F message tensor is never formed.
+ * ws: gnn_gat_fused_workspace(N, E, H, C, backward) bytes. */
+size_t gnn_gat_fused_workspace(int32_t N, int64_t E, int H, int C, int backward);
+gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, const float* a_dst,
+                         int H, int C, gnn_dtype dtype, float slope, void* out, float* alpha_csr,
+                         float* al, float* ar, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Backward for dL/dout = dOut [N,H,C]: dWx [N,H,C] of dtype, da_src, da_dst float [H,C].
+ * alpha_csr, al, ar are the forward call's outputs.  The derivative of LeakyReLU at 0 is slope. */
+gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float* a_src,
+                                  const float* a_dst, const float* alpha_csr, const float* al,
+                                  const float* ar, const void* dOut, int H, int C, gnn_dtype dtype,
+                                  float slope, void* dWx, float* da_src, float* da_dst, void* ws,
+                                  size_t ws_bytes, gnn_stream stream);
+
 /* ------------------------------------------------------------------ batched-graph pooling --- */
 
 /* A batch of graphs is one block-diagonal graph whose nodes are numbered graph by graph

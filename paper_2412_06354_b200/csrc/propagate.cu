@@ -22,7 +22,7 @@
 #define PF_U_WIDE 8
 #endif
 #ifndef PF_MIN_BLOCKS
-#define PF_MIN_BLOCKS 3
+#define PF_MIN_BLOCKS 4
 #endif
 
 namespace gnn {
@@ -48,6 +48,11 @@ struct PropParams {
     int32_t* tail_row;  // [nchunks] row whose tail partial lives in slot 1, or -1
     float* part_val;    // [nchunks][2][F]
     int32_t* part_arg;  // [nchunks][2][F] (MODE_MAX/MIN)
+    // MODE_HEADSUM: multiplier per (position, head), features of head h = [h*fph, (h+1)*fph)
+    const float* wh;  // [E,H]
+    int H, fph;
+    // optional rank-1 epilogue: out[r,f] += epi_l[r,h(f)]*epi_a[f] + epi_r[r,h(f)]*epi_b[f]
+    const float *epi_l, *epi_r, *epi_a, *epi_b;
 };
 
 // d.xy += w.xy * x.xy as one packed fp32x2 FMA (each half is an IEEE fused multiply-add)
@@ -118,13 +123,16 @@ struct Walker {
 
     // one gathered row chunk -> accumulator
     __device__ __forceinline__ static void consume(const PropParams& P, const int4& e, const uint4* buf,
-                                                   int32_t pos, int lane_chunk0, A& acc) {
+                                                   const float* hw, int32_t pos, int lane_chunk0, A& acc) {
         const float w0 = __int_as_float(e.z), w1 = __int_as_float(e.w);
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
             float x[EPC];
             Chunk<T>::unpack(buf[v], x);
-            if (MODE == MODE_SUM) {
+            if (MODE == MODE_HEADSUM) {
+#pragma unroll
+                for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], hw[v], hw[v]);
+            } else if (MODE == MODE_SUM) {
 #pragma unroll
                 for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], w0, w1);
             } else if (ARG) {
@@ -167,29 +175,50 @@ struct Walker {
             Xl[v] = reinterpret_cast<const char*>(P.X) + (size_t)c0[v] * 16;
         }
         const int lane_chunk0 = (li < P.nvec) ? li : 0;  // VPL > 1 only with full rows of 32 lanes
+        const float* whl[VPL];  // MODE_HEADSUM: this lane's head column of the multiplier matrix
+#pragma unroll
+        for (int v = 0; v < VPL; ++v)
+            whl[v] = (MODE == MODE_HEADSUM) ? P.wh + (size_t)sb * P.H + (c0[v] * EPC) / P.fph : nullptr;
         const int i1 = (int)(e1 - sb);
         int i = (int)(p0 - sb) + g;
         // full groups of U positions per lane group: no predicates
         for (; i + (U - 1) * NG < i1; i += NG * U) {
             int4 e[U];
             uint4 buf[U][VPL];
+            float hw[U][VPL];
 #pragma unroll
             for (int u = 0; u < U; ++u) e[u] = S.e[i + u * NG];
 #pragma unroll
             for (int u = 0; u < U; ++u)
 #pragma unroll
-                for (int v = 0; v < VPL; ++v)
+                for (int v = 0; v < VPL; ++v) {
                     buf[u][v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e[u].x * row_bytes, pol_keep);
+                    hw[u][v] = (MODE == MODE_HEADSUM) ? __ldg(whl[v] + (size_t)(i + u * NG) * P.H) : 0.f;
+                }
 #pragma unroll
-            for (int u = 0; u < U; ++u) consume(P, e[u], buf[u], (int32_t)(sb + i + u * NG), lane_chunk0, acc);
+            for (int u = 0; u < U; ++u) consume(P, e[u], buf[u], hw[u], (int32_t)(sb + i + u * NG), lane_chunk0, acc);
         }
         // remainder: fewer than U positions for this lane group
         for (; i < i1; i += NG) {
             const int4 e = S.e[i];
             uint4 buf[VPL];
+            float hw[VPL];
 #pragma unroll
-            for (int v = 0; v < VPL; ++v) buf[v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e.x * row_bytes, pol_keep);
-            consume(P, e, buf, (int32_t)(sb + i), lane_chunk0, acc);
+            for (int v = 0; v < VPL; ++v) {
+                buf[v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e.x * row_bytes, pol_keep);
+                hw[v] = (MODE == MODE_HEADSUM) ? __ldg(whl[v] + (size_t)i * P.H) : 0.f;
+            }
+            consume(P, e, buf, hw, (int32_t)(sb + i), lane_chunk0, acc);
+        }
+    }
+
+    // optional rank-1 update of a finished row chunk (see PropParams::epi_*)
+    __device__ __forceinline__ static void epilogue(const PropParams& P, int64_t row, int ci, float* v) {
+        if (!P.epi_l) return;
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) {
+            const int f = ci * EPC + j, h = f / P.fph;
+            v[j] += P.epi_l[(size_t)row * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)row * P.H + h] * P.epi_b[f];
         }
     }
 
@@ -229,6 +258,7 @@ struct Walker {
 #pragma unroll
                 for (int j = 0; j < EPC; ++j) acc.v[v][j] = acc.v[v][j] / d;
             }
+            if (MODE == MODE_HEADSUM) epilogue(P, row, ci, acc.v[v]);
             st_stream16(ob + (size_t)ci * 16, Chunk<T>::pack(acc.v[v]));
             if (ARG && P.argmax) {
                 int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
@@ -267,7 +297,7 @@ struct Walker {
 };
 
 template <typename T, int LPR, int VPL, int MODE>
-__global__ void __launch_bounds__(PF_WARPS * 32, (VPL == 1 && MODE == MODE_SUM) ? PF_MIN_BLOCKS : 2)
+__global__ void __launch_bounds__(PF_WARPS * 32, (VPL == 1 && (MODE == MODE_SUM || MODE == MODE_HEADSUM)) ? PF_MIN_BLOCKS : 2)
 propagate_chunk_kernel(const PropParams P) {
     using W = Walker<T, LPR, VPL, MODE>;
     __shared__ SlabSmem s_slab[PF_WARPS];
@@ -361,6 +391,13 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
 #pragma unroll
         for (int j = 0; j < EPC; ++j) v[j] = v[j] / d;
     }
+    if (MODE == MODE_HEADSUM && P.epi_l) {
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) {
+            const int f = ci * EPC + j, h = f / P.fph;
+            v[j] += P.epi_l[(size_t)r * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)r * P.H + h] * P.epi_b[f];
+        }
+    }
     char* ob = reinterpret_cast<char*>(P.out) + ((size_t)r * P.nvec + ci) * 16;
     *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
     if (ARG && P.argmax) {
@@ -384,6 +421,7 @@ struct SddmmParams {
     int nvec;
     int mean;
     int64_t nchunks;
+    int H, lph;  // lph > 0: one result per (edge, head), a head = lph adjacent 16-byte chunks
 };
 
 template <typename T, int LPR, int VPL>
@@ -443,21 +481,35 @@ sddmm_chunk_kernel(const SddmmParams P) {
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    float dot = 0.f;
-                    if (ok[u]) {
+                    float dotv[VPL];
 #pragma unroll
-                        for (int v = 0; v < VPL; ++v) {
-                            const int ci = v * LPR + li;
-                            if (ci >= P.nvec) continue;
+                    for (int v = 0; v < VPL; ++v) {
+                        dotv[v] = 0.f;
+                        const int ci = v * LPR + li;
+                        if (ok[u] && ci < P.nvec) {
                             float x[EPC];
                             Chunk<T>::unpack(buf[u][v], x);
 #pragma unroll
-                            for (int j = 0; j < EPC; ++j) dot = fmaf(x[j], d[v][j], dot);
+                            for (int j = 0; j < EPC; ++j) dotv[v] = fmaf(x[j], d[v][j], dotv[v]);
                         }
                     }
+                    const int64_t p = base + (r0 + u) * NG + g;
+                    if (P.lph == 0) {  // one dot product per edge over the whole row
+                        float dot = dotv[0];
 #pragma unroll
-                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    if (ok[u] && li == 0) P.dW[base + (r0 + u) * NG + g] = scale * dot;
+                        for (int v = 1; v < VPL; ++v) dot += dotv[v];
+#pragma unroll
+                        for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                        if (ok[u] && li == 0) P.dW[p] = scale * dot;
+                    } else {  // one per (edge, head): a head covers lph adjacent lanes
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            float dot = dotv[v];
+                            for (int o = P.lph >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                            const int ci = v * LPR + li;
+                            if (ok[u] && ci < P.nvec && (li % P.lph) == 0) P.dW[p * P.H + ci / P.lph] = scale * dot;
+                        }
+                    }
                 }
             }
         }
@@ -495,6 +547,7 @@ static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStr
         case MODE_SUM: launch_chunks<T, MODE_SUM>(P, lpr, vpl, st); break;
         case MODE_MAX: launch_chunks<T, MODE_MAX>(P, lpr, vpl, st); break;
         case MODE_MIN: launch_chunks<T, MODE_MIN>(P, lpr, vpl, st); break;
+        case MODE_HEADSUM: launch_chunks<T, MODE_HEADSUM>(P, lpr, vpl, st); break;
         default: launch_chunks<T, MODE_ROUTE>(P, lpr, vpl, st); break;
     }
 }
@@ -539,7 +592,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
                        const int32_t* col, const float* w, const void* X, void* out,
                        int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
                        const int32_t* route_pos, int mean, int F, gnn_dtype dtype, void* ws,
-                       size_t ws_bytes, cudaStream_t st) {
+                       size_t ws_bytes, cudaStream_t st, const HeadExtra* hx) {
     const int s = elem_size(dtype);
     GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED,
                 "%s: F*sizeof(element) = %d must be a multiple of 16 bytes", who, F * s);
@@ -558,8 +611,41 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
     P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
+    P.wh = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
+    if (hx) {
+        const int epc = 16 / s;
+        GNN_REQUIRE(mode == MODE_HEADSUM && (hx->wh || E == 0) && hx->H >= 1 && F % hx->H == 0 && (F / hx->H) % epc == 0, GNN_ERR_UNSUPPORTED,
+                    "%s: per-head weights need F divisible by H and F/H a multiple of %d elements", who, epc);
+        P.wh = hx->wh; P.H = hx->H; P.fph = F / hx->H;
+        P.epi_l = hx->epi_l; P.epi_r = hx->epi_r; P.epi_a = hx->epi_a; P.epi_b = hx->epi_b;
+    } else {
+        GNN_REQUIRE(mode != MODE_HEADSUM, GNN_ERR_INVALID_ARG, "%s: per-head mode without weights", who);
+    }
     if (dtype == GNN_F32) launch_mode<float>(P, mode, lpr, vpl, st);
     else launch_mode<__nv_bfloat16>(P, mode, lpr, vpl, st);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+// dW[p,h] = <X[col[p],h,:], dOut[i,h,:]> for p in row i: the per-head edge dot products of the
+// attention backward pass
+gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const void* dOut, int H, int C,
+                       gnn_dtype dtype, float* dW_EH, cudaStream_t st) {
+    const int s = elem_size(dtype), F = H * C;
+    GNN_REQUIRE(((size_t)C * s) % 16 == 0, GNN_ERR_UNSUPPORTED, "%s: a head must be a multiple of 16 bytes wide", who);
+    const int lph = C * s / 16;
+    GNN_REQUIRE(lph <= 32 && (lph & (lph - 1)) == 0, GNN_ERR_UNSUPPORTED,
+                "%s: a head must span a power-of-two number (<= 32) of 16-byte chunks (C=%d)", who, C);
+    int lpr, vpl;
+    GNN_REQUIRE(pick_shape(F * s / 16, &lpr, &vpl), GNN_ERR_UNSUPPORTED, "%s: feature rows wider than 2048 bytes", who);
+    GNN_REQUIRE(lph <= lpr, GNN_ERR_UNSUPPORTED, "%s: head wider than the row layout", who);
+    GNN_REQUIRE(aligned16(X) && aligned16(dOut), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
+    if (g->E == 0) return GNN_OK;
+    SddmmParams S;
+    S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW_EH;
+    S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = 0; S.nchunks = num_slabs(g->E); S.H = H; S.lph = lph;
+    if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
+    else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
@@ -635,7 +721,7 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
         if (g->E > 0) {
             SddmmParams S;
             S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW;
-            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_slabs(g->E);
+            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_slabs(g->E); S.H = 1; S.lph = 0;
             if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
             else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
             GNN_CHECK_LAUNCH(who);

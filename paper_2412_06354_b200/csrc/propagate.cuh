@@ -7,7 +7,16 @@ namespace gnn {
 constexpr int PF_SLAB = 256;   // positions staged in shared memory at a time
 constexpr int PF_WARPS = 8;    // warps per block
 
-enum { MODE_SUM = 0, MODE_MAX = 1, MODE_MIN = 2, MODE_ROUTE = 3 };
+enum { MODE_SUM = 0, MODE_MAX = 1, MODE_MIN = 2, MODE_ROUTE = 3, MODE_HEADSUM = 4 };
+
+// MODE_HEADSUM extras: multipliers per (position, head) and an optional rank-1 row epilogue
+//   out[r,f] += epi_l[r,h(f)] * epi_a[f] + epi_r[r,h(f)] * epi_b[f]
+struct HeadExtra {
+    const float* wh;  // [E,H]
+    int H;
+    const float *epi_l, *epi_r;  // [rows,H] or nullptr
+    const float *epi_a, *epi_b;  // [F]
+};
 
 // lanes per row (4..32) and 16-byte vectors per lane (1, 2, 4) for rows of nvec 16-byte chunks
 bool pick_shape(int nvec, int* lpr, int* vpl);
@@ -19,6 +28,6 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
                        const int32_t* col, const float* w, const void* X, void* out,
                        int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
                        const int32_t* route_pos, int mean, int F, gnn_dtype dtype, void* ws,
-                       size_t ws_bytes, cudaStream_t st);
+                       size_t ws_bytes, cudaStream_t st, const HeadExtra* hx = nullptr);
 
 }  // namespace gnn

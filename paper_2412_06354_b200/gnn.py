@@ -58,6 +58,9 @@ SIGNATURES = {
     "gnn_aggregate_backward": (_INT, [_CSR, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
     "gnn_edge_softmax": (_INT, [_CSR, _VP, _INT, _INT, _VP, _VP, _VP, _VP]),
     "gnn_edge_softmax_backward": (_INT, [_CSR, _VP, _VP, _INT, _INT, _VP, _VP]),
+    "gnn_gat_fused_workspace": (_SZ, [_I32, _I64, _INT, _INT, _INT]),
+    "gnn_gat_fused": (_INT, [_CSR, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_gat_fused_backward": (_INT, [_CSR, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_graph_ptr_from_ids": (_INT, [_VP, _I32, _I32, _VP, _VP, _SZ, _VP]),
     "gnn_reduce_nodes": (_INT, [_VP, _I32, _I32, _INT, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_reduce_nodes_backward": (_INT, [_VP, _I32, _I32, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
@@ -332,3 +335,37 @@ def reduce_nodes_backward(graph_ptr, dOut, N, op="mean", argmax=None):
     dX = torch.empty((N, F), dtype=dOut.dtype, device=dOut.device)
     _check(load().gnn_reduce_nodes_backward(_p(graph_ptr), G, N, _op(op), _p(dOut), _p(argmax), F, _dtype(dOut), _p(dX), _stream()))
     return dX
+
+
+# ------------------------------------------------------------------ GAT
+def gat_fused(g: Graph, Wx, a_src, a_dst, H, slope=0.2, ws=None):
+    """Wx [N, H*C] -> dict(out, alpha (float32 [E,H], CSR order), al, ar (float32 [N,H]))."""
+    Wx = _dev(Wx)
+    N, F = Wx.shape
+    Cw = F // H
+    dev = Wx.device
+    out = torch.empty_like(Wx)
+    alpha = torch.empty((max(g.E, 1), H), dtype=torch.float32, device=dev)
+    al = torch.empty((N, H), dtype=torch.float32, device=dev)
+    ar = torch.empty((N, H), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = torch.empty(load().gnn_gat_fused_workspace(N, g.E, H, Cw, 0), dtype=torch.uint8, device=dev)
+    _check(load().gnn_gat_fused(g.ref, _p(Wx), _p(a_src), _p(a_dst), H, Cw, _dtype(Wx), float(slope), _p(out), _p(alpha),
+                                _p(al), _p(ar), _p(ws), ws.numel(), _stream()))
+    return dict(out=out, alpha=alpha[:g.E], al=al, ar=ar)
+
+
+def gat_fused_backward(g: Graph, Wx, a_src, a_dst, fwd, dOut, H, slope=0.2, ws=None):
+    Wx, dOut = _dev(Wx), _dev(dOut)
+    N, F = Wx.shape
+    Cw = F // H
+    dev = Wx.device
+    dWx = torch.empty_like(Wx)
+    da_src = torch.empty((H, Cw), dtype=torch.float32, device=dev)
+    da_dst = torch.empty((H, Cw), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = torch.empty(load().gnn_gat_fused_workspace(N, g.E, H, Cw, 1), dtype=torch.uint8, device=dev)
+    _check(load().gnn_gat_fused_backward(g.ref, _p(Wx), _p(a_src), _p(a_dst), _p(fwd["alpha"]), _p(fwd["al"]), _p(fwd["ar"]),
+                                         _p(dOut), H, Cw, _dtype(Wx), float(slope), _p(dWx), _p(da_src), _p(da_dst),
+                                         _p(ws), ws.numel(), _stream()))
+    return dict(dWx=dWx, da_src=da_src, da_dst=da_dst)

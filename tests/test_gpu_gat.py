@@ -1,0 +1,104 @@
+"""GPU parity: fused GAT core, forward and backward, against the CPU checker."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2412_06354_b200 import synth
+from util import assert_close, to_dev, to_host64
+from test_gpu_propagate import build_graph, ragged_graph
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gnn():
+    from paper_2412_06354_b200 import gnn as g
+    g.load()
+    return g
+
+
+def run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, what):
+    F = H * C
+    g = build_graph(gnn, n, src, dst)
+    eid = g.eid[:g.E].cpu().numpy() if g.E else np.zeros(0, np.int64)
+    fwd = gnn.gat_fused(g, to_dev(Wx), to_dev(a_s), to_dev(a_d), H)
+    ref = oracle.gat(n, src, dst, Wx, a_s, a_d, H, C)
+    x64 = synth.to_f64(Wx).reshape(n, H, C)
+    Sal = np.einsum("nhc,hc->nh", np.abs(x64), np.abs(a_s.astype(np.float64)))
+    Sar = np.einsum("nhc,hc->nh", np.abs(x64), np.abs(a_d.astype(np.float64)))
+    assert_close(to_host64(fwd["al"]), ref["al"], Sal, "f32", what + " al")
+    assert_close(to_host64(fwd["ar"]), ref["ar"], Sar, "f32", what + " ar")
+    if g.E:
+        # a coefficient moves by about (error of its logit) * alpha; the logit is a two-dot-product sum
+        scale = ref["alpha"][eid] * np.maximum(1.0, Sal[src[eid]] + Sar[dst[eid]])
+        assert_close(to_host64(fwd["alpha"]), ref["alpha"][eid], scale, "f32", what + " alpha")
+    assert_close(to_host64(fwd["out"]), ref["out"], ref["S"], dtype, what + " out")
+
+    R = synth.normal((n, F), dtype, 4242, 3)
+    bw = gnn.gat_fused_backward(g, to_dev(Wx), to_dev(a_s), to_dev(a_d), fwd, to_dev(R), H)
+    rb = oracle.gat_backward(n, src, dst, Wx, a_s, a_d, H, C, ref, R)
+    # LeakyReLU'(z) is decided by the sign of z; where |z| is below fp32 resolution of its terms the
+    # two precisions may decide differently, so nodes touching such an edge are left out
+    z = ref["al"][src] + ref["ar"][dst]
+    risky = np.abs(z) < 1e-5 * (Sal[src] + Sar[dst])
+    skip = np.zeros(n, bool)
+    skip[src[risky.any(axis=1)]] = True
+    skip[dst[risky.any(axis=1)]] = True
+    assert skip.mean() < 0.01
+    keep = ~skip
+    assert_close(to_host64(bw["dWx"])[keep], rb["dWx"][keep], rb["SdWx"][keep], dtype, what + " dWx")
+    if not skip.any():
+        assert_close(to_host64(bw["da_src"]), rb["da_src"], rb["Sda_src"], "f32", what + " da_src")
+        assert_close(to_host64(bw["da_dst"]), rb["da_dst"], rb["Sda_dst"], "f32", what + " da_dst")
+    else:  # the attention-vector gradients sum over every node: compare norm-wise only
+        for k in ("da_src", "da_dst"):
+            err = np.abs(to_host64(bw[k]) - rb[k]).max() / np.abs(rb[k]).max()
+            assert err < 1e-3, (k, err)
+    return g, fwd
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("H,C", [(4, 16), (8, 32), (1, 64), (2, 8)])
+def test_gat_ragged(gnn, dtype, H, C):
+    n, src, dst = ragged_graph(90 + H)
+    Wx = synth.normal((n, H * C), dtype, 900 + H, 1)
+    a = (6.0 / (C + 1)) ** 0.5
+    a_s = synth.uniform_f32((H, C), -a, a, 901, 1)
+    a_d = synth.uniform_f32((H, C), -a, a, 902, 1)
+    run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, f"gat H={H} C={C} {dtype}")
+
+
+def test_gat_zero_attention_is_mean_aggregation(gnn):
+    n, src, dst = ragged_graph(95)
+    H, C = 4, 16
+    Wx = synth.normal_f32((n, H * C), 950)
+    zero = np.zeros((H, C), np.float32)
+    g = build_graph(gnn, n, src, dst)
+    fwd = gnn.gat_fused(g, to_dev(Wx), to_dev(zero), to_dev(zero), H)
+    o, S, _ = oracle.propagate("mean", n, src, dst, Wx)
+    assert_close(to_host64(fwd["out"]), o, S, "f32", "alpha = 1/deg")
+
+
+def test_gat_degenerate(gnn):
+    import torch
+    H, C = 2, 8
+    a_s = to_dev(synth.normal_f32((H, C), 1))
+    g = build_graph(gnn, 4, np.zeros(0, np.int32), np.zeros(0, np.int32))
+    Wx = to_dev(synth.normal_f32((4, H * C), 2))
+    fwd = gnn.gat_fused(g, Wx, a_s, a_s, H)
+    assert torch.count_nonzero(fwd["out"]) == 0
+    bw = gnn.gat_fused_backward(g, Wx, a_s, a_s, fwd, Wx, H)
+    assert torch.count_nonzero(bw["dWx"]) == 0 and torch.count_nonzero(bw["da_src"]) == 0
+    with pytest.raises(gnn.GnnError) as e:  # three heads
+        gnn.gat_fused(g, to_dev(synth.normal_f32((4, 24), 3)), a_s, a_s, 3)
+    assert e.value.status == 5
+
+
+def test_gat_attention_workload_full_size(gnn):
+    """R-MAT N=100000, 1.6M directed edges, 8 heads x 32 features bf16."""
+    wl = synth.workload_attention()
+    oracle.set_threads(8)
+    try:
+        run_case(gnn, wl["N"], wl["src"], wl["dst"], wl["Wx"], wl["a_src"], wl["a_dst"], wl["H"], wl["C"], "bf16", "attention workload")
+    finally:
+        oracle.set_threads(1)
