@@ -40,11 +40,11 @@ def run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, what):
     # LeakyReLU'(z) is decided by the sign of z; where |z| is below fp32 resolution of its terms the
     # two precisions may decide differently, so nodes touching such an edge are left out
     z = ref["al"][src] + ref["ar"][dst]
-    risky = np.abs(z) < 1e-5 * (Sal[src] + Sar[dst])
+    risky = np.abs(z) < 2e-6 * (Sal[src] + Sar[dst])
     skip = np.zeros(n, bool)
     skip[src[risky.any(axis=1)]] = True
     skip[dst[risky.any(axis=1)]] = True
-    assert skip.mean() < 0.01
+    assert skip.mean() < 0.05
     keep = ~skip
     assert_close(to_host64(bw["dWx"])[keep], rb["dWx"][keep], rb["SdWx"][keep], dtype, what + " dWx")
     if not skip.any():
