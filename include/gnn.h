@@ -135,6 +135,29 @@ gnn_status gnn_propagate_fused(const gnn_csr* g, gnn_msg msg, gnn_op op, const v
                                const float* w_csr, int F, gnn_dtype dtype, void* out,
                                int32_t* argmax, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* gnn_propagate_fused for callers that cannot provide a workspace.  (The paper has no counterpart;
+ * this exists for the way the library gets embedded.)  Some hosts give a plugin only the input and
+ * output buffers of a fixed memory plan and forbid it to allocate on the device: an inference
+ * server whose allocator has already claimed the GPU, so that a raw cudaMalloc may fail or
+ * fragment its pool; a latency-bound loop that cannot afford the device-wide synchronisation and
+ * unbounded cost of cudaMalloc / cudaFree.  For them the partial-row scratch of the fused propagate
+ * is a fixed 8 MiB array inside the library image (gnn_propagate_fused_static_max_bytes()); every
+ * GPU that loads the library holds those 8 MiB until the process exits.
+ *  - Same arguments and results as gnn_propagate_fused, minus ws / ws_bytes.  No cudaMalloc, cudaFree
+ *    or other allocating routine is called.
+ *  - Size limit: gnn_propagate_fused_workspace(E, F, op) must not exceed the 8 MiB (about 2 M edges
+ *    at F = 128 for SUM/MEAN, half that for MAX/MIN); larger problems are rejected with
+ *    GNN_ERR_WORKSPACE_TOO_SMALL and a message, before anything is launched.
+ *  - The first call on each device looks up the device address of the array (with that device
+ *    current) and caches it; make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left.  The
+ *    kernels write every word of it that they later read, so nothing has to be cleared between
+ *    calls; but two calls that overlap on the GPU (different streams, no ordering) race on it. */
+size_t gnn_propagate_fused_static_max_bytes(void);
+gnn_status gnn_propagate_fused_static(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* X,
+                                      const float* w_csr, int F, gnn_dtype dtype, void* out,
+                                      int32_t* argmax, gnn_stream stream);
+
 /* Backward of gnn_propagate_fused for dL/dout = dOut [N,F]:
  *   SUM/MEAN: dX[j,:] = sum over transposed positions q of row j of
  *                       wT[q] * scale(colT[q]) * dOut[colT[q],:],  scale = 1 or 1/indegree

@@ -13,6 +13,8 @@
 // Inside a warp, a feature row of F*s bytes is covered by LPR lanes holding one 16-byte chunk
 // each (times VPL when a row is wider than 512 bytes); the 32/LPR lane groups take alternating
 // edges, and are combined by an xor-shuffle tree at the end of each row.
+#include <mutex>
+
 #include "propagate.cuh"
 
 #ifndef PF_U_NARROW
@@ -650,6 +652,35 @@ gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const v
     return GNN_OK;
 }
 
+// ------------------------------------------------------------------ built-in scratch
+// Scratch for gnn_propagate_fused_static: lives in the library image, so every GPU that loads the
+// library carries these bytes until the process exits.  Host code must not hand this name to a
+// kernel: on the host it is only a handle for cudaGetSymbolAddress.
+constexpr size_t STATIC_WS_BYTES = (size_t)8 << 20;  // 8 MiB
+static __device__ __align__(256) unsigned char g_static_ws[STATIC_WS_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+static void* g_static_ws_addr[STATIC_MAX_DEVICES];  // device address of g_static_ws, per device ordinal
+static std::mutex g_static_ws_mutex;
+
+// device address of the built-in scratch on the current device (looked up once per device)
+static gnn_status static_ws_address(const char* who, void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaGetDevice: %s", who, cudaGetErrorString(e));
+    GNN_REQUIRE(dev >= 0 && dev < STATIC_MAX_DEVICES, GNN_ERR_UNSUPPORTED, "%s: device ordinal %d not supported", who, dev);
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (!g_static_ws_addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_ws);
+        if (e != cudaSuccess || !p)
+            GNN_FAIL(GNN_ERR_CUDA, "%s: cudaGetSymbolAddress failed: %s", who, cudaGetErrorString(e));
+        g_static_ws_addr[dev] = p;
+    }
+    *out = g_static_ws_addr[dev];
+    return GNN_OK;
+}
+
 }  // namespace gnn
 
 using namespace gnn;
@@ -769,6 +800,23 @@ gnn_status gnn_propagate_fused_backward_host(const gnn_csr* g, gnn_msg msg, gnn_
     rc = gnn_propagate_fused_backward(g, msg, op, d_in, nullptr, w_csrT, argmax, F, dtype, d_out, nullptr, ws, ws_bytes, stream);
     if (rc != GNN_OK) return rc;
     return copy_async(who, h_dX, d_out, bytes, cudaMemcpyDeviceToHost, st);
+}
+
+size_t gnn_propagate_fused_static_max_bytes(void) { return STATIC_WS_BYTES; }
+
+gnn_status gnn_propagate_fused_static(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* X,
+                                      const float* w_csr, int F, gnn_dtype dtype, void* out,
+                                      int32_t* argmax, gnn_stream stream) {
+    const char* who = "gnn_propagate_fused_static";
+    GNN_REQUIRE(g && F > 0, GNN_ERR_INVALID_ARG, "%s: null graph or bad F", who);
+    const size_t need = gnn_propagate_fused_workspace(g->E, F, op);
+    GNN_REQUIRE(need <= STATIC_WS_BYTES, GNN_ERR_WORKSPACE_TOO_SMALL,
+                "%s: E=%lld, F=%d needs %zu bytes of scratch; the built-in scratch holds %zu. "
+                "Use gnn_propagate_fused with a caller-provided workspace", who, (long long)g->E, F, need, STATIC_WS_BYTES);
+    void* ws = nullptr;
+    gnn_status rc = static_ws_address(who, &ws);
+    if (rc != GNN_OK) return rc;
+    return gnn_propagate_fused(g, msg, op, X, w_csr, F, dtype, out, argmax, ws, STATIC_WS_BYTES, stream);
 }
 
 }  // extern "C"

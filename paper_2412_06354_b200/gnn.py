@@ -51,6 +51,8 @@ SIGNATURES = {
     "gnn_propagate_fused_workspace": (_SZ, [_I64, _INT, _INT]),
     "gnn_propagate_fused": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_fused_static_max_bytes": (_SZ, []),
+    "gnn_propagate_fused_static": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP]),
     "gnn_gather": (_INT, [_VP, _I64, _VP, _I32, _INT, _INT, _VP, _VP]),
     "gnn_gather_backward": (_INT, [_CSR, _INT, _VP, _INT, _INT, _VP, _VP, _SZ, _VP]),
     "gnn_apply_edges": (_INT, [_CSR, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP]),
@@ -369,3 +371,19 @@ def gat_fused_backward(g: Graph, Wx, a_src, a_dst, fwd, dOut, H, slope=0.2, ws=N
                                          _p(dOut), H, Cw, _dtype(Wx), float(slope), _p(dWx), _p(da_src), _p(da_dst),
                                          _p(ws), ws.numel(), _stream()))
     return dict(dWx=dWx, da_src=da_src, da_dst=da_dst)
+
+
+def propagate_fused_static(g: Graph, X, w_csr=None, op="sum", out=None, argmax=None):
+    """gnn_propagate_fused_static: the fused propagate with the library's built-in 8 MiB scratch, for
+    embedders that may not allocate device memory.  The caller passes `out` (and `argmax` for max/min);
+    nothing is allocated here when they are given."""
+    X = _dev(X)
+    F = X.shape[1]
+    opc = _op(op)
+    if out is None:
+        out = torch.empty((g.N, F), dtype=X.dtype, device=X.device)
+    if opc in (MAX, MIN) and argmax is None:
+        argmax = torch.empty((g.N, F), dtype=torch.int32, device=X.device)
+    msg = COPY_XJ if w_csr is None else E_MUL_XJ
+    _check(load().gnn_propagate_fused_static(g.ref, msg, opc, _p(X), _p(w_csr), F, _dtype(X), _p(out), _p(argmax), _stream()))
+    return (out, argmax) if opc in (MAX, MIN) else out
