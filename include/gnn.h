@@ -268,6 +268,25 @@ gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_
                                      const void* dOut_GF, const int32_t* argmax, int F,
                                      gnn_dtype dtype, void* dX_NF, gnn_stream stream);
 
+/* ------------------------------------------------------------------ dense node-wise transform */
+
+/* Y = X * W (the Dense layer / the weight of a conv layer in the training example): X [N,K],
+ * W [K,M], Y [N,M], all row-major and of dtype.  bf16 with K and M multiples of 16 (16..256)
+ * runs on the tensor cores with fp32 accumulation; other cases use an fp32 FFMA kernel.
+ * ws: gnn_linear_workspace(N, K, M) bytes; its first 4 bytes are a device status word that the
+ * tensor-core path sets to GNN_ERR_TIMEOUT if one of its bounded waits expired (0 otherwise);
+ * read it after synchronising if you want to check. */
+size_t gnn_linear_workspace(int32_t N, int K, int M);
+gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype, void* Y,
+                      void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* dX = dY * W^T ([N,K]) and dW = X^T * dY ([K,M], of dtype); either output may be NULL.  dW sums
+ * over the N rows in slabs of 4096 rows whose fp32 partials are added in slab order, so the
+ * result is reproducible.  X is needed only for dW, W only for dX. */
+gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int32_t N, int K, int M,
+                               gnn_dtype dtype, void* dX, void* dW, void* ws, size_t ws_bytes,
+                               gnn_stream stream);
+
 /* Host-buffer variants for callers whose features live in host memory (one call = copy in,
  * compute, copy out; no counterpart in the paper beyond its "transfer the batch to the gpu"
  * step in the training example).  h_X / h_dOut and h_out / h_dX are HOST arrays [N,F] (pinned

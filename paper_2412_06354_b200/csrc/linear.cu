@@ -1,0 +1,184 @@
+// Dense node-wise transform (the Dense layer / layer weight of the training example):
+//   Y = X * W          X [N,K], W [K,M]
+//   dX = dY * W^T      dY [N,M]
+//   dW = X^T * dY      reduction over the N rows, split over row slabs and combined in slab order
+//
+// Two paths.  bf16 with K, M multiples of 16 (M <= 256, K <= 256) runs Y and dX on the 5th-generation
+// tensor cores (tcgen05.mma, accumulators in tensor memory); everything else (fp32, odd shapes, dW)
+// runs a shared-memory tiled FFMA kernel with fp32 accumulation.  All sums have a fixed order.
+#include "common.cuh"
+
+namespace gnn {
+
+// ------------------------------------------------------------------ FFMA path
+// C[m,n] = sum_k A(m,k) * B(k,n) with arbitrary element strides, so transposed operands are
+// stride swaps.  64x64 output tile per block, 16x16 threads, 4x4 outputs per thread, k in steps
+// of 16.  k range [k0, k1) per blockIdx.z slab; slab results go to C + z*slab_stride.
+constexpr int SG_TILE = 64, SG_K = 16;
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+template <typename TA, typename TB, typename TC>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* __restrict__ B, int64_t sbk,
+                 int64_t sbn, TC* __restrict__ C, int64_t Mr, int64_t Nc, int64_t Kd, int64_t k_per_slab,
+                 int64_t slab_stride) {
+    __shared__ float As[SG_K][SG_TILE + 1];
+    __shared__ float Bs[SG_K][SG_TILE + 1];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int64_t m0 = (int64_t)blockIdx.y * SG_TILE, n0 = (int64_t)blockIdx.x * SG_TILE;
+    const int64_t k0 = (int64_t)blockIdx.z * k_per_slab;
+    const int64_t k1 = (k0 + k_per_slab < Kd) ? k0 + k_per_slab : Kd;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int64_t kb = k0; kb < k1; kb += SG_K) {
+        for (int e = threadIdx.x; e < SG_K * SG_TILE; e += 256) {
+            // A tile: consecutive threads walk the faster-varying of (m, k) in memory
+            int kk, mm;
+            if (sak <= sam) { kk = e % SG_K; mm = e / SG_K; } else { mm = e % SG_TILE; kk = e / SG_TILE; }
+            const int64_t m = m0 + mm, k = kb + kk;
+            As[kk][mm] = (m < Mr && k < k1) ? to_f32(A[m * sam + k * sak]) : 0.f;
+            int kk2, nn;
+            if (sbn <= sbk) { nn = e % SG_TILE; kk2 = e / SG_TILE; } else { kk2 = e % SG_K; nn = e / SG_K; }
+            const int64_t n = n0 + nn, k2 = kb + kk2;
+            Bs[kk2][nn] = (n < Nc && k2 < k1) ? to_f32(B[k2 * sbk + n * sbn]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < SG_K; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    TC* Cz = C + (size_t)blockIdx.z * slab_stride;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + ty * 4 + i;
+        if (m >= Mr) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t n = n0 + tx * 4 + j;
+            if (n < Nc) Cz[m * Nc + n] = from_f32<TC>(acc[i][j]);
+        }
+    }
+}
+
+// out[i] = sum over slabs (ascending) of part[s][i]
+template <typename TC>
+__global__ void slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __restrict__ out) {
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int z = 0; z < slabs; ++z) s += part[(size_t)z * n + i];
+    out[i] = from_f32<TC>(s);
+}
+
+template <typename TA, typename TB, typename TC>
+static void launch_simt(const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbk, int64_t sbn, TC* C,
+                        int64_t Mr, int64_t Nc, int64_t Kd, int64_t k_per_slab, int slabs, int64_t slab_stride,
+                        cudaStream_t st) {
+    dim3 grid((unsigned)ceil_div(Nc, SG_TILE), (unsigned)ceil_div(Mr, SG_TILE), (unsigned)slabs);
+    gemm_simt_kernel<TA, TB, TC><<<grid, 256, 0, st>>>(A, sam, sak, B, sbk, sbn, C, Mr, Nc, Kd, k_per_slab, slab_stride);
+}
+
+constexpr int DW_SLAB_ROWS = 4096;  // rows of X / dY per partial of dW
+static int dw_slabs(int64_t N) { return (int)(N > 0 ? ceil_div(N, DW_SLAB_ROWS) : 1); }
+
+bool linear_tc_supported(int64_t N, int K, int M, gnn_dtype dtype);
+gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int M, int w_transposed, void* Y,
+                             int* d_flag, cudaStream_t st);
+
+}  // namespace gnn
+
+using namespace gnn;
+
+extern "C" {
+
+size_t gnn_linear_workspace(int32_t N, int K, int M) {
+    if (N < 0 || K <= 0 || M <= 0) return 0;
+    return 256 + up256((size_t)dw_slabs(N) * K * M * 4);
+}
+
+gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype, void* Y,
+                      void* ws, size_t ws_bytes, gnn_stream stream) {
+    const char* who = "gnn_linear";
+    GNN_REQUIRE(N >= 0 && K > 0 && M > 0, GNN_ERR_INVALID_ARG, "%s: bad shape", who);
+    GNN_REQUIRE(dtype == GNN_F32 || dtype == GNN_BF16, GNN_ERR_INVALID_ARG, "%s: bad dtype", who);
+    if (N == 0) return GNN_OK;
+    GNN_REQUIRE(X && W && Y, GNN_ERR_INVALID_ARG, "%s: null argument", who);
+    GNN_REQUIRE(ws && ws_bytes >= 256, GNN_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes needed", who, gnn_linear_workspace(N, K, M));
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemsetAsync(ws, 0, sizeof(int), st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed (is ws a device pointer?)", who);
+    if (linear_tc_supported(N, K, M, dtype)) return linear_tc_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
+    if (dtype == GNN_F32)
+        launch_simt<float, float, float>((const float*)X, K, 1, (const float*)W, M, 1, (float*)Y, N, M, K, K, 1, 0, st);
+    else
+        launch_simt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>((const __nv_bfloat16*)X, K, 1, (const __nv_bfloat16*)W, M, 1,
+                                                               (__nv_bfloat16*)Y, N, M, K, K, 1, 0, st);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int32_t N, int K, int M,
+                               gnn_dtype dtype, void* dX, void* dW, void* ws, size_t ws_bytes,
+                               gnn_stream stream) {
+    const char* who = "gnn_linear_backward";
+    GNN_REQUIRE(N >= 0 && K > 0 && M > 0, GNN_ERR_INVALID_ARG, "%s: bad shape", who);
+    GNN_REQUIRE(dtype == GNN_F32 || dtype == GNN_BF16, GNN_ERR_INVALID_ARG, "%s: bad dtype", who);
+    GNN_REQUIRE(dY || N == 0, GNN_ERR_INVALID_ARG, "%s: null dY", who);
+    const size_t need = gnn_linear_workspace(N, K, M);
+    GNN_REQUIRE(ws && ws_bytes >= need, GNN_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes needed", who, need);
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemsetAsync(ws, 0, sizeof(int), st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed (is ws a device pointer?)", who);
+    if (dX && N > 0) {
+        GNN_REQUIRE(W, GNN_ERR_INVALID_ARG, "%s: dX needs W", who);
+        // dX[n,k] = sum_m dY[n,m] * W[k,m]
+        if (linear_tc_supported(N, M, K, dtype)) {
+            gnn_status rc = linear_tc_forward(dY, W, N, M, K, 1, dX, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (dtype == GNN_F32) {
+            launch_simt<float, float, float>((const float*)dY, M, 1, (const float*)W, 1, M, (float*)dX, N, K, M, M, 1, 0, st);
+        } else {
+            launch_simt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>((const __nv_bfloat16*)dY, M, 1, (const __nv_bfloat16*)W, 1, M,
+                                                                   (__nv_bfloat16*)dX, N, K, M, M, 1, 0, st);
+        }
+        GNN_CHECK_LAUNCH(who);
+    }
+    if (dW) {
+        GNN_REQUIRE(X || N == 0, GNN_ERR_INVALID_ARG, "%s: dW needs X", who);
+        // dW[k,m] = sum_n X[n,k] * dY[n,m]: one fp32 partial per slab of rows, then summed in slab order
+        float* part = (float*)((char*)ws + 256);
+        const int slabs = dw_slabs(N);
+        const int64_t km = (int64_t)K * M;
+        if (N == 0) {
+            if (cudaMemsetAsync(part, 0, (size_t)km * 4, st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed", who);
+        } else if (dtype == GNN_F32) {
+            launch_simt<float, float, float>((const float*)X, 1, K, (const float*)dY, M, 1, part, K, M, N, DW_SLAB_ROWS, slabs, km, st);
+        } else {
+            launch_simt<__nv_bfloat16, __nv_bfloat16, float>((const __nv_bfloat16*)X, 1, K, (const __nv_bfloat16*)dY, M, 1, part, K, M, N,
+                                                           DW_SLAB_ROWS, slabs, km, st);
+        }
+        if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 256), 256, 0, st>>>(part, slabs, km, (float*)dW);
+        else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 256), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW);
+        GNN_CHECK_LAUNCH(who);
+    }
+    return GNN_OK;
+}
+
+}  // extern "C"

@@ -66,6 +66,9 @@ SIGNATURES = {
     "gnn_graph_ptr_from_ids": (_INT, [_VP, _I32, _I32, _VP, _VP, _SZ, _VP]),
     "gnn_reduce_nodes": (_INT, [_VP, _I32, _I32, _INT, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_reduce_nodes_backward": (_INT, [_VP, _I32, _I32, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
+    "gnn_linear_workspace": (_SZ, [_I32, _INT, _INT]),
+    "gnn_linear": (_INT, [_VP, _VP, _I32, _INT, _INT, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_linear_backward": (_INT, [_VP, _VP, _VP, _I32, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _SZ, _VP]),
 }
@@ -387,3 +390,26 @@ def propagate_fused_static(g: Graph, X, w_csr=None, op="sum", out=None, argmax=N
     msg = COPY_XJ if w_csr is None else E_MUL_XJ
     _check(load().gnn_propagate_fused_static(g.ref, msg, opc, _p(X), _p(w_csr), F, _dtype(X), _p(out), _p(argmax), _stream()))
     return (out, argmax) if opc in (MAX, MIN) else out
+
+
+# ------------------------------------------------------------------ dense transform
+def linear(X, W, ws=None, return_ws=False):
+    X, W = _dev(X), _dev(W)
+    (N, K), M = X.shape, W.shape[1]
+    Y = torch.empty((N, M), dtype=X.dtype, device=X.device)
+    if ws is None:
+        ws = torch.empty(load().gnn_linear_workspace(N, K, M), dtype=torch.uint8, device=X.device)
+    _check(load().gnn_linear(_p(X), _p(W), N, K, M, _dtype(X), _p(Y), _p(ws), ws.numel(), _stream()))
+    return (Y, ws) if return_ws else Y
+
+
+def linear_backward(X, W, dY, want_dX=True, want_dW=True, ws=None, return_ws=False):
+    dY = _dev(dY)
+    N, M = dY.shape
+    K = W.shape[0] if W is not None else X.shape[1]
+    dX = torch.empty((N, K), dtype=dY.dtype, device=dY.device) if want_dX else None
+    dW = torch.empty((K, M), dtype=dY.dtype, device=dY.device) if want_dW else None
+    if ws is None:
+        ws = torch.empty(load().gnn_linear_workspace(N, K, M), dtype=torch.uint8, device=dY.device)
+    _check(load().gnn_linear_backward(_p(X), _p(W), _p(dY), N, K, M, _dtype(dY), _p(dX), _p(dW), _p(ws), ws.numel(), _stream()))
+    return (dX, dW, ws) if return_ws else (dX, dW)

@@ -1,0 +1,87 @@
+"""GPU parity: dense node-wise transform Y = X*W, dX = dY*W^T, dW = X^T*dY against the CPU checker's
+triple loop.  bf16 shapes with K, M multiples of 16 take the tensor-core path."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2412_06354_b200 import synth
+from util import assert_close, bits, to_dev, to_host64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gnn():
+    from paper_2412_06354_b200 import gnn as g
+    g.load()
+    return g
+
+
+def status_word(ws):
+    import torch
+    torch.cuda.synchronize()
+    return int(ws[:4].view(torch.int32).item())
+
+
+CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), ("bf16", 2000, 64, 64),
+         ("bf16", 1000, 128, 128), ("bf16", 777, 256, 256), ("bf16", 129, 16, 32), ("bf16", 5, 256, 16),
+         ("bf16", 300, 48, 112), ("bf16", 257, 40, 24)]
+
+
+@pytest.mark.parametrize("dtype,n,K,M", CASES)
+def test_linear_forward_backward(gnn, dtype, n, K, M):
+    oracle.set_threads(8)
+    try:
+        X = synth.normal((n, K), dtype, 1000 + K)
+        a = (6.0 / (K + M)) ** 0.5
+        W32 = synth.uniform_f32((K, M), -a, a, 1001 + M)
+        W = W32
+        if dtype == "bf16":
+            import torch
+            W = torch.from_numpy(W32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        dY = synth.normal((n, M), dtype, 1002 + M, 1)
+        Y, ws = gnn.linear(to_dev(X), to_dev(W), return_ws=True)
+        assert status_word(ws) == 0
+        Yo, S = oracle.matmul(X, W)
+        assert_close(to_host64(Y), Yo, S, dtype, f"Y {dtype} {n}x{K}x{M}")
+        dX, dW, ws = gnn.linear_backward(to_dev(X), to_dev(W), to_dev(dY), return_ws=True)
+        assert status_word(ws) == 0
+        dXo, S = oracle.matmul(dY, W, tb=True)
+        assert_close(to_host64(dX), dXo, S, dtype, "dX")
+        dWo, S = oracle.matmul(X, dY, ta=True)
+        assert_close(to_host64(dW), dWo, S, dtype, "dW")
+        Y2 = gnn.linear(to_dev(X), to_dev(W))
+        assert np.array_equal(bits(Y), bits(Y2)), "not bit-reproducible"
+    finally:
+        oracle.set_threads(1)
+
+
+def test_linear_large_rows_tensor_core(gnn):
+    """N = 100000 rows, 256 -> 256 bf16 (the attention workload's transform): many tiles per CTA."""
+    import torch
+    n, K, M = 100_000, 256, 256
+    X = synth.normal_bf16((n, K), 1100)
+    W = torch.from_numpy(synth.glorot_f32(K, M, 1101)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    Y, ws = gnn.linear(to_dev(X), to_dev(W), return_ws=True)
+    assert status_word(ws) == 0
+    rows = np.random.default_rng(3).choice(n, 3000, replace=False)
+    rows = np.union1d(rows, [0, 127, 128, n - 1])
+    Yo, S = oracle.matmul(X[rows], W)
+    assert_close(to_host64(Y)[rows], Yo, S, "bf16", "sampled rows of Y")
+    # linearity in exact arithmetic: rows of zeros give zeros
+    Xz = X.copy()
+    Xz[::2] = 0
+    Yz = gnn.linear(to_dev(Xz), to_dev(W))
+    assert torch.count_nonzero(Yz[::2]) == 0 and torch.equal(Yz[1::2], Y[1::2])
+
+
+def test_linear_degenerate(gnn):
+    import torch
+    W = torch.zeros((64, 64), device="cuda")
+    Y = gnn.linear(torch.zeros((0, 64), device="cuda"), W)
+    assert Y.shape == (0, 64)
+    dX, dW = gnn.linear_backward(torch.zeros((0, 64), device="cuda"), W, torch.zeros((0, 64), device="cuda"))
+    assert torch.count_nonzero(dW) == 0
+    with pytest.raises(gnn.GnnError) as e:
+        gnn.linear(torch.zeros((8, 64), device="cuda"), W, ws=torch.empty(8, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
