@@ -148,6 +148,22 @@ def cpu_step(oracle, s):
     return time.perf_counter() - t0
 
 
+def all_max(x, device, world):
+    """Max over ranks of a host float (identity when single-process)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(work_per_rank, ms_per_step_max, world):
+    """Replicas only: every rank does the same work; the job's rate is all ranks' work over the slowest rank's time."""
+    return world * work_per_rank / (ms_per_step_max * 1e-3)
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -244,13 +260,10 @@ def main():
     barrier()
     clocks = sampler.stop()
     total_ms = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = all_max(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
     work = sum(E * F for F, _, _, _ in plan)  # edges*features per step (each fwd+bwd pair counted once)
-    value = world * work / (ms_per_step * 1e-3)
+    value = whole_job_value(work, ms_per_step, world)
 
     # ---- per-case breakdown and the roofline of the chunked propagate kernel
     peak, peak_src = measured_peak()
@@ -338,13 +351,9 @@ def run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, de
     t1.record(torch.cuda.current_stream())
     barrier()
     ms = t0.elapsed_time(t1) / args.e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = all_max(ms, dev, world)
     work = sum(E * F for F, _, _, _ in plan)
-    return {"value": world * work / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": args.e2e_steps,
+    return {"value": whole_job_value(work, ms, world), "unit": UNIT, "ms_per_step": ms, "steps": args.e2e_steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "note": "features and gradients copied from pinned host memory, results copied back, per case; graph and edge weights resident"}
 

@@ -208,6 +208,13 @@ gnn_status gnn_aggregate_backward(const gnn_csr* g, gnn_op op, const void* dOut_
                                   const int32_t* argmax, int F, gnn_dtype dtype, void* dm_EF,
                                   gnn_stream stream);
 
+/* out[i] = alpha*a[i] + beta*b[i] for i < n, computed in fp32 and rounded once (out may alias a or
+ * b).  The element-wise glue of layers built from the primitives: W_self*x_i + W_neigh*agg
+ * (GraphConv / SAGEConv), (1+eps)*x_i + sum_j x_j (the GIN layer named in Sec. 3 "Graph
+ * Convolutional Layers").  n must be a multiple of 16 bytes worth of elements. */
+gnn_status gnn_axpby(float alpha, const void* a, float beta, const void* b, int64_t n, gnn_dtype dtype,
+                     void* out, gnn_stream stream);
+
 /* ------------------------------------------------------------------ edge softmax ------------ */
 
 /* Attention normalisation of the GAT layer (Sec. 3 "Graph Convolutional Layers"): for every node

@@ -116,6 +116,23 @@ __global__ void graph_ptr_kernel(const int32_t* __restrict__ gid, int32_t N, int
     }
 }
 
+// out = alpha*a + beta*b, element-wise in fp32 (self terms of layers: W1*x_i + W2*agg, (1+eps)*x_i + sum)
+template <typename T>
+__global__ void axpby_kernel(float alpha, const uint4* __restrict__ a, float beta, const uint4* __restrict__ b,
+                             int64_t nvec, uint4* __restrict__ out) {
+    constexpr int EPC = Chunk<T>::N;
+    int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (; t < nvec; t += stride) {
+        float x[EPC], y[EPC];
+        Chunk<T>::unpack(a[t], x);
+        Chunk<T>::unpack(b[t], y);
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) x[j] = fmaf(alpha, x[j], beta * y[j]);
+        out[t] = Chunk<T>::pack(x);
+    }
+}
+
 }  // namespace gnn
 
 using namespace gnn;
@@ -272,6 +289,22 @@ gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_
         aggregate_backward_kernel<float><<<grid, 256, 0, st>>>(graph_ptr, G, N, (int)op, (const uint4*)dOut_GF, argmax, nvec, (uint4*)dX_NF);
     else
         aggregate_backward_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(graph_ptr, G, N, (int)op, (const uint4*)dOut_GF, argmax, nvec, (uint4*)dX_NF);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+gnn_status gnn_axpby(float alpha, const void* a, float beta, const void* b, int64_t n, gnn_dtype dtype,
+                     void* out, gnn_stream stream) {
+    const char* who = "gnn_axpby";
+    GNN_REQUIRE(n >= 0 && (dtype == GNN_F32 || dtype == GNN_BF16), GNN_ERR_INVALID_ARG, "%s: bad argument", who);
+    if (n == 0) return GNN_OK;
+    const int epc = 16 / elem_size(dtype);
+    GNN_REQUIRE(n % epc == 0, GNN_ERR_UNSUPPORTED, "%s: the element count must be a multiple of %d", who, epc);
+    GNN_REQUIRE(a && b && out && aligned16(a) && aligned16(b) && aligned16(out), GNN_ERR_INVALID_ARG, "%s: null or misaligned argument", who);
+    const int64_t nvec = n / epc;
+    cudaStream_t st = as_stream(stream);
+    if (dtype == GNN_F32) axpby_kernel<float><<<grid_for(nvec, 256), 256, 0, st>>>(alpha, (const uint4*)a, beta, (const uint4*)b, nvec, (uint4*)out);
+    else axpby_kernel<__nv_bfloat16><<<grid_for(nvec, 256), 256, 0, st>>>(alpha, (const uint4*)a, beta, (const uint4*)b, nvec, (uint4*)out);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }

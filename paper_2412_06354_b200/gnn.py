@@ -58,6 +58,7 @@ SIGNATURES = {
     "gnn_apply_edges": (_INT, [_CSR, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP]),
     "gnn_aggregate": (_INT, [_CSR, _INT, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_aggregate_backward": (_INT, [_CSR, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
+    "gnn_axpby": (_INT, [_F, _VP, _F, _VP, _I64, _INT, _VP, _VP]),
     "gnn_edge_softmax": (_INT, [_CSR, _VP, _INT, _INT, _VP, _VP, _VP, _VP]),
     "gnn_edge_softmax_backward": (_INT, [_CSR, _VP, _VP, _INT, _INT, _VP, _VP]),
     "gnn_gat_fused_workspace": (_SZ, [_I32, _I64, _INT, _INT, _INT]),
@@ -413,3 +414,11 @@ def linear_backward(X, W, dY, want_dX=True, want_dW=True, ws=None, return_ws=Fal
         ws = torch.empty(load().gnn_linear_workspace(N, K, M), dtype=torch.uint8, device=dY.device)
     _check(load().gnn_linear_backward(_p(X), _p(W), _p(dY), N, K, M, _dtype(dY), _p(dX), _p(dW), _p(ws), ws.numel(), _stream()))
     return (dX, dW, ws) if return_ws else (dX, dW)
+
+
+def axpby(alpha, a, beta, b, out=None):
+    a, b = _dev(a), _dev(b)
+    if out is None:
+        out = torch.empty_like(a)
+    _check(load().gnn_axpby(float(alpha), _p(a), float(beta), _p(b), a.numel(), _dtype(a), _p(out), _stream()))
+    return out
