@@ -34,6 +34,52 @@ UNIT = "edges*feat/s"
 ALL_CASES = [(F, dt) for dt in ("bf16", "f32") for F in (32, 64, 128, 256, 512)]
 FMAX = 512
 
+# DRAM bytes (read + write, GB) of one propagate_chunk_kernel launch at full size, from the single-pass ncu
+# capture summarised in profiles/propagate_sweep_full_size_dram_bytes.md.  Valid for the kernel as committed
+# with that capture; set an entry to None when the kernel changes.
+TRAFFIC_GB = {
+    "32:bf16:copy_xj:fwd": 1.47,
+    "32:bf16:copy_xj:bwd": 1.47,
+    "32:bf16:e_mul_xj:fwd": 1.98,
+    "32:bf16:e_mul_xj:bwd": 1.98,
+    "64:bf16:copy_xj:fwd": 2.08,
+    "64:bf16:copy_xj:bwd": 2.08,
+    "64:bf16:e_mul_xj:fwd": 2.59,
+    "64:bf16:e_mul_xj:bwd": 2.59,
+    "128:bf16:copy_xj:fwd": 6.25,
+    "128:bf16:copy_xj:bwd": 6.25,
+    "128:bf16:e_mul_xj:fwd": 6.76,
+    "128:bf16:e_mul_xj:bwd": 6.76,
+    "256:bf16:copy_xj:fwd": 19.34,
+    "256:bf16:copy_xj:bwd": 19.31,
+    "256:bf16:e_mul_xj:fwd": 19.85,
+    "256:bf16:e_mul_xj:bwd": 19.82,
+    "512:bf16:copy_xj:fwd": 54.24,
+    "512:bf16:copy_xj:bwd": 54.04,
+    "512:bf16:e_mul_xj:fwd": 54.75,
+    "512:bf16:e_mul_xj:bwd": 54.55,
+    "32:f32:copy_xj:fwd": 2.02,
+    "32:f32:copy_xj:bwd": 2.02,
+    "32:f32:e_mul_xj:fwd": 2.53,
+    "32:f32:e_mul_xj:bwd": 2.53,
+    "64:f32:copy_xj:fwd": 6.49,
+    "64:f32:copy_xj:bwd": 6.48,
+    "64:f32:e_mul_xj:fwd": 7.01,
+    "64:f32:e_mul_xj:bwd": 7.0,
+    "128:f32:copy_xj:fwd": 19.44,
+    "128:f32:copy_xj:bwd": 19.4,
+    "128:f32:e_mul_xj:fwd": 19.95,
+    "128:f32:e_mul_xj:bwd": 19.91,
+    "256:f32:copy_xj:fwd": 53.97,
+    "256:f32:copy_xj:bwd": 53.77,
+    "256:f32:e_mul_xj:fwd": 54.48,
+    "256:f32:e_mul_xj:bwd": 54.28,
+    "512:f32:copy_xj:fwd": 141.37,
+    "512:f32:copy_xj:bwd": 140.14,
+    "512:f32:e_mul_xj:fwd": 141.88,
+    "512:f32:e_mul_xj:bwd": 140.64,
+}
+
 
 def parse_cases(s):
     if not s or s == "sweep":
@@ -279,13 +325,27 @@ def main():
         per_case.append({"F": F, "dtype": dt, "msg": "e_mul_xj" if weighted else "copy_xj", "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
                          "edges_feat_per_s": E * F / ((f_ms + b_ms) * 1e-3), "compulsory_GBs_fwd": comp / f_ms / 1e6,
                          "gather_GBs_fwd": gath / f_ms / 1e6, "compulsory_frac_fwd": comp / f_ms / 1e6 / peak})
-    launches = 2 * len(plan)  # gnn_propagate_fused + _backward calls per step; each is 2 kernels
-    achieved = tot_comp / tot_ms / 1e6
-    roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel (+ fixup), all launches of the step",
-                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                "peak_source": peak_src, "bytes_model": "compulsory: 4E(+4E weights)+8N+2*N*F*s per launch",
-                "bytes_per_launch_avg": tot_comp / (2 * len(plan)), "ms_per_launch_avg": tot_ms / (2 * len(plan)),
-                "gather_upper_bound_GBs": tot_gath / tot_ms / 1e6}
+    # dominant kernel instance = the case with the largest share of the step
+    dom = max(per_case, key=lambda c: c["fwd_ms"] + c["bwd_ms"])
+    sdom = 2 if dom["dtype"] == "bf16" else 4
+    wdom = dom["msg"] == "e_mul_xj"
+    comp = compulsory_bytes(N, E, dom["F"], sdom, wdom)
+    tkey = "%d:%s:%s:fwd" % (dom["F"], dom["dtype"], dom["msg"])
+    traffic = TRAFFIC_GB.get(tkey) if shrink == 0 else None
+    achieved = comp / dom["fwd_ms"] / 1e6
+    roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel, forward launch of F=%d %s %s (largest share of the step: %.1f %%)"
+                % (dom["F"], dom["dtype"], dom["msg"], 100 * (dom["fwd_ms"] + dom["bwd_ms"]) / tot_ms),
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None if traffic is None else traffic * 1e9,
+                "peak_source": peak_src, "bytes_model": "compulsory bytes per launch: 4E(+4E weights)+8N+2*N*F*s = %d" % comp,
+                "ms_per_launch": dom["fwd_ms"],
+                "dram_traffic_GBs": None if traffic is None else traffic * 1e3 / dom["fwd_ms"],
+                "dram_traffic_frac_of_peak": None if traffic is None else traffic * 1e3 / dom["fwd_ms"] / peak,
+                "gather_upper_bound_GBs": gather_bytes(N, E, dom["F"], sdom, wdom) / dom["fwd_ms"] / 1e6,
+                "all_launches": {"compulsory_GBs": tot_comp / tot_ms / 1e6, "frac": tot_comp / tot_ms / 1e6 / peak,
+                                 "gather_upper_bound_GBs": tot_gath / tot_ms / 1e6,
+                                 "dram_traffic_GBs": (sum(TRAFFIC_GB["%d:%s:%s:%s" % (c["F"], c["dtype"], c["msg"], d)] for c in per_case for d in ("fwd", "bwd")) * 1e3 / tot_ms
+                                                      if shrink == 0 and all(TRAFFIC_GB.get("%d:%s:%s:fwd" % (c["F"], c["dtype"], c["msg"])) for c in per_case) else None)}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
