@@ -103,6 +103,9 @@ static int dw_slabs(int64_t N) { return (int)(N > 0 ? ceil_div(N, DW_SLAB_ROWS) 
 bool linear_tc_supported(int64_t N, int K, int M, gnn_dtype dtype);
 gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int M, int w_transposed, void* Y,
                              int* d_flag, cudaStream_t st);
+bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
+int linear_tc_dw_partials(int64_t N);
+gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
 
 }  // namespace gnn
 
@@ -112,7 +115,8 @@ extern "C" {
 
 size_t gnn_linear_workspace(int32_t N, int K, int M) {
     if (N < 0 || K <= 0 || M <= 0) return 0;
-    return 256 + up256((size_t)dw_slabs(N) * K * M * 4);
+    const size_t parts = (size_t)(dw_slabs(N) > 148 ? dw_slabs(N) : 148);  // FFMA slabs or tensor-core CTA partials
+    return 256 + up256(parts * K * M * 4);
 }
 
 gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype, void* Y,
@@ -164,9 +168,13 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         GNN_REQUIRE(X || N == 0, GNN_ERR_INVALID_ARG, "%s: dW needs X", who);
         // dW[k,m] = sum_n X[n,k] * dY[n,m]: one fp32 partial per slab of rows, then summed in slab order
         float* part = (float*)((char*)ws + 256);
-        const int slabs = dw_slabs(N);
+        int slabs = dw_slabs(N);
         const int64_t km = (int64_t)K * M;
-        if (N == 0) {
+        if (linear_tc_dw_supported(N, K, M, dtype)) {
+            slabs = linear_tc_dw_partials(N);
+            gnn_status rc = linear_tc_dw(X, dY, N, K, M, part, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (N == 0) {
             if (cudaMemsetAsync(part, 0, (size_t)km * 4, st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed", who);
         } else if (dtype == GNN_F32) {
             launch_simt<float, float, float>((const float*)X, 1, K, (const float*)dY, M, 1, part, K, M, N, DW_SLAB_ROWS, slabs, km, st);

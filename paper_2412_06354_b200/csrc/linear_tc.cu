@@ -17,7 +17,8 @@
 namespace gnn {
 
 constexpr int TC_ROWS = 128;     // rows of X per tile = MMA M
-constexpr int TC_THREADS = 128;  // 4 warps: warp w owns accumulator lanes 32w..32w+31
+constexpr int TC_THREADS = 256;   // 8 warps: warp w reads accumulator lanes 32*(w%4).. and column half w/4
+constexpr int TC_THREADS2 = 256;  // dW kernel, same split
 constexpr uint32_t TC_WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -152,10 +153,11 @@ linear_tc_kernel(const TcParams P) {
         if (!ok) {
             failed = true;
         } else {
-            // accumulator row = tensor-memory lane; this thread's row:
-            const int64_t row = row0 + warp * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
-            for (int c0 = 0; c0 < M; c0 += 16) {
+            // accumulator row = tensor-memory lane; this thread's row and its half of the columns:
+            const int lane_block = warp & 3, col_half = warp >> 2;
+            const int64_t row = row0 + lane_block * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(lane_block * 32) << 16);
+            for (int c0 = col_half * 16; c0 < M; c0 += 32) {
                 uint32_t r[16];
                 asm volatile(
                     "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
@@ -206,8 +208,165 @@ gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int
     cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
     const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
-    const int grid = (int)(ntiles < 148 ? ntiles : 148);
+    // several CTAs per SM when shared and tensor memory allow: one loads while another computes
+    int per_sm = (int)((200 * 1024) / (smem + 1024));
+    if (per_sm > 512 / cols) per_sm = 512 / cols;
+    per_sm = per_sm < 1 ? 1 : (per_sm > 3 ? 3 : per_sm);
+    const int64_t slots = (int64_t)148 * per_sm;
+    const int grid = (int)(ntiles < slots ? ntiles : slots);
     linear_tc_kernel<<<grid, TC_THREADS, smem, st>>>(P);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+// ------------------------------------------------------------------ dW = X^T * dY on tcgen05
+// Contraction over the N rows.  A = X^T (features x rows) and B = dY (rows x columns) are both
+// "MN-major" as stored: 16-byte chunk c of row n goes to c*sbo + (n/8)*128 + (n%8)*16 with
+// sbo = (128/8)*128.  MMA shape 128 x M x 16 (K = 256 uses two accumulators of 128 feature rows).
+// Each CTA accumulates its row tiles (t = blockIdx.x, +gridDim.x, ...) in tensor memory and writes
+// one fp32 partial [K,M]; the partials are summed in CTA order by slab_sum_kernel.
+struct TcDwParams {
+    const __nv_bfloat16* X;   // [N,K]
+    const __nv_bfloat16* dY;  // [N,M]
+    float* part;              // [gridDim.x][K][M]
+    int64_t N;
+    int K, M;
+    int tmem_cols;
+    int* status;
+};
+
+__global__ void __launch_bounds__(TC_THREADS2, 1)
+linear_tc_dw_kernel(const TcDwParams P) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ __align__(8) uint64_t mbar;
+    __shared__ uint32_t tmem_base_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = P.K, M = P.M;
+    const int kc = K / 8, mc = M / 8;            // 16-byte chunks per row of X / dY
+    constexpr uint32_t sbo = (TC_ROWS / 8) * 128;  // 2048: next chunk of 8 features / columns
+    unsigned char* sA = smem;                    // K x 128 rows  (bf16)
+    unsigned char* sB = smem + (size_t)K * TC_ROWS * 2;
+    const int halves = K / 128;
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)P.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar)) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t idesc = make_idesc(M, 1) | (1u << 15);  // A and B both MN-major
+    const uint32_t bar = smem_u32(&mbar);
+    const int64_t ntiles = (P.N + TC_ROWS - 1) / TC_ROWS;
+    const uint64_t pol_stream = policy_evict_first();
+    uint32_t parity = 0;
+    bool failed = false, first = true;
+
+    for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const int64_t row0 = t * TC_ROWS;
+        const uint4* srcX = reinterpret_cast<const uint4*>(P.X);
+        const uint4* srcY = reinterpret_cast<const uint4*>(P.dY);
+        for (int e = tid; e < TC_ROWS * kc; e += TC_THREADS2) {
+            const int r = e / kc, c = e - r * kc;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (row0 + r < P.N) v = ld_hint16(srcX + (size_t)(row0 + r) * kc + c, pol_stream);
+            *reinterpret_cast<uint4*>(sA + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16) = v;
+        }
+        for (int e = tid; e < TC_ROWS * mc; e += TC_THREADS2) {
+            const int r = e / mc, c = e - r * mc;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (row0 + r < P.N) v = ld_hint16(srcY + (size_t)(row0 + r) * mc + c, pol_stream);
+            *reinterpret_cast<uint4*>(sB + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (tid == 0) {
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            for (int h = 0; h < halves; ++h)
+                for (int kk = 0; kk < TC_ROWS / 16; ++kk) {
+                    // A: features [128h, 128h+128) = chunks 16h.., rows 16kk.. = row groups 2kk, 2kk+1
+                    const uint64_t adesc = make_smem_desc(a0 + (uint32_t)h * 16 * sbo + (uint32_t)kk * 256, 128, sbo);
+                    const uint64_t bdesc = make_smem_desc(b0 + (uint32_t)kk * 256, 128, sbo);
+                    mma_bf16_ss(tmem_base + (uint32_t)h * (uint32_t)M, adesc, bdesc, idesc, (first && kk == 0) ? 0u : 1u);
+                }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+        }
+        first = false;
+        // the shared-memory tiles may be overwritten only after the MMAs that read them have completed
+        const bool ok = mbar_wait_bounded(bar, parity);
+        parity ^= 1;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (!ok) failed = true;
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (failed) break;
+    }
+    // accumulator -> this CTA's partial.  Lane = feature row within the half; warps 4..7 take the
+    // upper half of the columns.
+    float* part = P.part + (size_t)blockIdx.x * K * M;
+    if (!failed) {
+        const int lane_block = warp & 3, col_half = warp >> 2;
+        const int cbeg = col_half * (M / 2), cend = cbeg + M / 2;
+        for (int h = 0; h < halves; ++h) {
+            const int krow = h * 128 + lane_block * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(lane_block * 32) << 16) + (uint32_t)h * (uint32_t)M;
+            for (int c0 = cbeg; c0 < cend; c0 += 8) {
+                uint32_t r[8];
+                if (first) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) r[j] = 0u;  // this CTA had no tile: its partial is zero
+                } else {
+                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                                 : "r"(taddr + (uint32_t)c0));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                }
+                float4* dst = reinterpret_cast<float4*>(part + (size_t)krow * M + c0);
+                dst[0] = make_float4(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]), __uint_as_float(r[3]));
+                dst[1] = make_float4(__uint_as_float(r[4]), __uint_as_float(r[5]), __uint_as_float(r[6]), __uint_as_float(r[7]));
+            }
+        }
+    }
+    if (failed && tid == 0) atomicExch(P.status, 7);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)P.tmem_cols) : "memory");
+}
+
+bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
+    if (dtype != GNN_BF16 || N <= 0) return false;
+    if (K != 128 && K != 256) return false;
+    if (M % 16 != 0 || M < 16 || M > 256) return false;
+    return true;
+}
+
+int linear_tc_dw_partials(int64_t N) {
+    const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
+    return (int)(ntiles < 148 ? (ntiles > 0 ? ntiles : 1) : 148);
+}
+
+// writes linear_tc_dw_partials(N) fp32 partials [K,M] to part
+gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
+    const char* who = "gnn_linear_backward (tensor-core dW)";
+    GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
+    TcDwParams P;
+    P.X = (const __nv_bfloat16*)X; P.dY = (const __nv_bfloat16*)dY; P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
+    int cols = 32;
+    while (cols < M * (K / 128)) cols <<= 1;
+    P.tmem_cols = cols;
+    const size_t smem = (size_t)TC_ROWS * K * 2 + (size_t)TC_ROWS * M * 2;
+    cudaError_t e = cudaFuncSetAttribute(linear_tc_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
+    linear_tc_dw_kernel<<<linear_tc_dw_partials(N), TC_THREADS2, smem, st>>>(P);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
