@@ -8,10 +8,12 @@
 // 128 x M x 16 into a 128-lane x M-column fp32 accumulator in tensor memory, the completion is
 // signalled on an mbarrier by tcgen05.commit, and four warps read the accumulator back
 // (tcgen05.ld), round to bf16 and store their rows.  The contraction is short (K <= 256), so the
-// kernel is bound by reading X and writing Y; the layout copies are plain 16-byte loads/stores.
+// kernel is bound by reading X and writing Y; the layout copies are 16-byte cp.async transfers (global to shared without registers).
 //
 // Every wait has an iteration limit: on expiry the CTA raises a status word, skips its stores,
 // still frees its tensor memory and returns.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace gnn {
@@ -22,6 +24,12 @@ constexpr int TC_THREADS2 = 256;  // dW kernel, same split
 constexpr uint32_t TC_WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 16-byte asynchronous copy global -> shared, bypassing registers; src_bytes = 0 writes zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // shared-memory matrix descriptor, no swizzle: start address, leading/stride byte offsets (all >> 4)
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -64,6 +72,18 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         if (done) return true;
     }
     return false;
+}
+
+// raise a kernel's dynamic shared memory limit to 200 KB, once per (device, kernel)
+static gnn_status allow_big_smem(const char* who, const void* kernel, int which) {
+    static std::atomic<unsigned char> done[64][2];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
+    if (dev >= 0 && done[dev][which].load()) return GNN_OK;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
+    if (dev >= 0) done[dev][which].store(1);
+    return GNN_OK;
 }
 
 struct TcParams {
@@ -119,19 +139,20 @@ linear_tc_kernel(const TcParams P) {
     const int64_t ntiles = (P.N + TC_ROWS - 1) / TC_ROWS;
     uint32_t parity = 0;
     bool failed = false;
-    const uint64_t pol_stream = policy_evict_first();
 
     for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
         const int64_t row0 = t * TC_ROWS;
         // X tile -> canonical K-major layout: chunk kc of row r at (r/8)*sbo + kc*128 + (r%8)*16
         {
             const uint4* src = reinterpret_cast<const uint4*>(P.X);
+            const uint32_t a0 = smem_u32(sA);
             for (int e = tid; e < TC_ROWS * kchunks; e += TC_THREADS) {
                 const int r = e / kchunks, kc = e - r * kchunks;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (row0 + r < P.N) v = ld_hint16(src + (size_t)(row0 + r) * kchunks + kc, pol_stream);
-                *reinterpret_cast<uint4*>(sA + (uint32_t)(r >> 3) * sbo + (uint32_t)kc * 128 + (uint32_t)(r & 7) * 16) = v;
+                const bool in = row0 + r < P.N;
+                cp_async16(a0 + (uint32_t)(r >> 3) * sbo + (uint32_t)kc * 128 + (uint32_t)(r & 7) * 16,
+                           src + (in ? (size_t)(row0 + r) * kchunks + kc : 0), in ? 16u : 0u);
             }
+            cp_async_wait_all();
         }
         // generic-proxy writes to shared memory -> visible to the tensor core (async proxy)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -205,8 +226,8 @@ gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int
     while (cols < M) cols <<= 1;
     P.tmem_cols = cols;
     const size_t smem = (size_t)M * K * 2 + (size_t)TC_ROWS * K * 2;
-    cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tc_kernel, 0);
+    if (rc != GNN_OK) return rc;
     const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
     // several CTAs per SM when shared and tensor memory allow: one loads while another computes
     int per_sm = (int)((200 * 1024) / (smem + 1024));
@@ -263,7 +284,6 @@ linear_tc_dw_kernel(const TcDwParams P) {
     const uint32_t idesc = make_idesc(M, 1) | (1u << 15);  // A and B both MN-major
     const uint32_t bar = smem_u32(&mbar);
     const int64_t ntiles = (P.N + TC_ROWS - 1) / TC_ROWS;
-    const uint64_t pol_stream = policy_evict_first();
     uint32_t parity = 0;
     bool failed = false, first = true;
 
@@ -271,18 +291,20 @@ linear_tc_dw_kernel(const TcDwParams P) {
         const int64_t row0 = t * TC_ROWS;
         const uint4* srcX = reinterpret_cast<const uint4*>(P.X);
         const uint4* srcY = reinterpret_cast<const uint4*>(P.dY);
+        const uint32_t sa0 = smem_u32(sA), sb0 = smem_u32(sB);
         for (int e = tid; e < TC_ROWS * kc; e += TC_THREADS2) {
             const int r = e / kc, c = e - r * kc;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (row0 + r < P.N) v = ld_hint16(srcX + (size_t)(row0 + r) * kc + c, pol_stream);
-            *reinterpret_cast<uint4*>(sA + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16) = v;
+            const bool in = row0 + r < P.N;
+            cp_async16(sa0 + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16,
+                       srcX + (in ? (size_t)(row0 + r) * kc + c : 0), in ? 16u : 0u);
         }
         for (int e = tid; e < TC_ROWS * mc; e += TC_THREADS2) {
             const int r = e / mc, c = e - r * mc;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (row0 + r < P.N) v = ld_hint16(srcY + (size_t)(row0 + r) * mc + c, pol_stream);
-            *reinterpret_cast<uint4*>(sB + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16) = v;
+            const bool in = row0 + r < P.N;
+            cp_async16(sb0 + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16,
+                       srcY + (in ? (size_t)(row0 + r) * mc + c : 0), in ? 16u : 0u);
         }
+        cp_async_wait_all();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
@@ -364,8 +386,8 @@ gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, 
     while (cols < M * (K / 128)) cols <<= 1;
     P.tmem_cols = cols;
     const size_t smem = (size_t)TC_ROWS * K * 2 + (size_t)TC_ROWS * M * 2;
-    cudaError_t e = cudaFuncSetAttribute(linear_tc_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tc_dw_kernel, 1);
+    if (rc != GNN_OK) return rc;
     linear_tc_dw_kernel<<<linear_tc_dw_partials(N), TC_THREADS2, smem, st>>>(P);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
