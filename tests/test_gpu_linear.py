@@ -23,7 +23,7 @@ def status_word(ws):
     return int(ws[:4].view(torch.int32).item())
 
 
-CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), ("bf16", 2000, 64, 64),
+CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), ("f32", 1000, 256, 64), ("f32", 700, 128, 48), ("f32", 5000, 16, 256), ("bf16", 2000, 64, 64),
          ("bf16", 1000, 128, 128), ("bf16", 777, 256, 256), ("bf16", 129, 16, 32), ("bf16", 5, 256, 16),
          ("bf16", 300, 48, 112), ("bf16", 257, 40, 24)]
 
