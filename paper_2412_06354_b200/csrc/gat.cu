@@ -62,31 +62,33 @@ gat_backward_rows_kernel(const int64_t* __restrict__ rowptr, const int32_t* __re
                          float* __restrict__ dar) {
     __shared__ float red[GB_BLOCK];
     constexpr int NT = LONG ? GB_BLOCK : 32;
-    const int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    if (row >= N) return;
-    const int64_t a = rowptr[row], b = rowptr[row + 1];
-    if (((b - a) > GB_LONG_ROW) != LONG) return;
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     const int h = tid % H;  // H is a power of two <= 32: fixed per thread
-    if (b == a) {
-        if (!LONG && tid < H) dar[(size_t)row * H + tid] = 0.f;
-        return;
+    int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int stride = LONG ? gridDim.x : (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > GB_LONG_ROW) != LONG) continue;  // uniform per warp / per block
+        if (b == a) {
+            if (tid < H) dar[(size_t)row * H + tid] = 0.f;
+            continue;
+        }
+        const size_t lo = (size_t)a * H, hi = (size_t)b * H;
+        float d = 0.f;
+        for (size_t t = lo + tid; t < hi; t += NT) d = fmaf(alpha[t], dalpha_dz[t], d);
+        d = sum_same_head<NT>(d, H, red);
+        const float arv = ar[(size_t)row * H + h];
+        float sdz = 0.f;
+        for (size_t t = lo + tid; t < hi; t += NT) {
+            const int64_t p = (int64_t)(t / H);
+            const float z = al[(size_t)col[p] * H + h] + arv;
+            const float dz = alpha[t] * (dalpha_dz[t] - d) * (z > 0.f ? 1.f : slope);
+            dalpha_dz[t] = dz;
+            sdz += dz;
+        }
+        sdz = sum_same_head<NT>(sdz, H, red);
+        if (tid < H) dar[(size_t)row * H + tid] = sdz;
     }
-    const size_t lo = (size_t)a * H, hi = (size_t)b * H;
-    float d = 0.f;
-    for (size_t t = lo + tid; t < hi; t += NT) d = fmaf(alpha[t], dalpha_dz[t], d);
-    d = sum_same_head<NT>(d, H, red);
-    const float arv = ar[(size_t)row * H + h];
-    float sdz = 0.f;
-    for (size_t t = lo + tid; t < hi; t += NT) {
-        const int64_t p = (int64_t)(t / H);
-        const float z = al[(size_t)col[p] * H + h] + arv;
-        const float dz = alpha[t] * (dalpha_dz[t] - d) * (z > 0.f ? 1.f : slope);
-        dalpha_dz[t] = dz;
-        sdz += dz;
-    }
-    sdz = sum_same_head<NT>(sdz, H, red);
-    if (tid < H) dar[(size_t)row * H + tid] = sdz;
 }
 
 // da_src[f] = sum_n dal[n,h(f)] * Wx[n,f], da_dst likewise with dar: fixed two-stage reduction
@@ -172,6 +174,9 @@ static gnn_status gat_check(const char* who, const gnn_csr* g, int H, int C, gnn
     return GNN_OK;
 }
 
+gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float slope, int H, float* alpha, cudaStream_t st);
+bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz, const float* al, const float* ar,
+                          float slope, int H, float* dar, cudaStream_t st);
 gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const void* dOut, int H, int C,
                        gnn_dtype dtype, float* dW_EH, cudaStream_t st);
 
@@ -203,10 +208,9 @@ gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, c
     else
         gat_scores_kernel<__nv_bfloat16><<<(int)ceil_div(NH, 256), 256, 0, st>>>((const __nv_bfloat16*)Wx, a_src, a_dst, NH, H, C, al, ar);
     GNN_CHECK_LAUNCH(who);
-    // logits into alpha_csr, then normalised in place (each element is read and written by one thread)
-    rc = gnn_apply_edges(g, GNN_MSG_GAT_LOGIT, al, ar, nullptr, 0, H, GNN_F32, slope, alpha_csr, stream);
-    if (rc != GNN_OK) return rc;
-    rc = gnn_edge_softmax(g, alpha_csr, H, GNN_F32, alpha_csr, nullptr, nullptr, stream);
+    // logits and their per-row softmax, written straight into alpha_csr
+    GNN_REQUIRE(g->E == 0 || g->col, GNN_ERR_INVALID_ARG, "%s: null col", who);
+    rc = gat_alpha(g, al, ar, slope, H, alpha_csr, st);
     if (rc != GNN_OK) return rc;
     HeadExtra hx = {alpha_csr, H, nullptr, nullptr, nullptr, nullptr};
     return run_chunked(who, MODE_HEADSUM, g->N, g->E, g->rowptr, g->col, nullptr, Wx, out, nullptr, nullptr,
@@ -237,9 +241,13 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
     rc = sddmm_heads(who, g, Wx, dOut, H, C, dtype, w.dz, st);
     if (rc != GNN_OK) return rc;
     // softmax and LeakyReLU derivatives, dz over dalpha, dar per row
-    gat_backward_rows_kernel<false><<<(int)ceil_div((int64_t)g->N * 32, GB_BLOCK), GB_BLOCK, 0, st>>>(
-        g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
-    gat_backward_rows_kernel<true><<<g->N, GB_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+    if (!gat_rows_backward_pl(g, alpha_csr, w.dz, al, ar, slope, H, w.dar, st)) {
+        const int64_t wwant = ceil_div((int64_t)g->N * 32, GB_BLOCK), cap = (int64_t)148 * 64;
+        gat_backward_rows_kernel<false><<<(int)(wwant < cap ? wwant : cap), GB_BLOCK, 0, st>>>(
+            g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+        gat_backward_rows_kernel<true><<<(int)(g->N < cap ? g->N : cap), GB_BLOCK, 0, st>>>(
+            g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+    }
     GNN_CHECK_LAUNCH(who);
     // dal[j,h] = sum over the out-edges of j of dz
     if (H % 4 == 0) {

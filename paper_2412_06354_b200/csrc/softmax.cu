@@ -109,25 +109,34 @@ __device__ __forceinline__ void softmax_bwd_row(const T* alpha, const T* dalpha,
 
 static __host__ __device__ inline bool head_pow2(int H) { return H >= 1 && H <= 32 && (H & (H - 1)) == 0; }
 
+// Row loops: every warp (LONG = false) or block (LONG = true) strides over the rows and takes the
+// ones of its kind, so the grids stay a few waves large whatever N is.
+template <bool LONG>
+__device__ __forceinline__ void row_loop_bounds(int* first, int* stride) {
+    if (LONG) { *first = blockIdx.x; *stride = gridDim.x; }
+    else { *first = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5); *stride = (int)((gridDim.x * (int64_t)blockDim.x) >> 5); }
+}
+
 template <typename T, bool LONG>
 __global__ void __launch_bounds__(SM_BLOCK)
 edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ s, int H,
                     T* __restrict__ alpha, float* __restrict__ rowmax, float* __restrict__ rowsum) {
     __shared__ float red[SM_BLOCK];
-    const int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    if (row >= N) return;
-    const int64_t a = rowptr[row], b = rowptr[row + 1];
-    const bool is_long = (b - a) > SM_LONG_ROW;
-    if (is_long != LONG) return;  // uniform per warp (LONG = false) or per block (LONG = true)
-    if (b == a) {
-        if (!LONG && (threadIdx.x & 31) < H) {
-            if (rowmax) rowmax[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
-            if (rowsum) rowsum[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
+    int row, stride;
+    row_loop_bounds<LONG>(&row, &stride);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > SM_LONG_ROW) != LONG) continue;  // uniform per warp (LONG = false) or per block (LONG = true)
+        if (b == a) {
+            if ((threadIdx.x & 31) < H) {
+                if (rowmax) rowmax[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
+                if (rowsum) rowsum[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
+            }
+            continue;
         }
-        return;
+        if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
+        else softmax_row_any<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
     }
-    if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
-    else softmax_row_any<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
 }
 
 template <typename T, bool LONG>
@@ -135,11 +144,239 @@ __global__ void __launch_bounds__(SM_BLOCK)
 edge_softmax_backward_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ alpha,
                              const T* __restrict__ dalpha, int H, T* __restrict__ ds) {
     __shared__ float red[SM_BLOCK];
-    const int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    if (row >= N) return;
-    const int64_t a = rowptr[row], b = rowptr[row + 1];
-    if (((b - a) > SM_LONG_ROW) != LONG || b == a) return;
-    softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
+    int row, stride;
+    row_loop_bounds<LONG>(&row, &stride);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
+        softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
+    }
+}
+
+// GAT attention coefficients in one kernel: logits z = LeakyReLU(al[col[p],h] + ar[i,h]) are written
+// to alpha in the first pass (each thread re-reads only what it wrote), then normalised in place.
+// H is a power of two <= 32.
+template <bool LONG>
+__global__ void __launch_bounds__(SM_BLOCK)
+gat_alpha_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N, int H,
+                 const float* __restrict__ al, const float* __restrict__ ar, float slope, float* __restrict__ alpha) {
+    __shared__ float red[SM_BLOCK];
+    constexpr int NT = LONG ? SM_BLOCK : 32;
+    const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
+    const int h = tid % H;
+    int row, stride;
+    row_loop_bounds<LONG>(&row, &stride);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
+        const size_t lo = (size_t)a * H, hi = (size_t)b * H;
+        const float arv = ar[(size_t)row * H + h];
+        float m = -INFINITY;
+        for (size_t t = lo + tid; t < hi; t += NT) {
+            float z = al[(size_t)col[t / H] * H + h] + arv;
+            z = z > 0.f ? z : slope * z;
+            alpha[t] = z;
+            m = fmaxf(m, z);
+        }
+        m = reduce_same_head<MaxOp, NT>(m, H, red);
+        float zs = 0.f;
+        for (size_t t = lo + tid; t < hi; t += NT) zs += expf(alpha[t] - m);
+        zs = reduce_same_head<SumOp, NT>(zs, H, red);
+        for (size_t t = lo + tid; t < hi; t += NT) alpha[t] = expf(alpha[t] - m) / zs;
+    }
+}
+
+// ---- position-per-lane layout for H = 4*HV heads: a lane owns whole positions (all heads of an
+// edge as HV float4), so a row of up to 32 edges is one vector load per array per lane, and the
+// per-head reductions run over lanes (warp) or over lanes and warps (block, long rows).
+template <int HV, int NT, bool IS_MAX>
+__device__ __forceinline__ void reduce_heads(float (&v)[4 * HV], float* red) {
+#pragma unroll
+    for (int j = 0; j < 4 * HV; ++j) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[j], o);
+            v[j] = IS_MAX ? fmaxf(v[j], other) : (((threadIdx.x & o) == 0) ? v[j] + other : other + v[j]);
+        }
+    }
+    if (NT > 32) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        __syncthreads();
+        if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < 4 * HV; ++j) red[warp * 32 + j] = v[j];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 4 * HV; ++j) {
+            float r = IS_MAX ? -INFINITY : 0.f;
+            for (int w = 0; w < NT / 32; ++w) r = IS_MAX ? fmaxf(r, red[w * 32 + j]) : r + red[w * 32 + j];
+            v[j] = r;
+        }
+    }
+}
+
+constexpr int PL_BLOCK = 512;  // threads per long row
+
+template <int HV, bool LONG>
+__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
+gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
+                    const float* __restrict__ al, const float* __restrict__ ar, float slope, float* __restrict__ alpha) {
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
+    __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
+    const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
+    int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int stride = LONG ? gridDim.x : (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
+        float arv[H], m[H], zs[H];
+#pragma unroll
+        for (int q = 0; q < HV; ++q) {
+            const float4 t = reinterpret_cast<const float4*>(ar + (size_t)row * H)[q];
+            arv[4 * q] = t.x; arv[4 * q + 1] = t.y; arv[4 * q + 2] = t.z; arv[4 * q + 3] = t.w;
+        }
+#pragma unroll
+        for (int j = 0; j < H; ++j) { m[j] = -INFINITY; zs[j] = 0.f; }
+        for (int64_t p = a + tid; p < b; p += NT) {
+            const float4* alp = reinterpret_cast<const float4*>(al + (size_t)col[p] * H);
+            float4* out = reinterpret_cast<float4*>(alpha + (size_t)p * H);
+#pragma unroll
+            for (int q = 0; q < HV; ++q) {
+                const float4 t = alp[q];
+                float z[4] = {t.x + arv[4 * q], t.y + arv[4 * q + 1], t.z + arv[4 * q + 2], t.w + arv[4 * q + 3]};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    z[j] = z[j] > 0.f ? z[j] : slope * z[j];
+                    m[4 * q + j] = fmaxf(m[4 * q + j], z[j]);
+                }
+                out[q] = make_float4(z[0], z[1], z[2], z[3]);
+            }
+        }
+        reduce_heads<HV, NT, true>(m, red);
+        for (int64_t p = a + tid; p < b; p += NT) {
+            const float4* in = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
+#pragma unroll
+            for (int q = 0; q < HV; ++q) {
+                const float4 t = in[q];
+                zs[4 * q] += expf(t.x - m[4 * q]); zs[4 * q + 1] += expf(t.y - m[4 * q + 1]);
+                zs[4 * q + 2] += expf(t.z - m[4 * q + 2]); zs[4 * q + 3] += expf(t.w - m[4 * q + 3]);
+            }
+        }
+        reduce_heads<HV, NT, false>(zs, red);
+        for (int64_t p = a + tid; p < b; p += NT) {
+            float4* io = reinterpret_cast<float4*>(alpha + (size_t)p * H);
+#pragma unroll
+            for (int q = 0; q < HV; ++q) {
+                const float4 t = io[q];
+                io[q] = make_float4(expf(t.x - m[4 * q]) / zs[4 * q], expf(t.y - m[4 * q + 1]) / zs[4 * q + 1],
+                                    expf(t.z - m[4 * q + 2]) / zs[4 * q + 2], expf(t.w - m[4 * q + 3]) / zs[4 * q + 3]);
+            }
+        }
+    }
+}
+
+// backward rows: d[h] = sum_p alpha*dalpha; dz = alpha*(dalpha - d)*LeakyReLU'(z), written over dalpha; dar = sum_p dz
+template <int HV, bool LONG>
+__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
+gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
+                       const float* __restrict__ alpha, float* __restrict__ dalpha_dz, const float* __restrict__ al,
+                       const float* __restrict__ ar, float slope, float* __restrict__ dar) {
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
+    __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
+    const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
+    int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int stride = LONG ? gridDim.x : (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
+    for (; row < N; row += stride) {
+        const int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (((b - a) > SM_LONG_ROW) != LONG) continue;
+        if (b == a) {
+            if (tid < H) dar[(size_t)row * H + tid] = 0.f;
+            continue;
+        }
+        float arv[H], d[H], sdz[H];
+#pragma unroll
+        for (int q = 0; q < HV; ++q) {
+            const float4 t = reinterpret_cast<const float4*>(ar + (size_t)row * H)[q];
+            arv[4 * q] = t.x; arv[4 * q + 1] = t.y; arv[4 * q + 2] = t.z; arv[4 * q + 3] = t.w;
+        }
+#pragma unroll
+        for (int j = 0; j < H; ++j) { d[j] = 0.f; sdz[j] = 0.f; }
+        for (int64_t p = a + tid; p < b; p += NT) {
+            const float4* ap = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
+            const float4* dp = reinterpret_cast<const float4*>(dalpha_dz + (size_t)p * H);
+#pragma unroll
+            for (int q = 0; q < HV; ++q) {
+                const float4 x = ap[q], y = dp[q];
+                d[4 * q] = fmaf(x.x, y.x, d[4 * q]); d[4 * q + 1] = fmaf(x.y, y.y, d[4 * q + 1]);
+                d[4 * q + 2] = fmaf(x.z, y.z, d[4 * q + 2]); d[4 * q + 3] = fmaf(x.w, y.w, d[4 * q + 3]);
+            }
+        }
+        reduce_heads<HV, NT, false>(d, red);
+        for (int64_t p = a + tid; p < b; p += NT) {
+            const float4* ap = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
+            float4* dp = reinterpret_cast<float4*>(dalpha_dz + (size_t)p * H);
+            const float4* alp = reinterpret_cast<const float4*>(al + (size_t)col[p] * H);
+#pragma unroll
+            for (int q = 0; q < HV; ++q) {
+                const float4 x = ap[q], y = dp[q], t = alp[q];
+                const float z[4] = {t.x + arv[4 * q], t.y + arv[4 * q + 1], t.z + arv[4 * q + 2], t.w + arv[4 * q + 3]};
+                const float xa[4] = {x.x, x.y, x.z, x.w}, ya[4] = {y.x, y.y, y.z, y.w};
+                float o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    o[j] = xa[j] * (ya[j] - d[4 * q + j]) * (z[j] > 0.f ? 1.f : slope);
+                    sdz[4 * q + j] += o[j];
+                }
+                dp[q] = make_float4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        reduce_heads<HV, NT, false>(sdz, red);
+        if (tid == 0) {
+#pragma unroll
+            for (int j = 0; j < H; ++j) dar[(size_t)row * H + j] = sdz[j];
+        }
+    }
+}
+
+static int row_grid(int N, bool is_long) {
+    const int64_t want = is_long ? N : ceil_div((int64_t)N * 32, SM_BLOCK);
+    const int64_t cap = 148 * 8;
+    return (int)(want < cap ? (want > 0 ? want : 1) : cap);
+}
+
+// grid for a row-strided kernel: one warp per row up to a few waves; one block per row for long rows
+static int row_grid_pl(int N, bool is_long) {
+    const int64_t want = is_long ? N : ceil_div((int64_t)N * 32, SM_BLOCK);
+    const int64_t cap = is_long ? 148 * 2 : (int64_t)148 * 64;
+    return (int)(want < cap ? (want > 0 ? want : 1) : cap);
+}
+
+gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float slope, int H, float* alpha, cudaStream_t st) {
+    if (g->N == 0 || g->E == 0) return GNN_OK;
+    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true);
+#define GNN_GA(HV)                                                                                                    \
+    gat_alpha_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);          \
+    gat_alpha_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);
+    if (H == 4) { GNN_GA(1) } else if (H == 8) { GNN_GA(2) } else if (H == 16) { GNN_GA(4) } else if (H == 32) { GNN_GA(8) } else {
+        gat_alpha_kernel<false><<<row_grid(g->N, false), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
+        gat_alpha_kernel<true><<<row_grid(g->N, true), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
+    }
+#undef GNN_GA
+    GNN_CHECK_LAUNCH("gnn_gat_fused (attention coefficients)");
+    return GNN_OK;
+}
+
+// returns false if H is not handled here (caller falls back to its generic kernel)
+bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz, const float* al, const float* ar,
+                          float slope, int H, float* dar, cudaStream_t st) {
+    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true);
+#define GNN_GB(HV)                                                                                                               \
+    gat_rows_bwd_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);  \
+    gat_rows_bwd_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);
+    if (H == 4) { GNN_GB(1) } else if (H == 8) { GNN_GB(2) } else if (H == 16) { GNN_GB(4) } else if (H == 32) { GNN_GB(8) } else return false;
+#undef GNN_GB
+    return true;
 }
 
 }  // namespace gnn
@@ -156,13 +393,13 @@ gnn_status gnn_edge_softmax(const gnn_csr* g, const void* logits_EH, int H, gnn_
     if (g->N == 0) return GNN_OK;
     GNN_REQUIRE(g->E == 0 || (logits_EH && alpha_EH), GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
-    const int wgrid = (int)ceil_div((int64_t)g->N * 32, SM_BLOCK);
+    const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
     if (dtype == GNN_F32) {
         edge_softmax_kernel<float, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum);
-        edge_softmax_kernel<float, true><<<g->N, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum);
+        edge_softmax_kernel<float, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum);
     } else {
         edge_softmax_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum);
-        edge_softmax_kernel<__nv_bfloat16, true><<<g->N, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum);
+        edge_softmax_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum);
     }
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
@@ -176,13 +413,13 @@ gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, con
     if (g->N == 0 || g->E == 0) return GNN_OK;
     GNN_REQUIRE(alpha_EH && dAlpha_EH && dLogits_EH, GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
-    const int wgrid = (int)ceil_div((int64_t)g->N * 32, SM_BLOCK);
+    const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
     if (dtype == GNN_F32) {
         edge_softmax_backward_kernel<float, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH);
-        edge_softmax_backward_kernel<float, true><<<g->N, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH);
+        edge_softmax_backward_kernel<float, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH);
     } else {
         edge_softmax_backward_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH);
-        edge_softmax_backward_kernel<__nv_bfloat16, true><<<g->N, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH);
+        edge_softmax_backward_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH);
     }
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
