@@ -254,9 +254,14 @@ def main():
     del src_d, dst_d
     w_csr = gnn.permute_edge_data(g.eid, torch.from_numpy(wl["w"]).to(dev))
     w_csrT = gnn.permute_edge_data(g.t2f, w_csr)
-    hX = torch.from_numpy(synth.normal_f32((N * fmax,), seed, 20))
-    hR = torch.from_numpy(synth.normal_f32((N * fmax,), seed, 21))
+    # features and incoming gradients are drawn straight into pinned host memory (reused by the end-to-end leg)
+    want_e2e = not args.no_e2e
+    hX = torch.empty(N * fmax, dtype=torch.float32, pin_memory=want_e2e)
+    hR = torch.empty(N * fmax, dtype=torch.float32, pin_memory=want_e2e)
+    synth.normal_f32_into(hX.numpy(), seed, 20)
+    synth.normal_f32_into(hR.numpy(), seed, 21)
     X32, R32 = hX.to(dev), hR.to(dev)
+    wl["src"] = wl["dst"] = None  # host copies of the topology are no longer needed
     Xb, Rb = X32.to(torch.bfloat16), R32.to(torch.bfloat16)  # RNE, same bits as the host bf16 generator
     out32 = torch.empty(N * fmax, dtype=torch.float32, device=dev)
     dX32 = torch.empty(N * fmax, dtype=torch.float32, device=dev)
@@ -377,10 +382,11 @@ def run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, de
     end in pinned host memory, every case, inside the timed region.  The graph and the edge
     weights stay resident (they do not change from step to step in full-graph training)."""
     pin = dict(pin_memory=True)
-    hXp, hRp = hX.pin_memory(), hR.pin_memory()
+    hXp, hRp = hX, hR  # already pinned
     hXb, hRb = hX.to(torch.bfloat16).pin_memory(), hR.to(torch.bfloat16).pin_memory()
+    # one pinned result buffer serves both calls: the copies are ordered on the stream
     hout = torch.empty(N * fmax, dtype=torch.float32, **pin)
-    hdX = torch.empty(N * fmax, dtype=torch.float32, **pin)
+    hdX = hout
     stage = [torch.empty(N * fmax, dtype=torch.float32, device=dev) for _ in range(2)]
     h2d = d2h = 0
     calls = []

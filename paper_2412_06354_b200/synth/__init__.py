@@ -66,6 +66,13 @@ def normal_f32(shape, seed, stream=0):
     return out
 
 
+def normal_f32_into(out, seed, stream=0):
+    """Fill an existing contiguous float32 array (e.g. a view of pinned memory) with the same draws as normal_f32."""
+    assert out.dtype == np.float32 and out.flags["C_CONTIGUOUS"]
+    _load().synth_fill_normal_f32(_p(out, C.c_float), out.size, seed, stream)
+    return out
+
+
 def normal_bf16(shape, seed, stream=0):
     out = np.empty(shape, dtype=np.uint16)
     _load().synth_fill_normal_bf16(_p(out, C.c_uint16), out.size, seed, stream)
