@@ -34,7 +34,8 @@ UNIT = "edges*feat/s"
 ALL_CASES = [(F, dt) for dt in ("bf16", "f32") for F in (32, 64, 128, 256, 512)]
 FMAX = 512
 
-# DRAM bytes (read + write, GB) of one propagate_chunk_kernel launch at full size, from the single-pass ncu
+# DRAM bytes (read + write, GB) of one gnn_propagate_fused / _backward call (all its propagate_chunk_kernel
+# launches: wide rows run as 512-byte column slabs) at full size, from the single-pass ncu
 # capture summarised in profiles/propagate_sweep_full_size_dram_bytes.md.  Valid for the kernel as committed
 # with that capture; set an entry to None when the kernel changes.
 TRAFFIC_GB = {
@@ -46,38 +47,38 @@ TRAFFIC_GB = {
     "64:bf16:copy_xj:bwd": 2.08,
     "64:bf16:e_mul_xj:fwd": 2.59,
     "64:bf16:e_mul_xj:bwd": 2.59,
-    "128:bf16:copy_xj:fwd": 6.25,
-    "128:bf16:copy_xj:bwd": 6.25,
-    "128:bf16:e_mul_xj:fwd": 6.76,
-    "128:bf16:e_mul_xj:bwd": 6.76,
-    "256:bf16:copy_xj:fwd": 19.34,
-    "256:bf16:copy_xj:bwd": 19.31,
-    "256:bf16:e_mul_xj:fwd": 19.85,
-    "256:bf16:e_mul_xj:bwd": 19.82,
-    "512:bf16:copy_xj:fwd": 54.24,
-    "512:bf16:copy_xj:bwd": 54.04,
-    "512:bf16:e_mul_xj:fwd": 54.75,
-    "512:bf16:e_mul_xj:bwd": 54.55,
-    "32:f32:copy_xj:fwd": 2.02,
-    "32:f32:copy_xj:bwd": 2.02,
-    "32:f32:e_mul_xj:fwd": 2.53,
-    "32:f32:e_mul_xj:bwd": 2.53,
-    "64:f32:copy_xj:fwd": 6.49,
-    "64:f32:copy_xj:bwd": 6.48,
-    "64:f32:e_mul_xj:fwd": 7.01,
-    "64:f32:e_mul_xj:bwd": 7.0,
-    "128:f32:copy_xj:fwd": 19.44,
-    "128:f32:copy_xj:bwd": 19.4,
-    "128:f32:e_mul_xj:fwd": 19.95,
-    "128:f32:e_mul_xj:bwd": 19.91,
-    "256:f32:copy_xj:fwd": 53.97,
-    "256:f32:copy_xj:bwd": 53.77,
-    "256:f32:e_mul_xj:fwd": 54.48,
-    "256:f32:e_mul_xj:bwd": 54.28,
-    "512:f32:copy_xj:fwd": 141.37,
-    "512:f32:copy_xj:bwd": 140.14,
-    "512:f32:e_mul_xj:fwd": 141.88,
-    "512:f32:e_mul_xj:bwd": 140.64,
+    "128:bf16:copy_xj:fwd": 6.38,
+    "128:bf16:copy_xj:bwd": 6.38,
+    "128:bf16:e_mul_xj:fwd": 6.89,
+    "128:bf16:e_mul_xj:bwd": 6.89,
+    "256:bf16:copy_xj:fwd": 19.25,
+    "256:bf16:copy_xj:bwd": 19.22,
+    "256:bf16:e_mul_xj:fwd": 19.76,
+    "256:bf16:e_mul_xj:bwd": 19.73,
+    "512:bf16:copy_xj:fwd": 38.51,
+    "512:bf16:copy_xj:bwd": 38.45,
+    "512:bf16:e_mul_xj:fwd": 39.54,
+    "512:bf16:e_mul_xj:bwd": 39.48,
+    "32:f32:copy_xj:fwd": 2.01,
+    "32:f32:copy_xj:bwd": 2.01,
+    "32:f32:e_mul_xj:fwd": 2.52,
+    "32:f32:e_mul_xj:bwd": 2.52,
+    "64:f32:copy_xj:fwd": 6.44,
+    "64:f32:copy_xj:bwd": 6.44,
+    "64:f32:e_mul_xj:fwd": 6.96,
+    "64:f32:e_mul_xj:bwd": 6.95,
+    "128:f32:copy_xj:fwd": 19.35,
+    "128:f32:copy_xj:bwd": 19.32,
+    "128:f32:e_mul_xj:fwd": 19.87,
+    "128:f32:e_mul_xj:bwd": 19.83,
+    "256:f32:copy_xj:fwd": 38.74,
+    "256:f32:copy_xj:bwd": 38.67,
+    "256:f32:e_mul_xj:fwd": 39.77,
+    "256:f32:e_mul_xj:bwd": 39.7,
+    "512:f32:copy_xj:fwd": 77.53,
+    "512:f32:copy_xj:bwd": 77.37,
+    "512:f32:e_mul_xj:fwd": 79.59,
+    "512:f32:e_mul_xj:bwd": 79.42,
 }
 
 
@@ -358,7 +359,7 @@ def main():
             "config": {"workload": WORKLOAD_NAME if shrink == 0 else f"REDUCED graph (R-MAT scale {args.graph_scale}) of: " + WORKLOAD_NAME, "N": N, "E": E, "cases": [f"{F}:{dt}" for F, dt in cases],
                        "l2": "inputs larger than L2: every launch streams >= 0.5 GB of indices and a feature matrix of 154 MB to 4.9 GB",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "clocks": clocks, "gpu_launches": 4 * len(plan) * args.steps, "roofline": roofline, "per_case": per_case}
+            "clocks": clocks, "gpu_launches": args.steps * sum(4 * max(1, F * (2 if dt == "bf16" else 4) // 512) for F, dt, _, _ in plan), "roofline": roofline, "per_case": per_case}
 
     # ---- end to end through the host-buffer entry points
     if not args.no_e2e and hasattr(gnn, "propagate_fused_host"):
