@@ -103,6 +103,9 @@ static int dw_slabs(int64_t N) { return (int)(N > 0 ? ceil_div(N, DW_SLAB_ROWS) 
 bool linear_tc_supported(int64_t N, int K, int M, gnn_dtype dtype);
 gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int M, int w_transposed, gnn_dtype dtype,
                              void* Y, int* d_flag, cudaStream_t st);
+bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype);
+gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
+                              cudaStream_t st);
 bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tc_dw_partials(int64_t N);
 gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, gnn_dtype dtype, float* part, int* d_flag,
@@ -130,6 +133,7 @@ gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn
     GNN_REQUIRE(ws && ws_bytes >= 256, GNN_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes needed", who, gnn_linear_workspace(N, K, M));
     cudaStream_t st = as_stream(stream);
     if (cudaMemsetAsync(ws, 0, sizeof(int), st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed (is ws a device pointer?)", who);
+    if (linear_tma_supported(N, K, M, 0, dtype)) return linear_tma_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
     if (linear_tc_supported(N, K, M, dtype)) return linear_tc_forward(X, W, N, K, M, 0, dtype, Y, (int*)ws, st);
     if (dtype == GNN_F32)
         launch_simt<float, float, float>((const float*)X, K, 1, (const float*)W, M, 1, (float*)Y, N, M, K, K, 1, 0, st);
@@ -154,7 +158,10 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
     if (dX && N > 0) {
         GNN_REQUIRE(W, GNN_ERR_INVALID_ARG, "%s: dX needs W", who);
         // dX[n,k] = sum_m dY[n,m] * W[k,m]
-        if (linear_tc_supported(N, M, K, dtype)) {
+        if (linear_tma_supported(N, M, K, 1, dtype)) {
+            gnn_status rc = linear_tma_forward(dY, W, N, M, K, 1, dX, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (linear_tc_supported(N, M, K, dtype)) {
             gnn_status rc = linear_tc_forward(dY, W, N, M, K, 1, dtype, dX, (int*)ws, st);
             if (rc != GNN_OK) return rc;
         } else if (dtype == GNN_F32) {

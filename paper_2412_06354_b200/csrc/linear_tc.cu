@@ -15,80 +15,12 @@
 //
 // Every wait has an iteration limit: on expiry the CTA raises a status word, skips its stores,
 // still frees its tensor memory and returns.
-#include <atomic>
-
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace gnn {
 
-constexpr int TC_ROWS = 128;     // rows of X per tile = MMA M
 constexpr int TC_THREADS = 256;   // 8 warps: warp w reads accumulator lanes 32*(w%4).. and column half w/4
 constexpr int TC_THREADS2 = 256;  // dW kernel, same split
-constexpr uint32_t TC_WAIT_LIMIT = 1u << 20;
-constexpr size_t TC_SMEM_LIMIT = 200 * 1024;  // dynamic shared memory the kernels may ask for
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// 16-byte asynchronous copy global -> shared, bypassing registers; src_bytes = 0 writes zeros
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
-// shared-memory matrix descriptor, no swizzle: start address, leading/stride byte offsets (all >> 4)
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version for sm_100
-    return d;                // base offset 0, layout type 0 (no swizzle)
-}
-
-// instruction descriptor for kind::f16: D = f32, A = B = bf16, A K-major, M = 128
-__host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(b_mn_major ? 1 : 0) << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(TC_ROWS >> 4) << 24);
-}
-
-__device__ __forceinline__ void mma_bf16_ss(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t"
-        "}\n"
-        :
-        : "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-        : "memory");
-}
-
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}\n"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
-// raise a kernel's dynamic shared memory limit to 200 KB, once per (device, kernel)
-static gnn_status allow_big_smem(const char* who, const void* kernel, int which) {
-    static std::atomic<unsigned char> done[64][4];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
-    if (dev >= 0 && done[dev][which].load()) return GNN_OK;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT);
-    if (e != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: cudaFuncSetAttribute: %s", who, cudaGetErrorString(e));
-    if (dev >= 0) done[dev][which].store(1);
-    return GNN_OK;
-}
 
 // ------------------------------------------------------------------ operand tiles
 // NS = number of bf16 terms per input value (1 for bf16 input, 3 for fp32 input).  A tile holds

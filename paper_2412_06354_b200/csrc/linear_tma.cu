@@ -1,0 +1,247 @@
+// Pipelined tensor-core path of the dense node-wise transform for bf16: Y[N,Mo] = X[N,Kc] * B with
+// B = W[Kc,Mo] as stored (b_transposed = 0: Y = X*W) or the transpose of W[Mo,Kc] (b_transposed = 1:
+// dX = dY*W^T), and dW = X^T * dY.
+//
+// One persistent CTA per SM, three roles:
+//   warp 0   loader: one thread issues bulk tensor copies (TMA).  The weight matrix is fetched once
+//            per CTA; X arrives as slices of 128 rows x 64 contraction elements (128 bytes per row,
+//            128-byte swizzle, 16 KB) into a ring of shared-memory slots, each copy signalling the
+//            slot's "full" mbarrier with its byte count.
+//   warp 1   MMA issuer: one thread waits for a slice, issues its four tcgen05.mma (128 x Mo x 16,
+//            fp32 accumulator in tensor memory) and commits them to the slot's "empty" barrier, so the
+//            loader can refill the slot as soon as the tensor core has read it.  Two accumulators
+//            alternate between tiles.
+//   warps 2..9  epilogue: wait for a tile's accumulator, read it back (tcgen05.ld), round to bf16,
+//            store the rows, and hand the accumulator back.
+// The contraction is short (Kc <= 256), so the kernel is bound by reading X and writing Y; the ring
+// keeps 64-100 KB of loads in flight per SM.
+//
+// Every wait has an iteration limit: on expiry the role raises a status word and leaves its loop, the
+// other roles run into their own limits, the loader waits (bounded) for copies still in flight, and
+// the CTA frees its tensor memory and returns.
+#include <cuda.h>  // CUtensorMap and its enums; the encoder itself is looked up through the runtime
+
+#include <mutex>
+
+#include "tc_common.cuh"
+
+namespace gnn {
+
+constexpr int TM_EPI_WARPS = 8;
+constexpr int TM_THREADS = 32 * (2 + TM_EPI_WARPS);
+constexpr int TM_KB = 64;                                    // contraction elements per slice = one 128-byte swizzle row
+constexpr uint32_t TM_SLICE_BYTES = TC_ROWS * TM_KB * 2;     // 16 KB
+constexpr int TM_MAX_STAGES = 8;
+constexpr size_t TM_SMEM_MAX = 225 * 1024;                   // dynamic shared memory per CTA (227 KB less the static part)
+constexpr uint32_t SW128 = 2;                                // descriptor layout code of the 128-byte swizzle
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+struct TmaParams {
+    __nv_bfloat16* Y;  // [N,Mo]
+    int64_t N;
+    int Kc, Mo;        // contraction length, output columns
+    int b_transposed;
+    int stages;        // ring slots
+    int acc_stride;    // tensor-memory columns between the two accumulators
+    int tmem_cols;
+    int* status;
+};
+
+__global__ void __launch_bounds__(TM_THREADS, 1)
+linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, const TmaParams P) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * TM_MAX_STAGES + 5];  // full[S], empty[S], wfull, acc_full[2], acc_empty[2]
+    __shared__ uint32_t tmem_base_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Kc = P.Kc, Mo = P.Mo, S = P.stages;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
+    const int kblocks = (Kc + TM_KB - 1) / TM_KB;
+    // weight blocks: one per 64 elements of the stored matrix's contiguous dimension
+    const int wblocks = P.b_transposed ? kblocks : (Mo + 63) / 64;
+    const uint32_t wblock_bytes = (uint32_t)(P.b_transposed ? Mo : Kc) * 128u;
+    const uint32_t w0 = base, ring0 = base + (uint32_t)wblocks * wblock_bytes;
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(TM_MAX_STAGES + s); };
+    const uint32_t wfull = bar0 + 8u * (2 * TM_MAX_STAGES);
+    auto acc_full = [&](int a) { return bar0 + 8u * (uint32_t)(2 * TM_MAX_STAGES + 1 + a); };
+    auto acc_empty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * TM_MAX_STAGES + 3 + a); };
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(wfull, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), TM_EPI_WARPS); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapW)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const int64_t ntiles = (P.N + TC_ROWS - 1) / TC_ROWS;
+    bool failed = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint64_t keep = policy_evict_last(), stream = policy_evict_first();
+            mbar_arrive_expect_tx(wfull, (uint32_t)wblocks * wblock_bytes);
+            for (int b = 0; b < wblocks; ++b) tma_load_2d(w0 + (uint32_t)b * wblock_bytes, &mapW, b * 64, 0, wfull, keep);
+            uint32_t it = 0;
+            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x)
+                for (int j = 0; j < kblocks; ++j, ++it) {
+                    const int s = (int)(it % (uint32_t)S);
+                    const uint32_t use = it / (uint32_t)S;
+                    // the slot's previous contents have been consumed (first use: passes at once)
+                    if (!mbar_wait_bounded(empty(s), (use & 1u) ^ 1u)) { failed = true; break; }
+                    mbar_arrive_expect_tx(full(s), TM_SLICE_BYTES);
+                    tma_load_2d(ring0 + (uint32_t)s * TM_SLICE_BYTES, &mapX, j * TM_KB, (int)(t * TC_ROWS), full(s), stream);
+                }
+            if (failed) {
+                // do not leave while copies into this CTA's shared memory may still be in flight
+                const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+                for (uint32_t i = first; i < it; ++i) mbar_wait_bounded(full((int)(i % (uint32_t)S)), (i / (uint32_t)S) & 1u);
+                mbar_wait_bounded(wfull, 0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(Mo, P.b_transposed ? 0 : 1);
+            failed = !mbar_wait_bounded(wfull, 0);
+            uint32_t it = 0, lt = 0;
+            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++lt) {
+                const uint32_t a = lt & 1u;
+                // the epilogue has drained this accumulator (first two tiles: passes at once)
+                if (!mbar_wait_bounded(acc_empty((int)a), ((lt >> 1) & 1u) ^ 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t dacc = tmem_base + a * (uint32_t)P.acc_stride;
+                for (int j = 0; j < kblocks; ++j, ++it) {
+                    const int s = (int)(it % (uint32_t)S);
+                    if (!mbar_wait_bounded(full(s), (it / (uint32_t)S) & 1u)) { failed = true; break; }
+                    tc_fence_after();
+                    const uint32_t a_slice = ring0 + (uint32_t)s * TM_SLICE_BYTES;
+                    const int ksteps = (Kc - j * TM_KB) >= TM_KB ? TM_KB / 16 : (Kc - j * TM_KB) / 16;
+                    for (int kk = 0; kk < ksteps; ++kk) {
+                        // A: rows 128 bytes apart, groups of 8 rows 1024 bytes apart; a k-step is 32 bytes along the row
+                        const uint64_t adesc = make_smem_desc(a_slice + (uint32_t)kk * 32u, 16, 1024, SW128);
+                        uint64_t bdesc;
+                        if (P.b_transposed)  // K-major: block j holds Mo rows (output columns) of 64 contraction elements
+                            bdesc = make_smem_desc(w0 + (uint32_t)j * wblock_bytes + (uint32_t)kk * 32u, 16, 1024, SW128);
+                        else  // MN-major: block m holds Kc rows (contraction) of 64 output columns; blocks LBO apart
+                            bdesc = make_smem_desc(w0 + (uint32_t)(j * TM_KB + kk * 16) * 128u, wblock_bytes, 1024, SW128);
+                        mma_bf16_ss(dacc, adesc, bdesc, idesc, (j > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    mma_commit(empty(s));  // slot reusable once these MMAs have read it
+                }
+                if (failed) break;
+                mma_commit(acc_full((int)a));
+            }
+        }
+    } else {
+        const int ew = warp - 2, quarter = warp & 3, half = ew >> 2;  // tensor-memory lanes 32*(warp % 4)..: hardware rule
+        uint32_t lt = 0;
+        for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++lt) {
+            const uint32_t a = lt & 1u;
+            if (!mbar_wait_bounded(acc_full((int)a), (lt >> 1) & 1u)) { failed = true; break; }
+            tc_fence_after();
+            const int64_t row = t * TC_ROWS + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * (uint32_t)P.acc_stride;
+            for (int c0 = half * 16; c0 < Mo; c0 += 32) {
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (row < P.N) {
+                    float f[16];
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) f[q] = __uint_as_float(r[q]);
+                    uint4* dst = reinterpret_cast<uint4*>(P.Y + (size_t)row * Mo + c0);
+                    st_stream16(dst, Chunk<__nv_bfloat16>::pack(f));
+                    st_stream16(dst + 1, Chunk<__nv_bfloat16>::pack(f + 8));
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty((int)a));
+        }
+    }
+    if (failed) atomicExch(P.status, 7);  // GNN_ERR_TIMEOUT
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encoder() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    });
+    return fn;
+}
+
+// row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes, swizzled) x box_rows rows; out-of-range reads give zeros
+static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+    EncodeTiledFn enc = encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static size_t tma_w_bytes(int Kc, int Mo, int b_transposed) {
+    return b_transposed ? (size_t)((Kc + 63) / 64) * Mo * 128 : (size_t)((Mo + 63) / 64) * Kc * 128;
+}
+
+bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype) {
+    if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
+    if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
+    if (tma_w_bytes(Kc, Mo, b_transposed) + 2 * TM_SLICE_BYTES + 1024 > TM_SMEM_MAX) return false;
+    return encoder() != nullptr;
+}
+
+gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
+                              cudaStream_t st) {
+    const char* who = "gnn_linear (pipelined tensor-core path)";
+    GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
+    CUtensorMap mapX, mapW;
+    const int w_rows = b_transposed ? Mo : Kc, w_cols = b_transposed ? Kc : Mo;
+    if (!make_map(&mapX, X, N, Kc, TC_ROWS) || !make_map(&mapW, W, w_rows, w_cols, w_rows))
+        GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    TmaParams P;
+    P.Y = (__nv_bfloat16*)Y; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
+    const size_t wbytes = tma_w_bytes(Kc, Mo, b_transposed);
+    int stages = (int)((TM_SMEM_MAX - 1024 - wbytes) / TM_SLICE_BYTES);
+    P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
+    P.acc_stride = (Mo + 31) & ~31;
+    int cols = 32;
+    while (cols < 2 * P.acc_stride) cols <<= 1;
+    P.tmem_cols = cols;
+    const size_t smem = 1024 + wbytes + (size_t)P.stages * TM_SLICE_BYTES;
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tma_kernel, 4, TM_SMEM_MAX);
+    if (rc != GNN_OK) return rc;
+    const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
+    linear_tma_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TM_THREADS, smem, st>>>(mapX, mapW, P);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+}  // namespace gnn
