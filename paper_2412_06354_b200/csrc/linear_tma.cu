@@ -12,7 +12,8 @@
 //            loader can refill the slot as soon as the tensor core has read it.  Two accumulators
 //            alternate between tiles.
 //   warps 2..9  epilogue: wait for a tile's accumulator, read it back (tcgen05.ld), round to bf16,
-//            store the rows, and hand the accumulator back.
+//            write 32 rows x 64 columns at a time into a swizzled staging block that one bulk tensor
+//            store sends to Y (rows past N are clipped by the copy engine), and hand the accumulator back.
 // The contraction is short (Kc <= 256), so the kernel is bound by reading X and writing Y; the ring
 // keeps 64-100 KB of loads in flight per SM.
 //
@@ -31,6 +32,7 @@ constexpr int TM_EPI_WARPS = 8;
 constexpr int TM_THREADS = 32 * (2 + TM_EPI_WARPS);
 constexpr int TM_KB = 64;                                    // contraction elements per slice = one 128-byte swizzle row
 constexpr uint32_t TM_SLICE_BYTES = TC_ROWS * TM_KB * 2;     // 16 KB
+constexpr uint32_t TM_STAGING_BYTES = 32 * 128;              // per epilogue warp: 32 rows x 64 bf16 columns of Y
 constexpr int TM_MAX_STAGES = 8;
 constexpr size_t TM_SMEM_MAX = 225 * 1024;                   // dynamic shared memory per CTA (227 KB less the static part)
 constexpr uint32_t SW128 = 2;                                // descriptor layout code of the 128-byte swizzle
@@ -43,7 +45,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 
 struct TmaParams {
-    __nv_bfloat16* Y;  // [N,Mo]
     int64_t N;
     int Kc, Mo;        // contraction length, output columns
     int b_transposed;
@@ -54,7 +55,8 @@ struct TmaParams {
 };
 
 __global__ void __launch_bounds__(TM_THREADS, 1)
-linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, const TmaParams P) {
+linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                  const __grid_constant__ CUtensorMap mapY, const TmaParams P) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bars[2 * TM_MAX_STAGES + 5];  // full[S], empty[S], wfull, acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_base_slot;
@@ -65,7 +67,8 @@ linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     // weight blocks: one per 64 elements of the stored matrix's contiguous dimension
     const int wblocks = P.b_transposed ? kblocks : (Mo + 63) / 64;
     const uint32_t wblock_bytes = (uint32_t)(P.b_transposed ? Mo : Kc) * 128u;
-    const uint32_t w0 = base, ring0 = base + (uint32_t)wblocks * wblock_bytes;
+    const uint32_t w0 = base, stage0 = base + (uint32_t)wblocks * wblock_bytes;
+    const uint32_t ring0 = stage0 + TM_EPI_WARPS * TM_STAGING_BYTES;
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(TM_MAX_STAGES + s); };
@@ -80,6 +83,7 @@ linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapW)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapY)) : "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
     tc_fence_before();
@@ -146,30 +150,49 @@ linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
     } else {
         const int ew = warp - 2, quarter = warp & 3, half = ew >> 2;  // tensor-memory lanes 32*(warp % 4)..: hardware rule
+        const uint32_t stg = stage0 + (uint32_t)ew * TM_STAGING_BYTES;
         uint32_t lt = 0;
         for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++lt) {
             const uint32_t a = lt & 1u;
             if (!mbar_wait_bounded(acc_full((int)a), (lt >> 1) & 1u)) { failed = true; break; }
             tc_fence_after();
-            const int64_t row = t * TC_ROWS + quarter * 32 + lane;
+            const int64_t row0 = t * TC_ROWS + quarter * 32;  // first of this warp's 32 rows
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * (uint32_t)P.acc_stride;
-            for (int c0 = half * 16; c0 < Mo; c0 += 32) {
-                uint32_t r[16];
-                tmem_ld16(taddr + (uint32_t)c0, r);
-                tmem_ld_wait();
-                if (row < P.N) {
+            for (int cb = half; cb * 64 < Mo; cb += 2) {
+                // the previous bulk store has finished reading the staging block
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                __syncwarp();
+                const int groups = (Mo - cb * 64 >= 64 ? 64 : Mo - cb * 64) / 16;
+                for (int g = 0; g < groups; ++g) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)(cb * 64 + g * 16), r);
+                    tmem_ld_wait();
                     float f[16];
 #pragma unroll
                     for (int q = 0; q < 16; ++q) f[q] = __uint_as_float(r[q]);
-                    uint4* dst = reinterpret_cast<uint4*>(P.Y + (size_t)row * Mo + c0);
-                    st_stream16(dst, Chunk<__nv_bfloat16>::pack(f));
-                    st_stream16(dst + 1, Chunk<__nv_bfloat16>::pack(f + 8));
+                    // row = lane, 128 bytes per row; 16-byte chunk c sits at position c ^ (row % 8)
+#pragma unroll
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        const uint4 v = Chunk<__nv_bfloat16>::pack(f + 8 * h2);
+                        const uint32_t dst = stg + (uint32_t)lane * 128u + ((uint32_t)((2 * g + h2) ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && row0 < P.N) {  // rows past N are clipped by the copy engine
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                     reinterpret_cast<uint64_t>(&mapY)),
+                                 "r"(cb * 64), "r"((int)row0), "r"(stg)
+                                 : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty((int)a));
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // staging block is read, rows are written
     }
     if (failed) atomicExch(P.status, 7);  // GNN_ERR_TIMEOUT
     tc_fence_before();
@@ -214,7 +237,7 @@ static size_t tma_w_bytes(int Kc, int Mo, int b_transposed) {
 bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype) {
     if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
     if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
-    if (tma_w_bytes(Kc, Mo, b_transposed) + 2 * TM_SLICE_BYTES + 1024 > TM_SMEM_MAX) return false;
+    if (tma_w_bytes(Kc, Mo, b_transposed) + TM_EPI_WARPS * TM_STAGING_BYTES + 2 * TM_SLICE_BYTES + 1024 > TM_SMEM_MAX) return false;
     return encoder() != nullptr;
 }
 
@@ -222,24 +245,26 @@ gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, i
                               cudaStream_t st) {
     const char* who = "gnn_linear (pipelined tensor-core path)";
     GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
-    CUtensorMap mapX, mapW;
+    CUtensorMap mapX, mapW, mapY;
     const int w_rows = b_transposed ? Mo : Kc, w_cols = b_transposed ? Kc : Mo;
-    if (!make_map(&mapX, X, N, Kc, TC_ROWS) || !make_map(&mapW, W, w_rows, w_cols, w_rows))
+    if (!make_map(&mapX, X, N, Kc, TC_ROWS) || !make_map(&mapW, W, w_rows, w_cols, w_rows) ||
+        !make_map(&mapY, Y, N, Mo, 32))
         GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaParams P;
-    P.Y = (__nv_bfloat16*)Y; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
+    P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
     const size_t wbytes = tma_w_bytes(Kc, Mo, b_transposed);
-    int stages = (int)((TM_SMEM_MAX - 1024 - wbytes) / TM_SLICE_BYTES);
+    const size_t fixed = 1024 + wbytes + (size_t)TM_EPI_WARPS * TM_STAGING_BYTES;
+    int stages = (int)((TM_SMEM_MAX - fixed) / TM_SLICE_BYTES);
     P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
     P.acc_stride = (Mo + 31) & ~31;
     int cols = 32;
     while (cols < 2 * P.acc_stride) cols <<= 1;
     P.tmem_cols = cols;
-    const size_t smem = 1024 + wbytes + (size_t)P.stages * TM_SLICE_BYTES;
+    const size_t smem = fixed + (size_t)P.stages * TM_SLICE_BYTES;
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_kernel, 4, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;
     const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
-    linear_tma_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TM_THREADS, smem, st>>>(mapX, mapW, P);
+    linear_tma_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TM_THREADS, smem, st>>>(mapX, mapW, mapY, P);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
