@@ -79,14 +79,29 @@ gemm_simt_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* _
     }
 }
 
-// out[i] = sum over slabs (ascending) of part[s][i]
+// out[i] = sum over slabs of part[s][i] in a fixed order: the slabs are cut into four contiguous
+// groups, each summed in ascending order by one thread, and the four group sums are added in
+// ascending group order.  64 elements x 4 groups per block.
 template <typename TC>
-__global__ void slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __restrict__ out) {
-    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i >= n) return;
+__global__ void __launch_bounds__(256)
+slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __restrict__ out) {
+    __shared__ float gsum[4][64];
+    const int e = threadIdx.x & 63, g = threadIdx.x >> 6;
+    const int64_t i = blockIdx.x * (int64_t)64 + e;
+    const int per = (slabs + 3) / 4, z0 = g * per, z1 = min(slabs, z0 + per);
     float s = 0.f;
-    for (int z = 0; z < slabs; ++z) s += part[(size_t)z * n + i];
-    out[i] = from_f32<TC>(s);
+    if (i < n) {
+        int z = z0;
+        for (; z + 4 <= z1; z += 4) {
+            const float a = part[(size_t)z * n + i], b = part[(size_t)(z + 1) * n + i], c = part[(size_t)(z + 2) * n + i],
+                        d = part[(size_t)(z + 3) * n + i];
+            s += a; s += b; s += c; s += d;
+        }
+        for (; z < z1; ++z) s += part[(size_t)z * n + i];
+    }
+    gsum[g][e] = s;
+    __syncthreads();
+    if (g == 0 && i < n) out[i] = from_f32<TC>(((gsum[0][e] + gsum[1][e]) + gsum[2][e]) + gsum[3][e]);
 }
 
 template <typename TA, typename TB, typename TC>
@@ -106,6 +121,9 @@ gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int
 bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype);
 gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
                               cudaStream_t st);
+bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
+int linear_tma_dw_partials(int64_t N);
+gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
 bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tc_dw_partials(int64_t N);
 gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, gnn_dtype dtype, float* part, int* d_flag,
@@ -178,7 +196,11 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         float* part = (float*)((char*)ws + 256);
         int slabs = dw_slabs(N);
         const int64_t km = (int64_t)K * M;
-        if (linear_tc_dw_supported(N, K, M, dtype)) {
+        if (linear_tma_dw_supported(N, K, M, dtype)) {
+            slabs = linear_tma_dw_partials(N);
+            gnn_status rc = linear_tma_dw(X, dY, N, K, M, part, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (linear_tc_dw_supported(N, K, M, dtype)) {
             slabs = linear_tc_dw_partials(N);
             gnn_status rc = linear_tc_dw(X, dY, N, K, M, dtype, part, (int*)ws, st);
             if (rc != GNN_OK) return rc;
@@ -190,8 +212,8 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
             launch_simt<__nv_bfloat16, __nv_bfloat16, float>((const __nv_bfloat16*)X, 1, K, (const __nv_bfloat16*)dY, M, 1, part, K, M, N,
                                                            DW_SLAB_ROWS, slabs, km, st);
         }
-        if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 256), 256, 0, st>>>(part, slabs, km, (float*)dW);
-        else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 256), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW);
+        if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (float*)dW);
+        else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW);
         GNN_CHECK_LAUNCH(who);
     }
     return GNN_OK;

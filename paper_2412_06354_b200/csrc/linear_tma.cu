@@ -269,4 +269,152 @@ gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, i
     return GNN_OK;
 }
 
+// ------------------------------------------------------------------ dW = X^T * dY
+// Contraction over the N rows.  A = X^T (features x rows) and B = dY (rows x columns) are both
+// MN-major as stored, so the same 64-column x 64-row swizzled boxes serve: a pipeline slot holds 64
+// rows of X (K/64 boxes) and of dY (M/64 boxes).  The MMA warp issues, per slot, four k-steps of 16
+// rows for each half of 128 features (MMA shape 128 x M x 16) into per-CTA accumulators that stay in
+// tensor memory for the whole kernel; at the end the epilogue warps write one fp32 partial [K,M] per
+// CTA, and the partials are summed in CTA order by the caller (fixed order: deterministic).
+constexpr int DW_ROWS = 64;                         // rows of X / dY per slot
+constexpr uint32_t DW_BOX_BYTES = DW_ROWS * 128;    // one 64 x 64 bf16 box
+
+struct TmaDwParams {
+    float* part;  // [gridDim.x][K][M]
+    int64_t N;
+    int K, M;
+    int stages;
+    int tmem_cols;
+    int* status;
+};
+
+__global__ void __launch_bounds__(TM_THREADS, 1)
+linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapD, const TmaDwParams P) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * TM_MAX_STAGES + 1];  // full[S], empty[S], acc_full
+    __shared__ uint32_t tmem_base_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = P.K, M = P.M, S = P.stages;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int xboxes = K / 64, dboxes = (M + 63) / 64, halves = K / 128;
+    const uint32_t slot_bytes = (uint32_t)(xboxes + dboxes) * DW_BOX_BYTES;
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(TM_MAX_STAGES + s); };
+    const uint32_t acc_full = bar0 + 8u * (2 * TM_MAX_STAGES);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(acc_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapD)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const int64_t nchunks = (P.N + DW_ROWS - 1) / DW_ROWS;  // gridDim.x <= nchunks: every CTA has work
+    bool failed = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint64_t stream = policy_evict_first();
+            uint32_t it = 0;
+            for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x, ++it) {
+                const int s = (int)(it % (uint32_t)S);
+                if (!mbar_wait_bounded(empty(s), ((it / (uint32_t)S) & 1u) ^ 1u)) { failed = true; break; }
+                mbar_arrive_expect_tx(full(s), slot_bytes);
+                const uint32_t slot = base + (uint32_t)s * slot_bytes;
+                for (int b = 0; b < xboxes; ++b) tma_load_2d(slot + (uint32_t)b * DW_BOX_BYTES, &mapX, b * 64, (int)(c * DW_ROWS), full(s), stream);
+                for (int b = 0; b < dboxes; ++b)
+                    tma_load_2d(slot + (uint32_t)(xboxes + b) * DW_BOX_BYTES, &mapD, b * 64, (int)(c * DW_ROWS), full(s), stream);
+            }
+            if (failed) {
+                const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+                for (uint32_t i = first; i < it; ++i) mbar_wait_bounded(full((int)(i % (uint32_t)S)), (i / (uint32_t)S) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(M, 1, 1);  // A and B both MN-major
+            uint32_t it = 0;
+            for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x, ++it) {
+                const int s = (int)(it % (uint32_t)S);
+                if (!mbar_wait_bounded(full(s), (it / (uint32_t)S) & 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t sa = base + (uint32_t)s * slot_bytes, sb = sa + (uint32_t)xboxes * DW_BOX_BYTES;
+                for (int h = 0; h < halves; ++h)
+                    for (int kk = 0; kk < DW_ROWS / 16; ++kk) {
+                        // rows (contraction) are 128 bytes apart, groups of 8 rows 1024 bytes, blocks of 64 features / columns one box
+                        const uint64_t adesc = make_smem_desc(sa + (uint32_t)(2 * h) * DW_BOX_BYTES + (uint32_t)kk * 2048u, DW_BOX_BYTES, 1024, SW128);
+                        const uint64_t bdesc = make_smem_desc(sb + (uint32_t)kk * 2048u, DW_BOX_BYTES, 1024, SW128);
+                        mma_bf16_ss(tmem_base + (uint32_t)(h * M), adesc, bdesc, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    }
+                mma_commit(empty(s));
+            }
+            if (!failed) mma_commit(acc_full);
+        }
+    } else {
+        const int ew = warp - 2, quarter = warp & 3, half = ew >> 2;
+        if (!mbar_wait_bounded(acc_full, 0)) {
+            failed = true;
+        } else {
+            tc_fence_after();
+            float* part = P.part + (size_t)blockIdx.x * K * M;
+            for (int h = 0; h < halves; ++h) {
+                const int krow = h * 128 + quarter * 32 + lane;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * M);
+                for (int c0 = half * 16; c0 < M; c0 += 32) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    float4* dst = reinterpret_cast<float4*>(part + (size_t)krow * M + c0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                                             __uint_as_float(r[4 * q + 3]));
+                }
+            }
+        }
+    }
+    if (failed) atomicExch(P.status, 7);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+}
+
+bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
+    if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
+    if ((K != 128 && K != 256) || M % 16 != 0 || M < 16 || M > 256) return false;
+    return encoder() != nullptr;
+}
+
+int linear_tma_dw_partials(int64_t N) {
+    const int64_t nchunks = (N + DW_ROWS - 1) / DW_ROWS;
+    return (int)(nchunks < 148 ? (nchunks > 0 ? nchunks : 1) : 148);
+}
+
+// writes linear_tma_dw_partials(N) fp32 partials [K,M] to part
+gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
+    const char* who = "gnn_linear_backward (pipelined tensor-core dW)";
+    GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
+    CUtensorMap mapX, mapD;
+    if (!make_map(&mapX, X, N, K, DW_ROWS) || !make_map(&mapD, dY, N, M, DW_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    TmaDwParams P;
+    P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
+    const size_t slot = (size_t)(K / 64 + (M + 63) / 64) * DW_BOX_BYTES;
+    int stages = (int)((TM_SMEM_MAX - 1024) / slot);
+    P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
+    int cols = 32;
+    while (cols < M * (K / 128)) cols <<= 1;
+    P.tmem_cols = cols;
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tma_dw_kernel, 5, TM_SMEM_MAX);
+    if (rc != GNN_OK) return rc;
+    linear_tma_dw_kernel<<<linear_tma_dw_partials(N), TM_THREADS, 1024 + (size_t)P.stages * slot, st>>>(mapX, mapD, P);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
 }  // namespace gnn
