@@ -112,8 +112,10 @@ static void launch_simt(const TA* A, int64_t sam, int64_t sak, const TB* B, int6
     gemm_simt_kernel<TA, TB, TC><<<grid, 256, 0, st>>>(A, sam, sak, B, sbk, sbn, C, Mr, Nc, Kd, k_per_slab, slab_stride);
 }
 
-constexpr int DW_SLAB_ROWS = 4096;  // rows of X / dY per partial of dW
-static int dw_slabs(int64_t N) { return (int)(N > 0 ? ceil_div(N, DW_SLAB_ROWS) : 1); }
+// FFMA dW: rows of X / dY per partial.  128 rows while that gives at most 148 partials (small inputs
+// still spread over many blocks), otherwise 4096.
+static int dw_slab_rows(int64_t N) { return N <= 148 * 128 ? 128 : 4096; }
+static int dw_slabs(int64_t N) { return (int)(N > 0 ? ceil_div(N, dw_slab_rows(N)) : 1); }
 
 bool linear_tc_supported(int64_t N, int K, int M, gnn_dtype dtype);
 gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int M, int w_transposed, gnn_dtype dtype,
@@ -207,10 +209,10 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         } else if (N == 0) {
             if (cudaMemsetAsync(part, 0, (size_t)km * 4, st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed", who);
         } else if (dtype == GNN_F32) {
-            launch_simt<float, float, float>((const float*)X, 1, K, (const float*)dY, M, 1, part, K, M, N, DW_SLAB_ROWS, slabs, km, st);
+            launch_simt<float, float, float>((const float*)X, 1, K, (const float*)dY, M, 1, part, K, M, N, dw_slab_rows(N), slabs, km, st);
         } else {
             launch_simt<__nv_bfloat16, __nv_bfloat16, float>((const __nv_bfloat16*)X, 1, K, (const __nv_bfloat16*)dY, M, 1, part, K, M, N,
-                                                           DW_SLAB_ROWS, slabs, km, st);
+                                                           dw_slab_rows(N), slabs, km, st);
         }
         if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (float*)dW);
         else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW);

@@ -104,6 +104,21 @@ def _p(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+def _pi(t, dtype, name):
+    """Pointer of an index tensor, after checking its element type (the C ABI cannot)."""
+    if t is None:
+        return None
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if t.numel() and not t.is_contiguous():
+        raise TypeError(f"{name} must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _pf32(t, name):
+    return _pi(t, torch.float32, name)
+
+
 def _dtype(t):
     if t.dtype == torch.float32:
         return F32
@@ -150,7 +165,7 @@ def coo_to_csr(N, src, dst, ws=None) -> Graph:
     need = load().gnn_coo_to_csr_workspace(N, E)
     if ws is None:
         ws = torch.empty(need, dtype=torch.uint8, device=src.device)
-    _check(load().gnn_coo_to_csr(N, E, _p(src), _p(dst), g.ref, _p(ws), ws.numel(), _stream()))
+    _check(load().gnn_coo_to_csr(N, E, _pi(src, torch.int32, "src"), _pi(dst, torch.int32, "dst"), g.ref, _p(ws), ws.numel(), _stream()))
     return g
 
 
@@ -164,7 +179,7 @@ def add_self_loops(N, src, dst):
     E = src.numel()
     so = torch.empty(E + N, dtype=torch.int32, device=src.device)
     do = torch.empty(E + N, dtype=torch.int32, device=src.device)
-    _check(load().gnn_add_self_loops(N, E, _p(src), _p(dst), _p(so), _p(do), _stream()))
+    _check(load().gnn_add_self_loops(N, E, _pi(src, torch.int32, "src"), _pi(dst, torch.int32, "dst"), _p(so), _p(do), _stream()))
     return so, do
 
 
@@ -173,7 +188,7 @@ def gcn_norm(g: Graph, w_csr=None, want_T=True):
     deg = torch.empty(g.N, dtype=torch.float32, device=dev)
     coef = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev)
     coefT = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev) if want_T else None
-    _check(load().gnn_gcn_norm(g.ref, _p(w_csr), _p(deg), _p(coef), _p(coefT), _stream()))
+    _check(load().gnn_gcn_norm(g.ref, _pf32(w_csr, "w_csr"), _p(deg), _p(coef), _p(coefT), _stream()))
     return deg, coef[:g.E], (coefT[:g.E] if want_T else None)
 
 
@@ -183,7 +198,7 @@ def permute_edge_data(perm, x, out=None):
     width = x.numel() // max(E, 1) if E else 1
     if out is None:
         out = torch.empty_like(x)
-    _check(load().gnn_permute_edge_data(_p(perm), E, max(width, 1), x.element_size(), _p(x), _p(out), _stream()))
+    _check(load().gnn_permute_edge_data(_pi(perm, torch.int32, "perm"), E, max(width, 1), x.element_size(), _p(x), _p(out), _stream()))
     return out
 
 
@@ -204,7 +219,7 @@ def propagate_fused(g: Graph, X, w_csr=None, op="sum", out=None, argmax=None, ws
     if ws is None:
         ws = torch.empty(propagate_fused_workspace(g.E, F, opc), dtype=torch.uint8, device=X.device)
     msg = COPY_XJ if w_csr is None else E_MUL_XJ
-    _check(load().gnn_propagate_fused(g.ref, msg, opc, _p(X), _p(w_csr), F, _dtype(X), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    _check(load().gnn_propagate_fused(g.ref, msg, opc, _p(X), _pf32(w_csr, "w_csr"), F, _dtype(X), _p(out), _pi(argmax, torch.int32, "argmax"), _p(ws), ws.numel(), _stream()))
     return (out, argmax) if opc in (MAX, MIN) else out
 
 
@@ -221,7 +236,7 @@ def propagate_fused_backward(g: Graph, dOut, op="sum", X=None, w_csrT=None, argm
     if ws is None:
         ws = torch.empty(propagate_fused_workspace(g.E, F, opc), dtype=torch.uint8, device=dOut.device)
     msg = COPY_XJ if (w_csrT is None) else E_MUL_XJ
-    _check(load().gnn_propagate_fused_backward(g.ref, msg, opc, _p(dOut), _p(X), _p(w_csrT), _p(argmax), F, _dtype(dOut),
+    _check(load().gnn_propagate_fused_backward(g.ref, msg, opc, _p(dOut), _p(X), _pf32(w_csrT, "w_csrT"), _pi(argmax, torch.int32, "argmax"), F, _dtype(dOut),
                                                _p(dX if want_dX else None), _p(dW if want_dW else None), _p(ws), ws.numel(), _stream()))
     return (dX if want_dX else None), (dW[:g.E] if want_dW else None)
 
@@ -230,7 +245,7 @@ def propagate_fused_host(g: Graph, h_X, w_csr, op, h_out, d_in, d_out, ws, argma
     """Host-buffer forward: h_X, h_out are (pinned) host tensors; d_in, d_out device staging."""
     F = h_X.shape[1]
     msg = COPY_XJ if w_csr is None else E_MUL_XJ
-    _check(load().gnn_propagate_fused_host(g.ref, msg, _op(op), _p(h_X), _p(w_csr), F, _dtype(h_X), _p(h_out), _p(argmax),
+    _check(load().gnn_propagate_fused_host(g.ref, msg, _op(op), _p(h_X), _pf32(w_csr, "w_csr"), F, _dtype(h_X), _p(h_out), _pi(argmax, torch.int32, "argmax"),
                                            _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
     return h_out
 
@@ -238,7 +253,7 @@ def propagate_fused_host(g: Graph, h_X, w_csr, op, h_out, d_in, d_out, ws, argma
 def propagate_fused_backward_host(g: Graph, h_dOut, op, w_csrT, h_dX, d_in, d_out, ws, argmax=None):
     F = h_dOut.shape[1]
     msg = COPY_XJ if w_csrT is None else E_MUL_XJ
-    _check(load().gnn_propagate_fused_backward_host(g.ref, msg, _op(op), _p(h_dOut), _p(w_csrT), _p(argmax), F, _dtype(h_dOut),
+    _check(load().gnn_propagate_fused_backward_host(g.ref, msg, _op(op), _p(h_dOut), _pf32(w_csrT, "w_csrT"), _pi(argmax, torch.int32, "argmax"), F, _dtype(h_dOut),
                                                     _p(h_dX), _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
     return h_dX
 
@@ -255,7 +270,7 @@ def gather(idx, X, out=None):
     E, F = idx.numel(), X.shape[1]
     if out is None:
         out = torch.empty((E, F), dtype=X.dtype, device=X.device)
-    _check(load().gnn_gather(_p(idx), E, _p(X), X.shape[0], F, _dtype(X), _p(out), _stream()))
+    _check(load().gnn_gather(_pi(idx, torch.int32, "idx"), E, _p(X), X.shape[0], F, _dtype(X), _p(out), _stream()))
     return out
 
 
@@ -286,7 +301,7 @@ def aggregate(g: Graph, m_EF, op="sum", ws=None):
     out = torch.empty((g.N, F), dtype=m_EF.dtype, device=m_EF.device)
     argmax = torch.empty((g.N, F), dtype=torch.int32, device=m_EF.device) if opc in (MAX, MIN) else None
     ws = _ws(g.E, F, opc, m_EF.device, ws)
-    _check(load().gnn_aggregate(g.ref, opc, _p(m_EF), F, _dtype(m_EF), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    _check(load().gnn_aggregate(g.ref, opc, _p(m_EF), F, _dtype(m_EF), _p(out), _pi(argmax, torch.int32, "argmax"), _p(ws), ws.numel(), _stream()))
     return (out, argmax) if opc in (MAX, MIN) else out
 
 
@@ -294,7 +309,7 @@ def aggregate_backward(g: Graph, dOut, op="sum", argmax=None):
     dOut = _dev(dOut)
     F = dOut.shape[1]
     dm = torch.empty((max(g.E, 1), F), dtype=dOut.dtype, device=dOut.device)
-    _check(load().gnn_aggregate_backward(g.ref, _op(op), _p(dOut), _p(argmax), F, _dtype(dOut), _p(dm), _stream()))
+    _check(load().gnn_aggregate_backward(g.ref, _op(op), _p(dOut), _pi(argmax, torch.int32, "argmax"), F, _dtype(dOut), _p(dm), _stream()))
     return dm[:g.E]
 
 
@@ -320,7 +335,7 @@ def graph_ptr_from_ids(graph_id, G):
     N = graph_id.numel()
     gptr = torch.empty(G + 1, dtype=torch.int64, device=graph_id.device)
     ws = torch.empty(256, dtype=torch.uint8, device=graph_id.device)
-    _check(load().gnn_graph_ptr_from_ids(_p(graph_id), N, G, _p(gptr), _p(ws), ws.numel(), _stream()))
+    _check(load().gnn_graph_ptr_from_ids(_pi(graph_id, torch.int32, "graph_id"), N, G, _p(gptr), _p(ws), ws.numel(), _stream()))
     return gptr
 
 
@@ -331,7 +346,7 @@ def reduce_nodes(graph_ptr, X, op="mean", ws=None):
     out = torch.empty((G, F), dtype=X.dtype, device=X.device)
     argmax = torch.empty((G, F), dtype=torch.int32, device=X.device) if opc in (MAX, MIN) else None
     ws = _ws(N, F, opc, X.device, ws)
-    _check(load().gnn_reduce_nodes(_p(graph_ptr), G, N, opc, _p(X), F, _dtype(X), _p(out), _p(argmax), _p(ws), ws.numel(), _stream()))
+    _check(load().gnn_reduce_nodes(_pi(graph_ptr, torch.int64, "graph_ptr"), G, N, opc, _p(X), F, _dtype(X), _p(out), _pi(argmax, torch.int32, "argmax"), _p(ws), ws.numel(), _stream()))
     return (out, argmax) if opc in (MAX, MIN) else out
 
 
@@ -339,7 +354,7 @@ def reduce_nodes_backward(graph_ptr, dOut, N, op="mean", argmax=None):
     dOut = _dev(dOut)
     G, F = dOut.shape
     dX = torch.empty((N, F), dtype=dOut.dtype, device=dOut.device)
-    _check(load().gnn_reduce_nodes_backward(_p(graph_ptr), G, N, _op(op), _p(dOut), _p(argmax), F, _dtype(dOut), _p(dX), _stream()))
+    _check(load().gnn_reduce_nodes_backward(_pi(graph_ptr, torch.int64, "graph_ptr"), G, N, _op(op), _p(dOut), _pi(argmax, torch.int32, "argmax"), F, _dtype(dOut), _p(dX), _stream()))
     return dX
 
 
@@ -389,7 +404,7 @@ def propagate_fused_static(g: Graph, X, w_csr=None, op="sum", out=None, argmax=N
     if opc in (MAX, MIN) and argmax is None:
         argmax = torch.empty((g.N, F), dtype=torch.int32, device=X.device)
     msg = COPY_XJ if w_csr is None else E_MUL_XJ
-    _check(load().gnn_propagate_fused_static(g.ref, msg, opc, _p(X), _p(w_csr), F, _dtype(X), _p(out), _p(argmax), _stream()))
+    _check(load().gnn_propagate_fused_static(g.ref, msg, opc, _p(X), _pf32(w_csr, "w_csr"), F, _dtype(X), _p(out), _pi(argmax, torch.int32, "argmax"), _stream()))
     return (out, argmax) if opc in (MAX, MIN) else out
 
 

@@ -3,6 +3,8 @@ import ctypes
 import os
 import re
 
+import pytest
+
 from paper_2412_06354_b200 import build, gnn
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -43,3 +45,15 @@ def test_argument_errors_are_reported_before_any_launch():
     assert lib.gnn_add_self_loops(3, 2, None, None, None, None, None) == 1
     assert lib.gnn_permute_edge_data(None, 5, 1, 3, None, None, None) == 1
     assert lib.gnn_degree(None, 0, None, None, None) == 1
+
+
+def test_binding_rejects_wrong_index_dtype():
+    """The C ABI takes raw pointers, so the binding checks the element type of index tensors."""
+    import torch
+    from paper_2412_06354_b200 import gnn
+    with pytest.raises(TypeError):
+        gnn._pi(torch.zeros(3, dtype=torch.int32), torch.int64, "graph_ptr")
+    with pytest.raises(TypeError):
+        gnn._pf32(torch.zeros(3, dtype=torch.float64), "w_csr")
+    assert gnn._pi(None, torch.int32, "argmax") is None
+    assert gnn._pi(torch.zeros(3, dtype=torch.int32), torch.int32, "src") is not None
