@@ -436,6 +436,264 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
     }
 }
 
+// ------------------------------------------------------------------ flat variant for short rows
+// Sum / mean over graphs whose rows are mostly much shorter than a chunk (citation-style graphs:
+// a handful of edges per row).  Walking such rows one at a time leaves one or two gathers in flight
+// per lane group.  Here the gathers do not depend on the row structure:
+//   1. the warp stages its 256 positions (gathered row, multiplier) and marks where rows start; a
+//      prefix maximum gives every position the index of its row's start entry (row id and length
+//      are kept per start entry);
+//   2. each lane group takes a contiguous run of 256/NG positions and issues U = 8 independent
+//      16-byte gathers at a time; the accumulator is flushed whenever the start entry changes;
+//   3. rows cut by a run boundary are stitched inside the warp in run order (through shared
+//      memory), rows cut by the chunk boundary leave the same head / tail partials as the
+//      row-walking kernel, so the same fix-up pass finishes them.
+// Empty rows are zero-filled by the chunk after whose last position they come (chunk 0 also takes
+// the leading ones).  All orders are fixed functions of (E, F, dtype).
+constexpr int FL_WARPS = 4;
+constexpr int FL_U = 8;
+
+template <int EPC>
+struct FlatSmem {
+    int4 e[PF_SLAB];         // x: gathered row, y: start entry of the position's row, z: multiplier
+    int32_t srow[PF_SLAB];   // [k] row starting at position k of the chunk ([0]: the row holding position 0)
+    int32_t sdeg[PF_SLAB];   // [k] its length
+    float head[32 * EPC];    // per lane: partial of the run's first row when that row began before the run
+    float tail[32 * EPC];    // per lane: partial of the run's last row when it continues past the run
+    int32_t hk[8], hclosed[8], tk[8];  // per run: start entries of those rows (-1: none), head row ends in the run
+};
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(FL_WARPS * 32, 6)
+propagate_flat_kernel(const PropParams P) {
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, L = PF_SLAB / NG, U = FL_U;
+    __shared__ FlatSmem<EPC> s_all[FL_WARPS];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int64_t c = (int64_t)blockIdx.x * FL_WARPS + wib;
+    if (c >= P.nchunks) return;
+    FlatSmem<EPC>& S = s_all[wib];
+    const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
+    const int64_t cs = c * PF_SLAB;
+    const int n = (int)((cs + PF_SLAB < P.E ? cs + PF_SLAB : P.E) - cs);  // 1..256 positions
+    const int g = lane / LPR, li = lane % LPR;
+    const bool col_lane = li < P.nvec;  // lanes past a narrow row gather chunk 0 and never store
+    char* const outb = reinterpret_cast<char*>(P.out);
+
+    // ---- 1a. the row holding position cs: largest r with rowptr[r] <= cs (32-way search)
+    int lo = 0, hi = P.N;  // rowptr[lo] <= cs < rowptr[hi]
+    while (hi - lo > 1) {
+        const int step = (hi - lo + 31) / 32;
+        const int idx = min(lo + (lane + 1) * step, hi);
+        const bool le = idx < hi && P.rowptr[idx] <= cs;
+        const int k = __popc(__ballot_sync(0xffffffffu, le));
+        const int nlo = lo + k * step;
+        hi = min(nlo + step, hi);
+        lo = nlo;
+    }
+    const int cur0 = lo;
+    const int64_t rs0 = P.rowptr[cur0], re0 = P.rowptr[cur0 + 1];
+    const bool row0_before = rs0 < cs;
+    const int end0 = (int)((re0 - cs) < (int64_t)PF_SLAB + 1 ? (re0 - cs) : (int64_t)PF_SLAB + 1);  // relative end of row cur0, capped
+
+    // ---- 1b. stage gathered rows and multipliers; start entries default to 0
+    for (int i = lane; i < n; i += 32) {
+        const int cc = P.col ? ld_hint_i32(P.col + cs + i, pol_stream) : (int)(cs + i);
+        float w = P.w ? ld_hint_f32(P.w + cs + i, pol_stream) : 1.0f;
+        if (P.gscale_rowptr) {
+            const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
+            w = w / (float)(d > 1 ? d : 1);
+        }
+        S.e[i] = make_int4(cc, 0, __float_as_int(w), 0);
+    }
+    if (lane == 0) { S.srow[0] = cur0; S.sdeg[0] = (int)((re0 - rs0) < 0x7fffffff ? (re0 - rs0) : 0x7fffffff); }
+    if (lane < 8) { S.hk[lane] = -1; S.hclosed[lane] = 0; S.tk[lane] = -1; }
+    __syncwarp();
+
+    // ---- 1c. rows after cur0 that start in (cs, cs+n]: mark non-empty ones, zero-fill empty ones
+    if (c == 0)  // leading empty rows
+        for (int r = 0; r < cur0; ++r)
+            for (int ci = lane; ci < P.nvec; ci += 32) st_stream16(outb + (size_t)r * P.out_ld + (size_t)ci * 16, make_uint4(0, 0, 0, 0));
+    for (int rb = cur0 + 1;; rb += 32) {
+        const int r = rb + lane;
+        int64_t rs = 0, re = 0;
+        bool live = false;
+        if (r < P.N) {
+            rs = P.rowptr[r];
+            live = rs <= cs + n;  // rows starting exactly at the chunk end: only their empty ones are ours
+            if (live) re = P.rowptr[r + 1];
+        }
+        const bool empty = live && re == rs;
+        if (live && !empty && rs < cs + n) {
+            const int k = (int)(rs - cs);
+            S.srow[k] = r;
+            S.sdeg[k] = (int)((re - rs) < 0x7fffffff ? (re - rs) : 0x7fffffff);
+            S.e[k].y = k;
+        }
+        unsigned em = __ballot_sync(0xffffffffu, empty);
+        while (em) {
+            const int bit = __ffs(em) - 1;
+            em &= em - 1;
+            for (int ci = lane; ci < P.nvec; ci += 32)
+                st_stream16(outb + (size_t)(rb + bit) * P.out_ld + (size_t)ci * 16, make_uint4(0, 0, 0, 0));
+        }
+        // rowptr is non-decreasing: once a lane is past the chunk (or past the last row) so are all later rows
+        if (!__all_sync(0xffffffffu, live)) break;
+    }
+    __syncwarp();
+
+    // ---- 1d. prefix maximum of the start marks: lane owns positions 8*lane .. 8*lane+7
+    {
+        int m[8];
+        int run = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = lane * 8 + q;
+            const int v = i < n ? S.e[i].y : 0;
+            run = max(run, v);
+            m[q] = run;
+        }
+        int incl = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl = max(incl, t);
+        }
+        int before = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) before = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = lane * 8 + q;
+            if (i < n) S.e[i].y = max(before, m[q]);
+        }
+    }
+    __syncwarp();
+
+    // ---- 2. gather: run [a, b) of this lane group
+    const int a = g * L, b = min(a + L, n);
+    const char* Xl = reinterpret_cast<const char*>(P.X) + (size_t)(col_lane ? li : 0) * 16;
+    float acc[EPC];
+#pragma unroll
+    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+    int curk = -1;
+    // a finished row segment [.., end) of start entry k, seen by lane group g
+    auto flush = [&](int k) {
+        const bool began_before = k < a || (k == 0 && a == 0 && row0_before);
+        if (began_before) {  // the run's first row, begun in an earlier run or chunk
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) S.head[lane * EPC + j] = acc[j];
+            if (li == 0) { S.hk[g] = k; S.hclosed[g] = 1; }
+        } else if (col_lane) {
+            float v[EPC];
+            const float d = (float)max(S.sdeg[k], 1);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) v[j] = P.mean ? acc[j] / d : acc[j];
+            st_stream16(outb + (size_t)S.srow[k] * P.out_ld + (size_t)li * 16, Chunk<T>::pack(v));
+        }
+    };
+    for (int i = a; i < b; i += U) {
+        uint4 buf[U];
+        const int nu = min(U, b - i);  // U except at the ragged end of the last chunk
+        if (nu == U) {
+            int cols[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) cols[u] = S.e[i + u].x;
+#pragma unroll
+            for (int u = 0; u < U; ++u) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
+        } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (u < nu) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)S.e[i + u].x * P.x_ld, pol_keep);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (u >= nu) break;
+            const int4 e = S.e[i + u];
+            if (e.y != curk) {
+                if (curk >= 0) flush(curk);
+                curk = e.y;
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+            }
+            float x[EPC];
+            Chunk<T>::unpack(buf[u], x);
+            const float w = __int_as_float(e.z);
+#pragma unroll
+            for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], w, w);
+        }
+    }
+    if (curk >= 0) {  // the run's last row
+        const int end = curk == 0 ? end0 : curk + min(S.sdeg[curk], PF_SLAB + 1);
+        if (end <= b) {
+            flush(curk);
+        } else {  // continues past the run
+            const bool began_before = curk < a || (curk == 0 && a == 0 && row0_before);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) (began_before ? S.head : S.tail)[lane * EPC + j] = acc[j];
+            if (li == 0) {
+                if (began_before) { S.hk[g] = curk; S.hclosed[g] = 0; }
+                else S.tk[g] = curk;
+            }
+        }
+    }
+    __syncwarp();
+
+    // ---- 3. stitch the runs in order; lanes 0..LPR-1 each own one 16-byte column
+    int32_t tail_row = -1;
+    if (lane < LPR) {
+        float carry[EPC];
+        bool have = false, before_chunk = false;
+        int ck = -1;
+        auto write_partial = [&](int which) {
+            if (!col_lane) return;
+            float* pv = P.part_val + ((size_t)c * 2 + which) * P.F + (size_t)lane * EPC;
+#pragma unroll
+            for (int j = 0; j < EPC; j += 4) *reinterpret_cast<float4*>(pv + j) = make_float4(carry[j], carry[j + 1], carry[j + 2], carry[j + 3]);
+        };
+        for (int gg = 0; gg < NG; ++gg) {
+            const int hk = S.hk[gg];
+            if (hk >= 0) {
+                const float* h = S.head + (gg * LPR + lane) * EPC;
+                if (have) {
+#pragma unroll
+                    for (int j = 0; j < EPC; ++j) carry[j] += h[j];
+                } else {  // only the chunk's first run can begin without a carry
+#pragma unroll
+                    for (int j = 0; j < EPC; ++j) carry[j] = h[j];
+                    before_chunk = true;
+                    have = true;
+                }
+                ck = hk;
+                if (S.hclosed[gg]) {
+                    if (before_chunk) {
+                        write_partial(0);
+                    } else if (col_lane) {
+                        float v[EPC];
+                        const float d = (float)max(S.sdeg[ck], 1);
+#pragma unroll
+                        for (int j = 0; j < EPC; ++j) v[j] = P.mean ? carry[j] / d : carry[j];
+                        st_stream16(outb + (size_t)S.srow[ck] * P.out_ld + (size_t)lane * 16, Chunk<T>::pack(v));
+                    }
+                    have = false;
+                }
+            }
+            const int tk = S.tk[gg];
+            if (tk >= 0) {
+                const float* t = S.tail + (gg * LPR + lane) * EPC;
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) carry[j] = t[j];
+                have = true;
+                before_chunk = false;
+                ck = tk;
+            }
+        }
+        if (have) {  // the row continues in the next chunk
+            write_partial(before_chunk ? 0 : 1);
+            if (!before_chunk) tail_row = S.srow[ck];
+        }
+    }
+    if (lane == 0) P.tail_row[c] = tail_row;
+}
+
 // ------------------------------------------------------------------ edge-weight gradient (SDDMM)
 // dW[p] = scale(i) * <X[col[p],:], dOut[i,:]> for p in row i.  Same chunking; every edge is
 // independent, so no partials.  The dOut row stays in registers along the row.
@@ -570,8 +828,27 @@ static void launch_chunks(const PropParams& P, int lpr, int vpl, cudaStream_t st
     propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
 }
 
+// sums over rows of at most 512 bytes on graphs small enough for one-slab chunks: the flat kernel
+template <typename T>
+static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
+    const int grid = (int)ceil_div(P.nchunks, FL_WARPS);
+    const int thr = FL_WARPS * 32;
+    switch (lpr) {
+        case 4: propagate_flat_kernel<T, 4><<<grid, thr, 0, st>>>(P); break;
+        case 8: propagate_flat_kernel<T, 8><<<grid, thr, 0, st>>>(P); break;
+        case 16: propagate_flat_kernel<T, 16><<<grid, thr, 0, st>>>(P); break;
+        default: propagate_flat_kernel<T, 32><<<grid, thr, 0, st>>>(P); break;
+    }
+    const int64_t threads = P.nchunks * P.nvec;
+    propagate_fixup_kernel<T, MODE_SUM><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
+}
+
 template <typename T>
 static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
+    if (mode == MODE_SUM && vpl == 1 && P.chunk == PF_SLAB && P.E > 0) {
+        launch_flat<T>(P, lpr, st);
+        return;
+    }
     switch (mode) {
         case MODE_SUM: launch_chunks<T, MODE_SUM>(P, lpr, vpl, st); break;
         case MODE_MAX: launch_chunks<T, MODE_MAX>(P, lpr, vpl, st); break;
