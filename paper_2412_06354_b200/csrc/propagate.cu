@@ -457,7 +457,8 @@ template <int EPC>
 struct FlatSmem {
     int4 e[PF_SLAB];         // x: gathered row, y: start entry of the position's row, z: multiplier
     int32_t srow[PF_SLAB];   // [k] row starting at position k of the chunk ([0]: the row holding position 0)
-    int32_t sdeg[PF_SLAB];   // [k] its length
+    int32_t send[PF_SLAB];   // [k] its end, as a position of the chunk, capped at PF_SLAB + 1
+    float sinv[PF_SLAB];     // [k] factor of the finished row: 1, or 1 / length for the mean
     float head[32 * EPC];    // per lane: partial of the run's first row when that row began before the run
     float tail[32 * EPC];    // per lane: partial of the run's last row when it continues past the run
     int32_t hk[8], hclosed[8], tk[8];  // per run: start entries of those rows (-1: none), head row ends in the run
@@ -493,7 +494,8 @@ propagate_flat_kernel(const PropParams P) {
     const int cur0 = lo;
     const int64_t rs0 = P.rowptr[cur0], re0 = P.rowptr[cur0 + 1];
     const bool row0_before = rs0 < cs;
-    const int end0 = (int)((re0 - cs) < (int64_t)PF_SLAB + 1 ? (re0 - cs) : (int64_t)PF_SLAB + 1);  // relative end of row cur0, capped
+    auto rel_end = [&](int64_t re) { return (int)((re - cs) < (int64_t)PF_SLAB + 1 ? (re - cs) : (int64_t)PF_SLAB + 1); };
+    auto row_factor = [&](int64_t len) { return P.mean ? 1.0f / (float)(len > 1 ? len : 1) : 1.0f; };
 
     // ---- 1b. stage gathered rows and multipliers; start entries default to 0
     for (int i = lane; i < n; i += 32) {
@@ -505,7 +507,7 @@ propagate_flat_kernel(const PropParams P) {
         }
         S.e[i] = make_int4(cc, 0, __float_as_int(w), 0);
     }
-    if (lane == 0) { S.srow[0] = cur0; S.sdeg[0] = (int)((re0 - rs0) < 0x7fffffff ? (re0 - rs0) : 0x7fffffff); }
+    if (lane == 0) { S.srow[0] = cur0; S.send[0] = rel_end(re0); S.sinv[0] = row_factor(re0 - rs0); }
     if (lane < 8) { S.hk[lane] = -1; S.hclosed[lane] = 0; S.tk[lane] = -1; }
     __syncwarp();
 
@@ -526,7 +528,8 @@ propagate_flat_kernel(const PropParams P) {
         if (live && !empty && rs < cs + n) {
             const int k = (int)(rs - cs);
             S.srow[k] = r;
-            S.sdeg[k] = (int)((re - rs) < 0x7fffffff ? (re - rs) : 0x7fffffff);
+            S.send[k] = rel_end(re);
+            S.sinv[k] = row_factor(re - rs);
             S.e[k].y = k;
         }
         unsigned em = __ballot_sync(0xffffffffu, empty);
@@ -575,18 +578,20 @@ propagate_flat_kernel(const PropParams P) {
 #pragma unroll
     for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
     int curk = -1;
-    // a finished row segment [.., end) of start entry k, seen by lane group g
+    // only the run's first row can have begun before the run (in an earlier run or chunk)
+    bool first_began_before = a < b && (S.e[a].y < a || (a == 0 && row0_before));
+    // the row of start entry k ends inside this run
     auto flush = [&](int k) {
-        const bool began_before = k < a || (k == 0 && a == 0 && row0_before);
-        if (began_before) {  // the run's first row, begun in an earlier run or chunk
+        if (first_began_before) {
 #pragma unroll
             for (int j = 0; j < EPC; ++j) S.head[lane * EPC + j] = acc[j];
             if (li == 0) { S.hk[g] = k; S.hclosed[g] = 1; }
+            first_began_before = false;
         } else if (col_lane) {
             float v[EPC];
-            const float d = (float)max(S.sdeg[k], 1);
+            const float f = S.sinv[k];
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) v[j] = P.mean ? acc[j] / d : acc[j];
+            for (int j = 0; j < EPC; ++j) v[j] = acc[j] * f;
             st_stream16(outb + (size_t)S.srow[k] * P.out_ld + (size_t)li * 16, Chunk<T>::pack(v));
         }
     };
@@ -622,15 +627,13 @@ propagate_flat_kernel(const PropParams P) {
         }
     }
     if (curk >= 0) {  // the run's last row
-        const int end = curk == 0 ? end0 : curk + min(S.sdeg[curk], PF_SLAB + 1);
-        if (end <= b) {
+        if (S.send[curk] <= b) {
             flush(curk);
         } else {  // continues past the run
-            const bool began_before = curk < a || (curk == 0 && a == 0 && row0_before);
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) (began_before ? S.head : S.tail)[lane * EPC + j] = acc[j];
+            for (int j = 0; j < EPC; ++j) (first_began_before ? S.head : S.tail)[lane * EPC + j] = acc[j];
             if (li == 0) {
-                if (began_before) { S.hk[g] = curk; S.hclosed[g] = 0; }
+                if (first_began_before) { S.hk[g] = curk; S.hclosed[g] = 0; }
                 else S.tk[g] = curk;
             }
         }
@@ -668,9 +671,9 @@ propagate_flat_kernel(const PropParams P) {
                         write_partial(0);
                     } else if (col_lane) {
                         float v[EPC];
-                        const float d = (float)max(S.sdeg[ck], 1);
+                        const float f = S.sinv[ck];
 #pragma unroll
-                        for (int j = 0; j < EPC; ++j) v[j] = P.mean ? carry[j] / d : carry[j];
+                        for (int j = 0; j < EPC; ++j) v[j] = carry[j] * f;
                         st_stream16(outb + (size_t)S.srow[ck] * P.out_ld + (size_t)lane * 16, Chunk<T>::pack(v));
                     }
                     have = false;
