@@ -46,7 +46,7 @@ struct PropParams {
     uint32_t x_ld, out_ld;  // bytes between consecutive rows of X and of out (>= nvec*16)
     int F;
     int mean;  // divide the finished row by max(1, row length)
-    int chunk;  // edges per warp, a multiple of PF_SLAB
+    int chunk;  // edges per warp: 64, 128, 256 or 1024
     int64_t nchunks;
     int32_t* tail_row;  // [nchunks] row whose tail partial lives in slot 1, or -1
     float* part_val;    // [nchunks][2][F]
@@ -467,15 +467,16 @@ struct FlatSmem {
 template <typename T, int LPR>
 __global__ void __launch_bounds__(FL_WARPS * 32, 6)
 propagate_flat_kernel(const PropParams P) {
-    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, L = PF_SLAB / NG, U = FL_U;
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = FL_U;
+    const int L = P.chunk / NG;  // positions per lane group; P.chunk is 64, 128 or 256 here
     __shared__ FlatSmem<EPC> s_all[FL_WARPS];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int64_t c = (int64_t)blockIdx.x * FL_WARPS + wib;
     if (c >= P.nchunks) return;
     FlatSmem<EPC>& S = s_all[wib];
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
-    const int64_t cs = c * PF_SLAB;
-    const int n = (int)((cs + PF_SLAB < P.E ? cs + PF_SLAB : P.E) - cs);  // 1..256 positions
+    const int64_t cs = c * P.chunk;
+    const int n = (int)((cs + P.chunk < P.E ? cs + P.chunk : P.E) - cs);  // 1..256 positions
     const int g = lane / LPR, li = lane % LPR;
     const bool col_lane = li < P.nvec;  // lanes past a narrow row gather chunk 0 and never store
     char* const outb = reinterpret_cast<char*>(P.out);
@@ -848,7 +849,7 @@ static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
 
 template <typename T>
 static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
-    if (mode == MODE_SUM && vpl == 1 && P.chunk == PF_SLAB && P.E > 0) {
+    if (mode == MODE_SUM && vpl == 1 && P.chunk <= PF_SLAB && P.E > 0) {
         launch_flat<T>(P, lpr, st);
         return;
     }
@@ -871,9 +872,14 @@ static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st
 #undef GNN_SD_CASE
 }
 
-// edges per warp: one slab on small graphs (more warps), four slabs once there are enough
-// edges to fill the machine many times over (fewer partial rows to write and re-read)
-static int chunk_edges(int64_t E) { return E >= (int64_t)8 * 1024 * 1024 ? 4 * PF_SLAB : PF_SLAB; }
+// edges per warp: four slabs once there are enough edges to fill the machine many times over (fewer
+// partial rows to write and re-read), one slab below that, and a half or a quarter slab on graphs so
+// small that whole slabs would leave most SMs without a warp
+static int chunk_edges(int64_t E) {
+    if (E >= (int64_t)8 * 1024 * 1024) return 4 * PF_SLAB;
+    if (E >= 512 * 1024) return PF_SLAB;
+    return E >= 128 * 1024 ? PF_SLAB / 2 : PF_SLAB / 4;
+}
 static int64_t num_chunks(int64_t E) { return E > 0 ? ceil_div(E, chunk_edges(E)) : 1; }
 static int64_t num_slabs(int64_t E) { return E > 0 ? ceil_div(E, PF_SLAB) : 1; }
 
