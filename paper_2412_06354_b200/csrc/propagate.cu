@@ -453,7 +453,7 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
 constexpr int FL_WARPS = 4;
 constexpr int FL_U = 8;
 
-template <int EPC>
+template <int EPC, bool ARG>
 struct FlatSmem {
     int4 e[PF_SLAB];         // x: gathered row, y: start entry of the position's row, z: multiplier
     int32_t srow[PF_SLAB];   // [k] row starting at position k of the chunk ([0]: the row holding position 0)
@@ -461,25 +461,47 @@ struct FlatSmem {
     float sinv[PF_SLAB];     // [k] factor of the finished row: 1, or 1 / length for the mean
     float head[32 * EPC];    // per lane: partial of the run's first row when that row began before the run
     float tail[32 * EPC];    // per lane: partial of the run's last row when it continues past the run
+    int32_t head_a[ARG ? 32 * EPC : 1];  // max/min: winner positions of those partials
+    int32_t tail_a[ARG ? 32 * EPC : 1];
     int32_t hk[8], hclosed[8], tk[8];  // per run: start entries of those rows (-1: none), head row ends in the run
 };
 
-template <typename T, int LPR>
-__global__ void __launch_bounds__(FL_WARPS * 32, 6)
+// MODE_SUM (sum / mean) or MODE_MAX / MODE_MIN (winner = smallest position among equal values)
+template <typename T, int LPR, int MODE>
+__global__ void __launch_bounds__(FL_WARPS * 32, MODE == MODE_SUM ? 6 : 4)
 propagate_flat_kernel(const PropParams P) {
     constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = FL_U;
+    constexpr bool ARG = MODE != MODE_SUM;
     const int L = P.chunk / NG;  // positions per lane group; P.chunk is 64, 128 or 256 here
-    __shared__ FlatSmem<EPC> s_all[FL_WARPS];
+    __shared__ FlatSmem<EPC, ARG> s_all[FL_WARPS];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int64_t c = (int64_t)blockIdx.x * FL_WARPS + wib;
     if (c >= P.nchunks) return;
-    FlatSmem<EPC>& S = s_all[wib];
+    FlatSmem<EPC, ARG>& S = s_all[wib];
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
     const int64_t cs = c * P.chunk;
     const int n = (int)((cs + P.chunk < P.E ? cs + P.chunk : P.E) - cs);  // 1..256 positions
     const int g = lane / LPR, li = lane % LPR;
     const bool col_lane = li < P.nvec;  // lanes past a narrow row gather chunk 0 and never store
     char* const outb = reinterpret_cast<char*>(P.out);
+
+    // a finished row: values (already scaled) and, for max/min, winner positions of 16-byte column ci
+    auto store_row = [&](int row, int ci, const float* v, const int32_t* wa) {
+        st_stream16(outb + (size_t)row * P.out_ld + (size_t)ci * 16, Chunk<T>::pack(v));
+        if (ARG && P.argmax) {
+            int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
+#pragma unroll
+            for (int j = 0; j < EPC; j += 4) *reinterpret_cast<int4*>(ap + j) = make_int4(wa[j], wa[j + 1], wa[j + 2], wa[j + 3]);
+        }
+    };
+    // a row without edges: zeros (and no winner)
+    auto store_empty_row = [&](int row) {
+        float z[EPC];
+        int32_t none[EPC];
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) { z[j] = 0.f; none[j] = -1; }
+        for (int ci = lane; ci < P.nvec; ci += 32) store_row(row, ci, z, none);
+    };
 
     // ---- 1a. the row holding position cs: largest r with rowptr[r] <= cs (32-way search)
     int lo = 0, hi = P.N;  // rowptr[lo] <= cs < rowptr[hi]
@@ -512,10 +534,9 @@ propagate_flat_kernel(const PropParams P) {
     if (lane < 8) { S.hk[lane] = -1; S.hclosed[lane] = 0; S.tk[lane] = -1; }
     __syncwarp();
 
-    // ---- 1c. rows after cur0 that start in (cs, cs+n]: mark non-empty ones, zero-fill empty ones
+    // ---- 1c. rows after cur0 that start in (cs, cs+n]: mark non-empty ones, fill empty ones
     if (c == 0)  // leading empty rows
-        for (int r = 0; r < cur0; ++r)
-            for (int ci = lane; ci < P.nvec; ci += 32) st_stream16(outb + (size_t)r * P.out_ld + (size_t)ci * 16, make_uint4(0, 0, 0, 0));
+        for (int r = 0; r < cur0; ++r) store_empty_row(r);
     for (int rb = cur0 + 1;; rb += 32) {
         const int r = rb + lane;
         int64_t rs = 0, re = 0;
@@ -537,8 +558,7 @@ propagate_flat_kernel(const PropParams P) {
         while (em) {
             const int bit = __ffs(em) - 1;
             em &= em - 1;
-            for (int ci = lane; ci < P.nvec; ci += 32)
-                st_stream16(outb + (size_t)(rb + bit) * P.out_ld + (size_t)ci * 16, make_uint4(0, 0, 0, 0));
+            store_empty_row(rb + bit);
         }
         // rowptr is non-decreasing: once a lane is past the chunk (or past the last row) so are all later rows
         if (!__all_sync(0xffffffffu, live)) break;
@@ -576,24 +596,37 @@ propagate_flat_kernel(const PropParams P) {
     const int a = g * L, b = min(a + L, n);
     const char* Xl = reinterpret_cast<const char*>(P.X) + (size_t)(col_lane ? li : 0) * 16;
     float acc[EPC];
+    int32_t arg[ARG ? EPC : 1];
+    auto clear = [&]() {
 #pragma unroll
-    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+        for (int j = 0; j < EPC; ++j) {
+            acc[j] = 0.f;
+            if (ARG) arg[j] = -1;
+        }
+    };
+    clear();
     int curk = -1;
     // only the run's first row can have begun before the run (in an earlier run or chunk)
     bool first_began_before = a < b && (S.e[a].y < a || (a == 0 && row0_before));
+    auto park = [&](float* dv, int32_t* da) {  // accumulator -> this lane's slot of a head / tail array
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) {
+            dv[lane * EPC + j] = acc[j];
+            if (ARG) da[lane * EPC + j] = arg[j];
+        }
+    };
     // the row of start entry k ends inside this run
     auto flush = [&](int k) {
         if (first_began_before) {
-#pragma unroll
-            for (int j = 0; j < EPC; ++j) S.head[lane * EPC + j] = acc[j];
+            park(S.head, S.head_a);
             if (li == 0) { S.hk[g] = k; S.hclosed[g] = 1; }
             first_began_before = false;
         } else if (col_lane) {
             float v[EPC];
             const float f = S.sinv[k];
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) v[j] = acc[j] * f;
-            st_stream16(outb + (size_t)S.srow[k] * P.out_ld + (size_t)li * 16, Chunk<T>::pack(v));
+            for (int j = 0; j < EPC; ++j) v[j] = ARG ? acc[j] : acc[j] * f;
+            store_row(S.srow[k], li, v, arg);
         }
     };
     for (int i = a; i < b; i += U) {
@@ -617,22 +650,32 @@ propagate_flat_kernel(const PropParams P) {
             if (e.y != curk) {
                 if (curk >= 0) flush(curk);
                 curk = e.y;
-#pragma unroll
-                for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+                clear();
             }
             float x[EPC];
             Chunk<T>::unpack(buf[u], x);
             const float w = __int_as_float(e.z);
+            if (ARG) {
+                const int32_t pos = (int32_t)(cs + i + u);
 #pragma unroll
-            for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], w, w);
+                for (int j = 0; j < EPC; ++j) {
+                    const float m = P.w ? w * x[j] : x[j];
+                    // positions ascend along a run: a strict comparison keeps the first of equal values
+                    const bool take = arg[ARG ? j : 0] < 0 || (MODE == MODE_MAX ? m > acc[j] : m < acc[j]);
+                    if (take) { acc[j] = m; arg[ARG ? j : 0] = pos; }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], w, w);
+            }
         }
     }
     if (curk >= 0) {  // the run's last row
         if (S.send[curk] <= b) {
             flush(curk);
         } else {  // continues past the run
-#pragma unroll
-            for (int j = 0; j < EPC; ++j) (first_began_before ? S.head : S.tail)[lane * EPC + j] = acc[j];
+            if (first_began_before) park(S.head, S.head_a);
+            else park(S.tail, S.tail_a);
             if (li == 0) {
                 if (first_began_before) { S.hk[g] = curk; S.hclosed[g] = 0; }
                 else S.tk[g] = curk;
@@ -645,24 +688,42 @@ propagate_flat_kernel(const PropParams P) {
     int32_t tail_row = -1;
     if (lane < LPR) {
         float carry[EPC];
+        int32_t carg[ARG ? EPC : 1];
         bool have = false, before_chunk = false;
         int ck = -1;
         auto write_partial = [&](int which) {
             if (!col_lane) return;
-            float* pv = P.part_val + ((size_t)c * 2 + which) * P.F + (size_t)lane * EPC;
+            const size_t off = ((size_t)c * 2 + which) * P.F + (size_t)lane * EPC;
 #pragma unroll
-            for (int j = 0; j < EPC; j += 4) *reinterpret_cast<float4*>(pv + j) = make_float4(carry[j], carry[j + 1], carry[j + 2], carry[j + 3]);
+            for (int j = 0; j < EPC; j += 4) {
+                *reinterpret_cast<float4*>(P.part_val + off + j) = make_float4(carry[j], carry[j + 1], carry[j + 2], carry[j + 3]);
+                if (ARG)
+                    *reinterpret_cast<int4*>(P.part_arg + off + j) =
+                        make_int4(carg[ARG ? j : 0], carg[ARG ? j + 1 : 0], carg[ARG ? j + 2 : 0], carg[ARG ? j + 3 : 0]);
+            }
         };
         for (int gg = 0; gg < NG; ++gg) {
             const int hk = S.hk[gg];
             if (hk >= 0) {
-                const float* h = S.head + (gg * LPR + lane) * EPC;
-                if (have) {
+                const int slot = (gg * LPR + lane) * EPC;
+                if (have) {  // later positions: the carry wins ties
 #pragma unroll
-                    for (int j = 0; j < EPC; ++j) carry[j] += h[j];
+                    for (int j = 0; j < EPC; ++j) {
+                        if (ARG) {
+                            if (beats<MODE>(S.head[slot + j], S.head_a[ARG ? slot + j : 0], carry[j], carg[ARG ? j : 0])) {
+                                carry[j] = S.head[slot + j];
+                                carg[ARG ? j : 0] = S.head_a[ARG ? slot + j : 0];
+                            }
+                        } else {
+                            carry[j] += S.head[slot + j];
+                        }
+                    }
                 } else {  // only the chunk's first run can begin without a carry
 #pragma unroll
-                    for (int j = 0; j < EPC; ++j) carry[j] = h[j];
+                    for (int j = 0; j < EPC; ++j) {
+                        carry[j] = S.head[slot + j];
+                        if (ARG) carg[ARG ? j : 0] = S.head_a[ARG ? slot + j : 0];
+                    }
                     before_chunk = true;
                     have = true;
                 }
@@ -674,17 +735,20 @@ propagate_flat_kernel(const PropParams P) {
                         float v[EPC];
                         const float f = S.sinv[ck];
 #pragma unroll
-                        for (int j = 0; j < EPC; ++j) v[j] = carry[j] * f;
-                        st_stream16(outb + (size_t)S.srow[ck] * P.out_ld + (size_t)lane * 16, Chunk<T>::pack(v));
+                        for (int j = 0; j < EPC; ++j) v[j] = ARG ? carry[j] : carry[j] * f;
+                        store_row(S.srow[ck], lane, v, carg);
                     }
                     have = false;
                 }
             }
             const int tk = S.tk[gg];
             if (tk >= 0) {
-                const float* t = S.tail + (gg * LPR + lane) * EPC;
+                const int slot = (gg * LPR + lane) * EPC;
 #pragma unroll
-                for (int j = 0; j < EPC; ++j) carry[j] = t[j];
+                for (int j = 0; j < EPC; ++j) {
+                    carry[j] = S.tail[slot + j];
+                    if (ARG) carg[ARG ? j : 0] = S.tail_a[ARG ? slot + j : 0];
+                }
                 have = true;
                 before_chunk = false;
                 ck = tk;
@@ -832,25 +896,27 @@ static void launch_chunks(const PropParams& P, int lpr, int vpl, cudaStream_t st
     propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
 }
 
-// sums over rows of at most 512 bytes on graphs small enough for one-slab chunks: the flat kernel
-template <typename T>
+// sum / mean / max / min over rows of at most 512 bytes on graphs small enough for one-slab chunks
+template <typename T, int MODE>
 static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
     const int grid = (int)ceil_div(P.nchunks, FL_WARPS);
     const int thr = FL_WARPS * 32;
     switch (lpr) {
-        case 4: propagate_flat_kernel<T, 4><<<grid, thr, 0, st>>>(P); break;
-        case 8: propagate_flat_kernel<T, 8><<<grid, thr, 0, st>>>(P); break;
-        case 16: propagate_flat_kernel<T, 16><<<grid, thr, 0, st>>>(P); break;
-        default: propagate_flat_kernel<T, 32><<<grid, thr, 0, st>>>(P); break;
+        case 4: propagate_flat_kernel<T, 4, MODE><<<grid, thr, 0, st>>>(P); break;
+        case 8: propagate_flat_kernel<T, 8, MODE><<<grid, thr, 0, st>>>(P); break;
+        case 16: propagate_flat_kernel<T, 16, MODE><<<grid, thr, 0, st>>>(P); break;
+        default: propagate_flat_kernel<T, 32, MODE><<<grid, thr, 0, st>>>(P); break;
     }
     const int64_t threads = P.nchunks * P.nvec;
-    propagate_fixup_kernel<T, MODE_SUM><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
+    propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
 }
 
 template <typename T>
 static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
-    if (mode == MODE_SUM && vpl == 1 && P.chunk <= PF_SLAB && P.E > 0) {
-        launch_flat<T>(P, lpr, st);
+    if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0 && (mode == MODE_SUM || mode == MODE_MAX || mode == MODE_MIN)) {
+        if (mode == MODE_SUM) launch_flat<T, MODE_SUM>(P, lpr, st);
+        else if (mode == MODE_MAX) launch_flat<T, MODE_MAX>(P, lpr, st);
+        else launch_flat<T, MODE_MIN>(P, lpr, st);
         return;
     }
     switch (mode) {
