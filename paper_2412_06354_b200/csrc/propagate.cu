@@ -466,12 +466,13 @@ struct FlatSmem {
     int32_t hk[8], hclosed[8], tk[8];  // per run: start entries of those rows (-1: none), head row ends in the run
 };
 
-// MODE_SUM (sum / mean) or MODE_MAX / MODE_MIN (winner = smallest position among equal values)
+// MODE_SUM (sum / mean), MODE_MAX / MODE_MIN (winner = smallest position among equal values), or
+// MODE_ROUTE (backward of max/min: a sum that keeps dOut[c,f] only where position route_pos won (c,f))
 template <typename T, int LPR, int MODE>
 __global__ void __launch_bounds__(FL_WARPS * 32, MODE == MODE_SUM ? 6 : 4)
 propagate_flat_kernel(const PropParams P) {
-    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = FL_U;
-    constexpr bool ARG = MODE != MODE_SUM;
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = MODE == MODE_ROUTE ? FL_U / 2 : FL_U;
+    constexpr bool ARG = MODE == MODE_MAX || MODE == MODE_MIN;
     const int L = P.chunk / NG;  // positions per lane group; P.chunk is 64, 128 or 256 here
     __shared__ FlatSmem<EPC, ARG> s_all[FL_WARPS];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -528,7 +529,8 @@ propagate_flat_kernel(const PropParams P) {
             const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
             w = w / (float)(d > 1 ? d : 1);
         }
-        S.e[i] = make_int4(cc, 0, __float_as_int(w), 0);
+        const int t = (MODE == MODE_ROUTE) ? ld_hint_i32(P.route_pos + cs + i, pol_stream) : 0;
+        S.e[i] = make_int4(cc, 0, __float_as_int(w), t);
     }
     if (lane == 0) { S.srow[0] = cur0; S.send[0] = rel_end(re0); S.sinv[0] = row_factor(re0 - rs0); }
     if (lane < 8) { S.hk[lane] = -1; S.hclosed[lane] = 0; S.tk[lane] = -1; }
@@ -629,19 +631,38 @@ propagate_flat_kernel(const PropParams P) {
             store_row(S.srow[k], li, v, arg);
         }
     };
+    const int32_t* const route_l = (MODE == MODE_ROUTE) ? P.route_arg + (size_t)(col_lane ? li : 0) * EPC : nullptr;
     for (int i = a; i < b; i += U) {
         uint4 buf[U];
+        int4 win[MODE == MODE_ROUTE ? U : 1][MODE == MODE_ROUTE ? EPC / 4 : 1];
         const int nu = min(U, b - i);  // U except at the ragged end of the last chunk
         if (nu == U) {
             int cols[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) cols[u] = S.e[i + u].x;
 #pragma unroll
-            for (int u = 0; u < U; ++u) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
+            for (int u = 0; u < U; ++u) {
+                buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
+                if (MODE == MODE_ROUTE) {
+#pragma unroll
+                    for (int q = 0; q < EPC / 4; ++q)
+                        win[MODE == MODE_ROUTE ? u : 0][MODE == MODE_ROUTE ? q : 0] =
+                            __ldg(reinterpret_cast<const int4*>(route_l + (size_t)cols[u] * P.F) + q);
+                }
+            }
         } else {
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (u < nu) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)S.e[i + u].x * P.x_ld, pol_keep);
+                if (u < nu) {
+                    const int cc = S.e[i + u].x;
+                    buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * P.x_ld, pol_keep);
+                    if (MODE == MODE_ROUTE) {
+#pragma unroll
+                        for (int q = 0; q < EPC / 4; ++q)
+                            win[MODE == MODE_ROUTE ? u : 0][MODE == MODE_ROUTE ? q : 0] =
+                                __ldg(reinterpret_cast<const int4*>(route_l + (size_t)cc * P.F) + q);
+                    }
+                }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -663,6 +684,15 @@ propagate_flat_kernel(const PropParams P) {
                     // positions ascend along a run: a strict comparison keeps the first of equal values
                     const bool take = arg[ARG ? j : 0] < 0 || (MODE == MODE_MAX ? m > acc[j] : m < acc[j]);
                     if (take) { acc[j] = m; arg[ARG ? j : 0] = pos; }
+                }
+            } else if (MODE == MODE_ROUTE) {
+#pragma unroll
+                for (int q = 0; q < EPC / 4; ++q) {
+                    const int4 t = win[MODE == MODE_ROUTE ? u : 0][MODE == MODE_ROUTE ? q : 0];
+                    if (t.x == e.w) acc[4 * q] = fmaf(w, x[4 * q], acc[4 * q]);
+                    if (t.y == e.w) acc[4 * q + 1] = fmaf(w, x[4 * q + 1], acc[4 * q + 1]);
+                    if (t.z == e.w) acc[4 * q + 2] = fmaf(w, x[4 * q + 2], acc[4 * q + 2]);
+                    if (t.w == e.w) acc[4 * q + 3] = fmaf(w, x[4 * q + 3], acc[4 * q + 3]);
                 }
             } else {
 #pragma unroll
@@ -913,10 +943,11 @@ static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
 
 template <typename T>
 static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
-    if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0 && (mode == MODE_SUM || mode == MODE_MAX || mode == MODE_MIN)) {
+    if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0 && mode != MODE_HEADSUM) {
         if (mode == MODE_SUM) launch_flat<T, MODE_SUM>(P, lpr, st);
         else if (mode == MODE_MAX) launch_flat<T, MODE_MAX>(P, lpr, st);
-        else launch_flat<T, MODE_MIN>(P, lpr, st);
+        else if (mode == MODE_MIN) launch_flat<T, MODE_MIN>(P, lpr, st);
+        else launch_flat<T, MODE_ROUTE>(P, lpr, st);
         return;
     }
     switch (mode) {
