@@ -109,12 +109,43 @@ __device__ __forceinline__ void softmax_bwd_row(const T* alpha, const T* dalpha,
 
 static __host__ __device__ inline bool head_pow2(int H) { return H >= 1 && H <= 32 && (H & (H - 1)) == 0; }
 
-// Row loops: every warp (LONG = false) or block (LONG = true) strides over the rows and takes the
-// ones of its kind, so the grids stay a few waves large whatever N is.
-template <bool LONG>
-__device__ __forceinline__ void row_loop_bounds(int* first, int* stride) {
-    if (LONG) { *first = blockIdx.x; *stride = gridDim.x; }
-    else { *first = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5); *stride = (int)((gridDim.x * (int64_t)blockDim.x) >> 5); }
+// Row loops.  LONG = false: every warp strides over the rows and takes the ones of at most
+// SM_LONG_ROW positions.  LONG = true: every block takes a contiguous share of the rows, scans it
+// NT rows at a time (one rowptr pair per thread), lists the rows longer than SM_LONG_ROW in shared
+// memory and works through the list with all its threads.  The list order varies from run to run;
+// each row's arithmetic does not depend on it.
+struct LongRows {
+    int list[512];
+    int count;
+};
+
+template <bool LONG, int NT, class Body>
+__device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr, int N, LongRows& L, Body body) {
+    if (LONG) {
+        const int per = (N + (int)gridDim.x - 1) / (int)gridDim.x;
+        const int r0 = (int)blockIdx.x * per, r1 = min(N, r0 + per);
+        for (int base = r0; base < r1; base += NT) {
+            __syncthreads();  // every thread is done with the previous list
+            if (threadIdx.x == 0) L.count = 0;
+            __syncthreads();
+            const int r = base + (int)threadIdx.x;
+            if (r < r1 && rowptr[r + 1] - rowptr[r] > SM_LONG_ROW) L.list[atomicAdd(&L.count, 1)] = r;
+            __syncthreads();
+            const int n = L.count;
+            for (int i = 0; i < n; ++i) {
+                const int row = L.list[i];
+                body(row, rowptr[row], rowptr[row + 1]);
+            }
+        }
+    } else {
+        int row = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+        const int stride = (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
+        for (; row < N; row += stride) {
+            const int64_t a = rowptr[row], b = rowptr[row + 1];
+            if (b - a > SM_LONG_ROW) continue;  // uniform per warp
+            body(row, a, b);
+        }
+    }
 }
 
 template <typename T, bool LONG>
@@ -122,21 +153,18 @@ __global__ void __launch_bounds__(SM_BLOCK)
 edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ s, int H,
                     T* __restrict__ alpha, float* __restrict__ rowmax, float* __restrict__ rowsum) {
     __shared__ float red[SM_BLOCK];
-    int row, stride;
-    row_loop_bounds<LONG>(&row, &stride);
-    for (; row < N; row += stride) {
-        const int64_t a = rowptr[row], b = rowptr[row + 1];
-        if (((b - a) > SM_LONG_ROW) != LONG) continue;  // uniform per warp (LONG = false) or per block (LONG = true)
+    __shared__ LongRows lrows;
+    for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) {
             if ((threadIdx.x & 31) < H) {
                 if (rowmax) rowmax[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
                 if (rowsum) rowsum[(size_t)row * H + (threadIdx.x & 31)] = 0.f;
             }
-            continue;
+            return;
         }
         if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
         else softmax_row_any<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
-    }
+    });
 }
 
 template <typename T, bool LONG>
@@ -144,13 +172,10 @@ __global__ void __launch_bounds__(SM_BLOCK)
 edge_softmax_backward_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ alpha,
                              const T* __restrict__ dalpha, int H, T* __restrict__ ds) {
     __shared__ float red[SM_BLOCK];
-    int row, stride;
-    row_loop_bounds<LONG>(&row, &stride);
-    for (; row < N; row += stride) {
-        const int64_t a = rowptr[row], b = rowptr[row + 1];
-        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
-        softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
-    }
+    __shared__ LongRows lrows;
+    for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int, int64_t a, int64_t b) {
+        if (b > a) softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
+    });
 }
 
 // GAT attention coefficients in one kernel: logits z = LeakyReLU(al[col[p],h] + ar[i,h]) are written
@@ -164,11 +189,9 @@ gat_alpha_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__
     constexpr int NT = LONG ? SM_BLOCK : 32;
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     const int h = tid % H;
-    int row, stride;
-    row_loop_bounds<LONG>(&row, &stride);
-    for (; row < N; row += stride) {
-        const int64_t a = rowptr[row], b = rowptr[row + 1];
-        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
+    __shared__ LongRows lrows;
+    for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+        if (b == a) return;
         const size_t lo = (size_t)a * H, hi = (size_t)b * H;
         const float arv = ar[(size_t)row * H + h];
         float m = -INFINITY;
@@ -183,7 +206,7 @@ gat_alpha_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__
         for (size_t t = lo + tid; t < hi; t += NT) zs += expf(alpha[t] - m);
         zs = reduce_same_head<SumOp, NT>(zs, H, red);
         for (size_t t = lo + tid; t < hi; t += NT) alpha[t] = expf(alpha[t] - m) / zs;
-    }
+    });
 }
 
 // ---- position-per-lane layout for H = 4*HV heads: a lane owns whole positions (all heads of an
@@ -225,11 +248,9 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
     constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
-    int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    const int stride = LONG ? gridDim.x : (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
-    for (; row < N; row += stride) {
-        const int64_t a = rowptr[row], b = rowptr[row + 1];
-        if (((b - a) > SM_LONG_ROW) != LONG || b == a) continue;
+    __shared__ LongRows lrows;
+    for_each_row<LONG, PL_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+        if (b == a) return;
         float arv[H], m[H], zs[H];
 #pragma unroll
         for (int q = 0; q < HV; ++q) {
@@ -273,7 +294,7 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
                                     expf(t.z - m[4 * q + 2]) / zs[4 * q + 2], expf(t.w - m[4 * q + 3]) / zs[4 * q + 3]);
             }
         }
-    }
+    });
 }
 
 // backward rows: d[h] = sum_p alpha*dalpha; dz = alpha*(dalpha - d)*LeakyReLU'(z), written over dalpha; dar = sum_p dz
@@ -285,14 +306,11 @@ gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __rest
     constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
-    int row = LONG ? blockIdx.x : (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    const int stride = LONG ? gridDim.x : (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
-    for (; row < N; row += stride) {
-        const int64_t a = rowptr[row], b = rowptr[row + 1];
-        if (((b - a) > SM_LONG_ROW) != LONG) continue;
+    __shared__ LongRows lrows;
+    for_each_row<LONG, PL_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) {
             if (tid < H) dar[(size_t)row * H + tid] = 0.f;
-            continue;
+            return;
         }
         float arv[H], d[H], sdz[H];
 #pragma unroll
@@ -336,7 +354,7 @@ gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __rest
 #pragma unroll
             for (int j = 0; j < H; ++j) dar[(size_t)row * H + j] = sdz[j];
         }
-    }
+    });
 }
 
 static int row_grid(int N, bool is_long) {
