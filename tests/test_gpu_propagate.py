@@ -303,3 +303,41 @@ def test_powerlaw_workload_full_size(gnn, dtype):
         assert_close(to_host64(dW), bw["dw"][eid], bw["Sdw"][eid], "f32", "dW")
     finally:
         oracle.set_threads(1)
+
+
+@pytest.mark.parametrize("e,dtype,F", [(200_000, "f32", 32), (200_000, "bf16", 8), (600_000, "bf16", 64), (600_000, "f32", 12),
+                                       (70_000, "bf16", 128), (130_000, "f32", 128)])
+def test_chunk_regimes_with_empty_rows_everywhere(gnn, e, dtype, F):
+    """Edge counts on both sides of the chunk-size thresholds (64 / 128 / 256 positions per warp), rows
+    without edges at the front, in the middle and at the end, a hub cut by many chunks, every lane layout."""
+    n = 5000
+    rng = np.random.default_rng(e + F)
+    # targets only in [300, 4000) and never a multiple of 7: empty rows lead, trail and are interspersed
+    dst = rng.integers(300, 4000, e).astype(np.int32)
+    dst[dst % 7 == 0] += 1
+    dst[: e // 20] = 1234  # hub
+    src = rng.integers(0, n, e).astype(np.int32)
+    g = build_graph(gnn, n, src, dst)
+    ref = host_csr(n, src, dst)
+    eid, eidT = ref["eid"], ref["eidT"]
+    X = feats((n, F), dtype, 300 + F)
+    w = synth.uniform_f32((e,), 0.0, 1.0, 11)
+    Xd = to_dev(X)
+    for op, weighted in (("sum", True), ("mean", False)):
+        out = gnn.propagate_fused(g, Xd, to_dev(w[eid]) if weighted else None, op)
+        o, S, _ = oracle.propagate(op, n, src, dst, X, w if weighted else None)
+        assert_close(to_host64(out), o, S, dtype, f"{op} E={e}")
+        R = feats((n, F), dtype, 301 + F)
+        dX, _ = gnn.propagate_fused_backward(g, to_dev(R), op, w_csrT=to_dev(w[eidT]) if weighted else None)
+        bw = oracle.propagate_backward(op, n, src, dst, X, w if weighted else None, R)
+        assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, f"{op} backward E={e}")
+    for op in ("max", "min"):
+        out, arg = gnn.propagate_fused(g, Xd, None, op)
+        o, _, a = oracle.propagate(op, n, src, dst, X)
+        assert np.array_equal(bits(out), f64_to_dtype_bits(o, dtype))
+        ga = arg.cpu().numpy()
+        assert np.array_equal(np.where(ga >= 0, eid[np.maximum(ga, 0)], -1), a)
+        R = feats((n, F), dtype, 302 + F)
+        dX, _ = gnn.propagate_fused_backward(g, to_dev(R), op, argmax=arg)
+        bw = oracle.propagate_backward(op, n, src, dst, X, None, R, arg=a)
+        assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, f"{op} backward E={e}")
