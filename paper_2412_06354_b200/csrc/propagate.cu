@@ -466,10 +466,11 @@ struct FlatSmem {
     int32_t hk[8], hclosed[8], tk[8];  // per run: start entries of those rows (-1: none), head row ends in the run
 };
 
-// MODE_SUM (sum / mean), MODE_MAX / MODE_MIN (winner = smallest position among equal values), or
-// MODE_ROUTE (backward of max/min: a sum that keeps dOut[c,f] only where position route_pos won (c,f))
+// MODE_SUM (sum / mean), MODE_MAX / MODE_MIN (winner = smallest position among equal values),
+// MODE_ROUTE (backward of max/min: a sum that keeps dOut[c,f] only where position route_pos won (c,f)) or
+// MODE_HEADSUM (one multiplier per position and head, optional rank-1 row epilogue)
 template <typename T, int LPR, int MODE>
-__global__ void __launch_bounds__(FL_WARPS * 32, MODE == MODE_SUM ? 6 : 4)
+__global__ void __launch_bounds__(FL_WARPS * 32, (MODE == MODE_SUM || MODE == MODE_HEADSUM) ? 6 : 4)
 propagate_flat_kernel(const PropParams P) {
     constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = MODE == MODE_ROUTE ? FL_U / 2 : FL_U;
     constexpr bool ARG = MODE == MODE_MAX || MODE == MODE_MIN;
@@ -487,7 +488,14 @@ propagate_flat_kernel(const PropParams P) {
     char* const outb = reinterpret_cast<char*>(P.out);
 
     // a finished row: values (already scaled) and, for max/min, winner positions of 16-byte column ci
-    auto store_row = [&](int row, int ci, const float* v, const int32_t* wa) {
+    auto store_row = [&](int row, int ci, float* v, const int32_t* wa) {
+        if (MODE == MODE_HEADSUM && P.epi_l) {  // rank-1 row epilogue of the per-head mode
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) {
+                const int f = ci * EPC + j, h = f / P.fph;
+                v[j] += P.epi_l[(size_t)row * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)row * P.H + h] * P.epi_b[f];
+            }
+        }
         st_stream16(outb + (size_t)row * P.out_ld + (size_t)ci * 16, Chunk<T>::pack(v));
         if (ARG && P.argmax) {
             int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
@@ -497,11 +505,13 @@ propagate_flat_kernel(const PropParams P) {
     };
     // a row without edges: zeros (and no winner)
     auto store_empty_row = [&](int row) {
-        float z[EPC];
-        int32_t none[EPC];
+        for (int ci = lane; ci < P.nvec; ci += 32) {
+            float z[EPC];
+            int32_t none[EPC];
 #pragma unroll
-        for (int j = 0; j < EPC; ++j) { z[j] = 0.f; none[j] = -1; }
-        for (int ci = lane; ci < P.nvec; ci += 32) store_row(row, ci, z, none);
+            for (int j = 0; j < EPC; ++j) { z[j] = 0.f; none[j] = -1; }
+            store_row(row, ci, z, none);
+        }
     };
 
     // ---- 1a. the row holding position cs: largest r with rowptr[r] <= cs (32-way search)
@@ -632,8 +642,11 @@ propagate_flat_kernel(const PropParams P) {
         }
     };
     const int32_t* const route_l = (MODE == MODE_ROUTE) ? P.route_arg + (size_t)(col_lane ? li : 0) * EPC : nullptr;
+    // per-head mode: this lane's head column of the [E,H] multiplier matrix, at the chunk's first position
+    const float* const wh_l = (MODE == MODE_HEADSUM) ? P.wh + (size_t)cs * P.H + ((col_lane ? li : 0) * EPC) / P.fph : nullptr;
     for (int i = a; i < b; i += U) {
         uint4 buf[U];
+        float hw[MODE == MODE_HEADSUM ? U : 1];
         int4 win[MODE == MODE_ROUTE ? U : 1][MODE == MODE_ROUTE ? EPC / 4 : 1];
         const int nu = min(U, b - i);  // U except at the ragged end of the last chunk
         if (nu == U) {
@@ -643,6 +656,7 @@ propagate_flat_kernel(const PropParams P) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
+                if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(i + u) * P.H);
                 if (MODE == MODE_ROUTE) {
 #pragma unroll
                     for (int q = 0; q < EPC / 4; ++q)
@@ -656,6 +670,7 @@ propagate_flat_kernel(const PropParams P) {
                 if (u < nu) {
                     const int cc = S.e[i + u].x;
                     buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * P.x_ld, pol_keep);
+                    if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(i + u) * P.H);
                     if (MODE == MODE_ROUTE) {
 #pragma unroll
                         for (int q = 0; q < EPC / 4; ++q)
@@ -695,8 +710,9 @@ propagate_flat_kernel(const PropParams P) {
                     if (t.w == e.w) acc[4 * q + 3] = fmaf(w, x[4 * q + 3], acc[4 * q + 3]);
                 }
             } else {
+                const float m = (MODE == MODE_HEADSUM) ? hw[MODE == MODE_HEADSUM ? u : 0] : w;
 #pragma unroll
-                for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], w, w);
+                for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], m, m);
             }
         }
     }
@@ -943,8 +959,9 @@ static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
 
 template <typename T>
 static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStream_t st) {
-    if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0 && mode != MODE_HEADSUM) {
+    if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0) {
         if (mode == MODE_SUM) launch_flat<T, MODE_SUM>(P, lpr, st);
+        else if (mode == MODE_HEADSUM) launch_flat<T, MODE_HEADSUM>(P, lpr, st);
         else if (mode == MODE_MAX) launch_flat<T, MODE_MAX>(P, lpr, st);
         else if (mode == MODE_MIN) launch_flat<T, MODE_MIN>(P, lpr, st);
         else launch_flat<T, MODE_ROUTE>(P, lpr, st);
