@@ -10,7 +10,7 @@
 
 namespace gnn {
 
-// thread per (node, head): the two score dot products
+// thread per (node, head): the two score dot products (any C)
 template <typename T>
 __global__ void gat_scores_kernel(const T* __restrict__ Wx, const float* __restrict__ a_src,
                                   const float* __restrict__ a_dst, int64_t NH, int H, int C,
@@ -27,6 +27,43 @@ __global__ void gat_scores_kernel(const T* __restrict__ Wx, const float* __restr
     }
     al[t] = sl;
     ar[t] = sr;
+}
+
+// Rows of at most 32 16-byte chunks whose heads span a power-of-two number of chunks: LPR lanes
+// cover a node's row with one coalesced 16-byte load each (32/LPR nodes per warp), keep their slice
+// of both attention vectors in registers, and the lanes of a head add up by xor-shuffles (fixed tree).
+template <typename T, int LPR>
+__global__ void __launch_bounds__(256)
+gat_scores_rows_kernel(const T* __restrict__ Wx, const float* __restrict__ a_src, const float* __restrict__ a_dst,
+                       int N, int H, int nvec, int lph, float* __restrict__ al, float* __restrict__ ar) {
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR;
+    const int lane = threadIdx.x & 31, g = lane / LPR, li = lane % LPR;
+    const bool on = li < nvec;
+    float as[EPC], ad[EPC];
+#pragma unroll
+    for (int j = 0; j < EPC; ++j) {
+        as[j] = on ? a_src[li * EPC + j] : 0.f;
+        ad[j] = on ? a_dst[li * EPC + j] : 0.f;
+    }
+    const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * (int64_t)blockDim.x) >> 5;
+    for (int64_t n0 = warp * NG; n0 < N; n0 += nwarps * NG) {
+        const int64_t n = n0 + g;
+        float sl = 0.f, sr = 0.f;
+        if (n < N && on) {
+            float x[EPC];
+            Chunk<T>::unpack(*reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(Wx) + ((size_t)n * nvec + li) * 16), x);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) { sl = fmaf(as[j], x[j], sl); sr = fmaf(ad[j], x[j], sr); }
+        }
+        for (int o = lph >> 1; o > 0; o >>= 1) {
+            sl += __shfl_xor_sync(0xffffffffu, sl, o);
+            sr += __shfl_xor_sync(0xffffffffu, sr, o);
+        }
+        if (n < N && on && (li % lph) == 0) {
+            al[(size_t)n * H + li / lph] = sl;
+            ar[(size_t)n * H + li / lph] = sr;
+        }
+    }
 }
 
 // Row-local part of the backward pass, one warp per row (a whole block for long rows):
@@ -92,7 +129,7 @@ gat_backward_rows_kernel(const int64_t* __restrict__ rowptr, const int32_t* __re
 }
 
 // da_src[f] = sum_n dal[n,h(f)] * Wx[n,f], da_dst likewise with dar: fixed two-stage reduction
-constexpr int GA_BLOCKS = 296;
+constexpr int GA_BLOCKS = 1184;  // 8 per SM: short serial chains over the rows
 template <typename T>
 __global__ void gat_da_partial_kernel(const T* __restrict__ Wx, const float* __restrict__ dal,
                                       const float* __restrict__ dar, int N, int H, int C,
@@ -111,17 +148,27 @@ __global__ void gat_da_partial_kernel(const T* __restrict__ Wx, const float* __r
         partial[((size_t)blockIdx.x * 2 + 1) * F + f] = s1;
     }
 }
-__global__ void gat_da_final_kernel(const float* __restrict__ partial, int nblocks, int F,
-                                    float* __restrict__ da_src, float* __restrict__ da_dst) {
-    const int f = blockIdx.x * blockDim.x + threadIdx.x;
-    if (f >= F) return;
+// 64 features x 4 groups of partials per block; group sums in ascending order, then ((g0+g1)+g2)+g3
+__global__ void __launch_bounds__(256)
+gat_da_final_kernel(const float* __restrict__ partial, int nblocks, int F,
+                    float* __restrict__ da_src, float* __restrict__ da_dst) {
+    __shared__ float sh[2][4][64];
+    const int e = threadIdx.x & 63, gq = threadIdx.x >> 6;
+    const int f = blockIdx.x * 64 + e;
+    const int per = (nblocks + 3) / 4, b0 = gq * per, b1 = min(nblocks, b0 + per);
     float s0 = 0.f, s1 = 0.f;
-    for (int b = 0; b < nblocks; ++b) {
-        s0 += partial[((size_t)b * 2) * F + f];
-        s1 += partial[((size_t)b * 2 + 1) * F + f];
+    if (f < F)
+        for (int b = b0; b < b1; ++b) {
+            s0 += partial[((size_t)b * 2) * F + f];
+            s1 += partial[((size_t)b * 2 + 1) * F + f];
+        }
+    sh[0][gq][e] = s0;
+    sh[1][gq][e] = s1;
+    __syncthreads();
+    if (gq == 0 && f < F) {
+        da_src[f] = ((sh[0][0][e] + sh[0][1][e]) + sh[0][2][e]) + sh[0][3][e];
+        da_dst[f] = ((sh[1][0][e] + sh[1][1][e]) + sh[1][2][e]) + sh[1][3][e];
     }
-    da_src[f] = s0;
-    da_dst[f] = s1;
 }
 
 // dal[j,h] = sum over transposed positions q of row j of dz[t2f[q],h]  (any H; H % 4 == 0 goes
@@ -203,7 +250,15 @@ gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, c
     if (g->N == 0) return GNN_OK;
     cudaStream_t st = as_stream(stream);
     const int64_t NH = (int64_t)g->N * H;
-    if (dtype == GNN_F32)
+    const int s_el = elem_size(dtype), nvec = H * C * s_el / 16, lph = C * s_el / 16;  // chunks per row / per head
+    int lpr = 0, vpl = 0;
+    if (((size_t)C * s_el) % 16 == 0 && (lph & (lph - 1)) == 0 && pick_shape(nvec, &lpr, &vpl) && vpl == 1) {
+        const int grid = grid_for(ceil_div(g->N, 32 / lpr) * 32, 256);
+#define GNN_GS(T, L) gat_scores_rows_kernel<T, L><<<grid, 256, 0, st>>>((const T*)Wx, a_src, a_dst, g->N, H, nvec, lph, al, ar)
+        if (dtype == GNN_F32) { if (lpr == 4) GNN_GS(float, 4); else if (lpr == 8) GNN_GS(float, 8); else if (lpr == 16) GNN_GS(float, 16); else GNN_GS(float, 32); }
+        else { if (lpr == 4) GNN_GS(__nv_bfloat16, 4); else if (lpr == 8) GNN_GS(__nv_bfloat16, 8); else if (lpr == 16) GNN_GS(__nv_bfloat16, 16); else GNN_GS(__nv_bfloat16, 32); }
+#undef GNN_GS
+    } else if (dtype == GNN_F32)
         gat_scores_kernel<float><<<(int)ceil_div(NH, 256), 256, 0, st>>>((const float*)Wx, a_src, a_dst, NH, H, C, al, ar);
     else
         gat_scores_kernel<__nv_bfloat16><<<(int)ceil_div(NH, 256), 256, 0, st>>>((const __nv_bfloat16*)Wx, a_src, a_dst, NH, H, C, al, ar);
@@ -263,7 +318,7 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
         gat_da_partial_kernel<float><<<GA_BLOCKS, 256, 0, st>>>((const float*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
     else
         gat_da_partial_kernel<__nv_bfloat16><<<GA_BLOCKS, 256, 0, st>>>((const __nv_bfloat16*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
-    gat_da_final_kernel<<<(int)ceil_div(F, 256), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
+    gat_da_final_kernel<<<(int)ceil_div(F, 64), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
     GNN_CHECK_LAUNCH(who);
     // dWx[j,h,:] = sum_q alpha[t2f[q],h]*dOut[colT[q],h,:] + dal[j,h]*a_src[h,:] + dar[j,h]*a_dst[h,:]
     if (g->E > 0) {

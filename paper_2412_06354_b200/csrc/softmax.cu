@@ -119,7 +119,7 @@ struct LongRows {
     int count;
 };
 
-template <bool LONG, int NT, class Body>
+template <bool LONG, int NT, int THRESH = SM_LONG_ROW, class Body>
 __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr, int N, LongRows& L, Body body) {
     if (LONG) {
         const int per = (N + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -129,7 +129,7 @@ __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr,
             if (threadIdx.x == 0) L.count = 0;
             __syncthreads();
             const int r = base + (int)threadIdx.x;
-            if (r < r1 && rowptr[r + 1] - rowptr[r] > SM_LONG_ROW) L.list[atomicAdd(&L.count, 1)] = r;
+            if (r < r1 && rowptr[r + 1] - rowptr[r] > THRESH) L.list[atomicAdd(&L.count, 1)] = r;
             __syncthreads();
             const int n = L.count;
             for (int i = 0; i < n; ++i) {
@@ -142,7 +142,7 @@ __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr,
         const int stride = (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
         for (; row < N; row += stride) {
             const int64_t a = rowptr[row], b = rowptr[row + 1];
-            if (b - a > SM_LONG_ROW) continue;  // uniform per warp
+            if (b - a > THRESH) continue;  // uniform per warp
             body(row, a, b);
         }
     }
@@ -239,17 +239,24 @@ __device__ __forceinline__ void reduce_heads(float (&v)[4 * HV], float* red) {
     }
 }
 
-constexpr int PL_BLOCK = 512;  // threads per long row
+constexpr int PL_BLOCK = 512;     // threads per long row
+constexpr int PL_LONG_ROW = 512;  // rows above this many positions get a block instead of a warp
+// positions per thread and batch (their loads are all in flight together): 32 head values per thread
+constexpr int pl_unroll(int HV) { return HV <= 2 ? 4 : (HV == 4 ? 2 : 1); }
 
+// Attention coefficients of one row.  The threads take the row in batches of NT*PL_UNR positions;
+// the gathers of a batch (col, then al[col]) are independent.  A row that fits in one batch (the
+// common case) keeps its logits in registers through the max, sum and normalise steps; longer rows
+// park the logits in alpha and re-read them.
 template <int HV, bool LONG>
 __global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
 gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                     const float* __restrict__ al, const float* __restrict__ ar, float slope, float* __restrict__ alpha) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = pl_unroll(HV);
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     __shared__ LongRows lrows;
-    for_each_row<LONG, PL_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+    for_each_row<LONG, PL_BLOCK, PL_LONG_ROW>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) return;
         float arv[H], m[H], zs[H];
 #pragma unroll
@@ -259,22 +266,67 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
         }
 #pragma unroll
         for (int j = 0; j < H; ++j) { m[j] = -INFINITY; zs[j] = 0.f; }
-        for (int64_t p = a + tid; p < b; p += NT) {
-            const float4* alp = reinterpret_cast<const float4*>(al + (size_t)col[p] * H);
-            float4* out = reinterpret_cast<float4*>(alpha + (size_t)p * H);
+        const bool one_batch = (b - a) <= (int64_t)NT * U;
+        float z[U][H];
+        for (int64_t p0 = a + tid; p0 < b + tid; p0 += (int64_t)NT * U) {  // uniform trip count: p0 - tid < b
+            int c[U];
 #pragma unroll
-            for (int q = 0; q < HV; ++q) {
-                const float4 t = alp[q];
-                float z[4] = {t.x + arv[4 * q], t.y + arv[4 * q + 1], t.z + arv[4 * q + 2], t.w + arv[4 * q + 3]};
+            for (int u = 0; u < U; ++u) {
+                const int64_t p = p0 + (int64_t)u * NT;
+                c[u] = p < b ? col[p] : -1;
+            }
+            float4 t[U][HV];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    z[j] = z[j] > 0.f ? z[j] : slope * z[j];
-                    m[4 * q + j] = fmaxf(m[4 * q + j], z[j]);
+            for (int u = 0; u < U; ++u)
+                if (c[u] >= 0) {
+#pragma unroll
+                    for (int q = 0; q < HV; ++q) t[u][q] = reinterpret_cast<const float4*>(al + (size_t)c[u] * H)[q];
                 }
-                out[q] = make_float4(z[0], z[1], z[2], z[3]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (c[u] < 0) continue;
+#pragma unroll
+                for (int q = 0; q < HV; ++q) {
+                    const float v[4] = {t[u][q].x + arv[4 * q], t[u][q].y + arv[4 * q + 1], t[u][q].z + arv[4 * q + 2], t[u][q].w + arv[4 * q + 3]};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float zz = v[j] > 0.f ? v[j] : slope * v[j];
+                        z[u][4 * q + j] = zz;
+                        m[4 * q + j] = fmaxf(m[4 * q + j], zz);
+                    }
+                }
+                if (!one_batch) {
+                    float4* out = reinterpret_cast<float4*>(alpha + (size_t)(p0 + (int64_t)u * NT) * H);
+#pragma unroll
+                    for (int q = 0; q < HV; ++q) out[q] = make_float4(z[u][4 * q], z[u][4 * q + 1], z[u][4 * q + 2], z[u][4 * q + 3]);
+                }
             }
         }
         reduce_heads<HV, NT, true>(m, red);
+        if (one_batch) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (a + tid + (int64_t)u * NT >= b) continue;
+#pragma unroll
+                for (int j = 0; j < H; ++j) {
+                    z[u][j] = expf(z[u][j] - m[j]);
+                    zs[j] += z[u][j];
+                }
+            }
+            reduce_heads<HV, NT, false>(zs, red);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t p = a + tid + (int64_t)u * NT;
+                if (p >= b) continue;
+                float4* out = reinterpret_cast<float4*>(alpha + (size_t)p * H);
+#pragma unroll
+                for (int q = 0; q < HV; ++q)
+                    out[q] = make_float4(z[u][4 * q] / zs[4 * q], z[u][4 * q + 1] / zs[4 * q + 1], z[u][4 * q + 2] / zs[4 * q + 2],
+                                         z[u][4 * q + 3] / zs[4 * q + 3]);
+            }
+            return;
+        }
+#pragma unroll 4
         for (int64_t p = a + tid; p < b; p += NT) {
             const float4* in = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
 #pragma unroll
@@ -285,6 +337,7 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
             }
         }
         reduce_heads<HV, NT, false>(zs, red);
+#pragma unroll 4
         for (int64_t p = a + tid; p < b; p += NT) {
             float4* io = reinterpret_cast<float4*>(alpha + (size_t)p * H);
 #pragma unroll
@@ -303,11 +356,11 @@ __global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
 gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                        const float* __restrict__ alpha, float* __restrict__ dalpha_dz, const float* __restrict__ al,
                        const float* __restrict__ ar, float slope, float* __restrict__ dar) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32;
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = pl_unroll(HV);
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     __shared__ LongRows lrows;
-    for_each_row<LONG, PL_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+    for_each_row<LONG, PL_BLOCK, PL_LONG_ROW>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) {
             if (tid < H) dar[(size_t)row * H + tid] = 0.f;
             return;
@@ -320,6 +373,7 @@ gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __rest
         }
 #pragma unroll
         for (int j = 0; j < H; ++j) { d[j] = 0.f; sdz[j] = 0.f; }
+#pragma unroll 4
         for (int64_t p = a + tid; p < b; p += NT) {
             const float4* ap = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
             const float4* dp = reinterpret_cast<const float4*>(dalpha_dz + (size_t)p * H);
@@ -331,22 +385,40 @@ gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __rest
             }
         }
         reduce_heads<HV, NT, false>(d, red);
-        for (int64_t p = a + tid; p < b; p += NT) {
-            const float4* ap = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
-            float4* dp = reinterpret_cast<float4*>(dalpha_dz + (size_t)p * H);
-            const float4* alp = reinterpret_cast<const float4*>(al + (size_t)col[p] * H);
+        // second pass in batches of U positions per thread: the col -> al gathers of a batch overlap
+        for (int64_t p0 = a + tid; p0 < b + tid; p0 += (int64_t)NT * U) {
+            int c[U];
 #pragma unroll
-            for (int q = 0; q < HV; ++q) {
-                const float4 x = ap[q], y = dp[q], t = alp[q];
-                const float z[4] = {t.x + arv[4 * q], t.y + arv[4 * q + 1], t.z + arv[4 * q + 2], t.w + arv[4 * q + 3]};
-                const float xa[4] = {x.x, x.y, x.z, x.w}, ya[4] = {y.x, y.y, y.z, y.w};
-                float o[4];
+            for (int u = 0; u < U; ++u) {
+                const int64_t p = p0 + (int64_t)u * NT;
+                c[u] = p < b ? col[p] : -1;
+            }
+            float4 t[U][HV];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    o[j] = xa[j] * (ya[j] - d[4 * q + j]) * (z[j] > 0.f ? 1.f : slope);
-                    sdz[4 * q + j] += o[j];
+            for (int u = 0; u < U; ++u)
+                if (c[u] >= 0) {
+#pragma unroll
+                    for (int q = 0; q < HV; ++q) t[u][q] = reinterpret_cast<const float4*>(al + (size_t)c[u] * H)[q];
                 }
-                dp[q] = make_float4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (c[u] < 0) continue;
+                const int64_t p = p0 + (int64_t)u * NT;
+                const float4* ap = reinterpret_cast<const float4*>(alpha + (size_t)p * H);
+                float4* dp = reinterpret_cast<float4*>(dalpha_dz + (size_t)p * H);
+#pragma unroll
+                for (int q = 0; q < HV; ++q) {
+                    const float4 x = ap[q], y = dp[q];
+                    const float z[4] = {t[u][q].x + arv[4 * q], t[u][q].y + arv[4 * q + 1], t[u][q].z + arv[4 * q + 2], t[u][q].w + arv[4 * q + 3]};
+                    const float xa[4] = {x.x, x.y, x.z, x.w}, ya[4] = {y.x, y.y, y.z, y.w};
+                    float o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        o[j] = xa[j] * (ya[j] - d[4 * q + j]) * (z[j] > 0.f ? 1.f : slope);
+                        sdz[4 * q + j] += o[j];
+                    }
+                    dp[q] = make_float4(o[0], o[1], o[2], o[3]);
+                }
             }
         }
         reduce_heads<HV, NT, false>(sdz, red);
