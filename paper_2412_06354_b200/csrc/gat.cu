@@ -148,26 +148,32 @@ __global__ void gat_da_partial_kernel(const T* __restrict__ Wx, const float* __r
         partial[((size_t)blockIdx.x * 2 + 1) * F + f] = s1;
     }
 }
-// 64 features x 4 groups of partials per block; group sums in ascending order, then ((g0+g1)+g2)+g3
+// 16 features x 16 groups of partials per block; each group is summed in ascending order with
+// independent loads in flight, then the group sums are added in ascending group order
 __global__ void __launch_bounds__(256)
 gat_da_final_kernel(const float* __restrict__ partial, int nblocks, int F,
                     float* __restrict__ da_src, float* __restrict__ da_dst) {
-    __shared__ float sh[2][4][64];
-    const int e = threadIdx.x & 63, gq = threadIdx.x >> 6;
-    const int f = blockIdx.x * 64 + e;
-    const int per = (nblocks + 3) / 4, b0 = gq * per, b1 = min(nblocks, b0 + per);
+    __shared__ float sh[2][16][16];
+    const int e = threadIdx.x & 15, gq = threadIdx.x >> 4;
+    const int f = blockIdx.x * 16 + e;
+    const int per = (nblocks + 15) / 16, b0 = gq * per, b1 = min(nblocks, b0 + per);
     float s0 = 0.f, s1 = 0.f;
-    if (f < F)
+    if (f < F) {
+#pragma unroll 8
         for (int b = b0; b < b1; ++b) {
             s0 += partial[((size_t)b * 2) * F + f];
             s1 += partial[((size_t)b * 2 + 1) * F + f];
         }
+    }
     sh[0][gq][e] = s0;
     sh[1][gq][e] = s1;
     __syncthreads();
     if (gq == 0 && f < F) {
-        da_src[f] = ((sh[0][0][e] + sh[0][1][e]) + sh[0][2][e]) + sh[0][3][e];
-        da_dst[f] = ((sh[1][0][e] + sh[1][1][e]) + sh[1][2][e]) + sh[1][3][e];
+        float t0 = sh[0][0][e], t1 = sh[1][0][e];
+#pragma unroll
+        for (int q = 1; q < 16; ++q) { t0 += sh[0][q][e]; t1 += sh[1][q][e]; }
+        da_src[f] = t0;
+        da_dst[f] = t1;
     }
 }
 
@@ -318,7 +324,7 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
         gat_da_partial_kernel<float><<<GA_BLOCKS, 256, 0, st>>>((const float*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
     else
         gat_da_partial_kernel<__nv_bfloat16><<<GA_BLOCKS, 256, 0, st>>>((const __nv_bfloat16*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
-    gat_da_final_kernel<<<(int)ceil_div(F, 64), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
+    gat_da_final_kernel<<<(int)ceil_div(F, 16), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
     GNN_CHECK_LAUNCH(who);
     // dWx[j,h,:] = sum_q alpha[t2f[q],h]*dOut[colT[q],h,:] + dal[j,h]*a_src[h,:] + dar[j,h]*a_dst[h,:]
     if (g->E > 0) {

@@ -242,17 +242,17 @@ __device__ __forceinline__ void reduce_heads(float (&v)[4 * HV], float* red) {
 constexpr int PL_BLOCK = 512;     // threads per long row
 constexpr int PL_LONG_ROW = 512;  // rows above this many positions get a block instead of a warp
 // positions per thread and batch (their loads are all in flight together): 32 head values per thread
-constexpr int pl_unroll(int HV) { return HV <= 2 ? 4 : (HV == 4 ? 2 : 1); }
+__host__ __device__ constexpr int pl_unroll(int HV) { return HV <= 2 ? 4 : (HV == 4 ? 2 : 1); }
 
 // Attention coefficients of one row.  The threads take the row in batches of NT*PL_UNR positions;
 // the gathers of a batch (col, then al[col]) are independent.  A row that fits in one batch (the
 // common case) keeps its logits in registers through the max, sum and normalise steps; longer rows
 // park the logits in alpha and re-read them.
 template <int HV, bool LONG>
-__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
+__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK, LONG ? 1 : (HV <= 2 ? 3 : 2))
 gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                     const float* __restrict__ al, const float* __restrict__ ar, float slope, float* __restrict__ alpha) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = pl_unroll(HV);
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     __shared__ LongRows lrows;
@@ -352,11 +352,11 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
 
 // backward rows: d[h] = sum_p alpha*dalpha; dz = alpha*(dalpha - d)*LeakyReLU'(z), written over dalpha; dar = sum_p dz
 template <int HV, bool LONG>
-__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK)
+__global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK, LONG ? 1 : (HV <= 2 ? 3 : 2))
 gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                        const float* __restrict__ alpha, float* __restrict__ dalpha_dz, const float* __restrict__ al,
                        const float* __restrict__ ar, float slope, float* __restrict__ dar) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = pl_unroll(HV);
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
     const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
     __shared__ LongRows lrows;
