@@ -244,11 +244,10 @@ struct Walker {
     // optional rank-1 update of a finished row chunk (see PropParams::epi_*)
     __device__ __forceinline__ static void epilogue(const PropParams& P, int64_t row, int ci, float* v) {
         if (!P.epi_l) return;
+        const int h = (ci * EPC) / P.fph;  // a 16-byte chunk lies inside one head
+        const float el = P.epi_l[(size_t)row * P.H + h], er = P.epi_r[(size_t)row * P.H + h];
 #pragma unroll
-        for (int j = 0; j < EPC; ++j) {
-            const int f = ci * EPC + j, h = f / P.fph;
-            v[j] += P.epi_l[(size_t)row * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)row * P.H + h] * P.epi_b[f];
-        }
+        for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
     }
 
     // combine the lane groups; afterwards every lane holds the result for its chunk index
@@ -421,11 +420,10 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
         for (int j = 0; j < EPC; ++j) v[j] = v[j] / d;
     }
     if (MODE == MODE_HEADSUM && P.epi_l) {
+        const int h = (ci * EPC) / P.fph;  // a 16-byte chunk lies inside one head
+        const float el = P.epi_l[(size_t)r * P.H + h], er = P.epi_r[(size_t)r * P.H + h];
 #pragma unroll
-        for (int j = 0; j < EPC; ++j) {
-            const int f = ci * EPC + j, h = f / P.fph;
-            v[j] += P.epi_l[(size_t)r * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)r * P.H + h] * P.epi_b[f];
-        }
+        for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
     }
     char* ob = reinterpret_cast<char*>(P.out) + (size_t)r * P.out_ld + (size_t)ci * 16;
     *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
@@ -490,11 +488,10 @@ propagate_flat_kernel(const PropParams P) {
     // a finished row: values (already scaled) and, for max/min, winner positions of 16-byte column ci
     auto store_row = [&](int row, int ci, float* v, const int32_t* wa) {
         if (MODE == MODE_HEADSUM && P.epi_l) {  // rank-1 row epilogue of the per-head mode
+            const int h = (ci * EPC) / P.fph;  // a 16-byte chunk lies inside one head
+            const float el = P.epi_l[(size_t)row * P.H + h], er = P.epi_r[(size_t)row * P.H + h];
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) {
-                const int f = ci * EPC + j, h = f / P.fph;
-                v[j] += P.epi_l[(size_t)row * P.H + h] * P.epi_a[f] + P.epi_r[(size_t)row * P.H + h] * P.epi_b[f];
-            }
+            for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
         }
         st_stream16(outb + (size_t)row * P.out_ld + (size_t)ci * 16, Chunk<T>::pack(v));
         if (ARG && P.argmax) {
@@ -918,6 +915,132 @@ sddmm_chunk_kernel(const SddmmParams P) {
     }
 }
 
+// ------------------------------------------------------------------ flat SDDMM for short rows
+// Same idea as propagate_flat_kernel: positions first, rows second.  The warp stages the gathered
+// rows of its 256 positions and finds, by marking row starts and a prefix maximum, the row of every
+// position; each lane group then takes a contiguous run and issues, per batch of 4 positions, the
+// independent loads of X[col[p]] and dOut[row(p)] (the latter mostly from L1: neighbouring positions
+// share it).  Every position is independent, so there are no partials and no second pass.
+constexpr int SF_U = 4;
+
+struct SddmmFlatSmem {
+    int2 e[PF_SLAB];        // x: gathered row of X, y: start entry of the position's row
+    int32_t srow[PF_SLAB];  // [k] row starting at position k of the chunk ([0]: the row holding position 0)
+    float sinv[PF_SLAB];    // [k] 1, or 1 / row length for the mean
+};
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(FL_WARPS * 32, 8)
+sddmm_flat_kernel(const SddmmParams P) {
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = SF_U, L = PF_SLAB / NG;
+    __shared__ SddmmFlatSmem s_all[FL_WARPS];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int64_t c = (int64_t)blockIdx.x * FL_WARPS + wib;
+    if (c >= P.nchunks) return;
+    SddmmFlatSmem& S = s_all[wib];
+    const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
+    const int64_t cs = c * PF_SLAB;
+    const int n = (int)((cs + PF_SLAB < P.E ? cs + PF_SLAB : P.E) - cs);
+    const int g = lane / LPR, li = lane % LPR;
+    const bool col_lane = li < P.nvec;
+
+    // the row holding position cs: largest r with rowptr[r] <= cs (32-way search)
+    int lo = 0, hi = P.N;
+    while (hi - lo > 1) {
+        const int step = (hi - lo + 31) / 32;
+        const int idx = min(lo + (lane + 1) * step, hi);
+        const bool le = idx < hi && P.rowptr[idx] <= cs;
+        const int k = __popc(__ballot_sync(0xffffffffu, le));
+        const int nlo = lo + k * step;
+        hi = min(nlo + step, hi);
+        lo = nlo;
+    }
+    const int cur0 = lo;
+    auto row_factor = [&](int64_t len) { return P.mean ? 1.0f / (float)(len > 1 ? len : 1) : 1.0f; };
+    for (int i = lane; i < n; i += 32) S.e[i] = make_int2(ld_hint_i32(P.col + cs + i, pol_stream), 0);
+    if (lane == 0) { S.srow[0] = cur0; S.sinv[0] = row_factor(P.rowptr[cur0 + 1] - P.rowptr[cur0]); }
+    __syncwarp();
+    for (int rb = cur0 + 1;; rb += 32) {  // non-empty rows starting inside the chunk
+        const int r = rb + lane;
+        bool live = false;
+        if (r < P.N) {
+            const int64_t rs = P.rowptr[r];
+            live = rs < cs + n;
+            if (live) {
+                const int64_t re = P.rowptr[r + 1];
+                if (re > rs) {
+                    const int k = (int)(rs - cs);
+                    S.srow[k] = r;
+                    S.sinv[k] = row_factor(re - rs);
+                    S.e[k].y = k;
+                }
+            }
+        }
+        if (!__all_sync(0xffffffffu, live)) break;
+    }
+    __syncwarp();
+    {  // prefix maximum of the start marks: lane owns positions 8*lane .. 8*lane+7
+        int m[8];
+        int run = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = lane * 8 + q;
+            run = max(run, i < n ? S.e[i].y : 0);
+            m[q] = run;
+        }
+        int incl = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl = max(incl, t);
+        }
+        int before = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) before = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = lane * 8 + q;
+            if (i < n) S.e[i].y = max(before, m[q]);
+        }
+    }
+    __syncwarp();
+
+    const int a = g * L, b = min(a + L, n);
+    const size_t row_bytes = (size_t)P.nvec * 16;
+    const char* Xl = reinterpret_cast<const char*>(P.X) + (size_t)(col_lane ? li : 0) * 16;
+    const char* Dl = reinterpret_cast<const char*>(P.dOut) + (size_t)(col_lane ? li : 0) * 16;
+    const int span = P.lph == 0 ? LPR : P.lph;  // lanes per result: the whole row, or one head
+    const bool writer = col_lane && (li % span) == 0;
+    const int head = P.lph == 0 ? 0 : li / P.lph, wstride = P.lph == 0 ? 1 : P.H;
+    const uint32_t row_bytes32 = (uint32_t)row_bytes;
+    for (int i = a; i < a + L; i += U) {  // same trip count in every lane: the shuffles below are warp-wide
+        uint4 xb[U], db[U];
+        int k[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool ok = i + u < b;
+            const int2 e = S.e[ok ? i + u : 0];
+            k[u] = ok ? e.y : -1;
+            if (ok) {
+                xb[u] = ld_hint16(Xl + (size_t)((uint32_t)e.x) * row_bytes32, pol_keep);
+                db[u] = __ldg(reinterpret_cast<const uint4*>(Dl + (size_t)((uint32_t)S.srow[e.y]) * row_bytes32));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float dot = 0.f;
+            if (k[u] >= 0 && col_lane) {
+                float x[EPC], d[EPC];
+                Chunk<T>::unpack(xb[u], x);
+                Chunk<T>::unpack(db[u], d);
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) dot = fmaf(x[j], d[j], dot);
+            }
+            for (int o = span >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (k[u] >= 0 && writer) P.dW[(cs + i + u) * wstride + head] = S.sinv[k[u]] * dot;
+        }
+    }
+}
+
 // ------------------------------------------------------------------ host dispatch
 bool pick_shape(int nvec, int* lpr, int* vpl) {
     if (nvec < 1 || nvec > 128) return false;
@@ -978,6 +1101,16 @@ static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStr
 
 template <typename T>
 static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st) {
+    if (vpl == 1 && P.E < (int64_t)8 * 1024 * 1024) {  // short-row regime: positions first
+        const int grid = (int)ceil_div(P.nchunks, FL_WARPS);
+        switch (lpr) {
+            case 4: sddmm_flat_kernel<T, 4><<<grid, FL_WARPS * 32, 0, st>>>(P); break;
+            case 8: sddmm_flat_kernel<T, 8><<<grid, FL_WARPS * 32, 0, st>>>(P); break;
+            case 16: sddmm_flat_kernel<T, 16><<<grid, FL_WARPS * 32, 0, st>>>(P); break;
+            default: sddmm_flat_kernel<T, 32><<<grid, FL_WARPS * 32, 0, st>>>(P); break;
+        }
+        return;
+    }
     const int grid = (int)ceil_div(P.nchunks, PF_WARPS);
     const int thr = PF_WARPS * 32;
 #define GNN_SD_CASE(L, V) \
