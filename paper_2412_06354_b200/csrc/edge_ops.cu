@@ -11,16 +11,26 @@ __device__ __forceinline__ int row_of_position(const int64_t* rowptr, int N, int
     return lower_bound_i64(rowptr, N + 1, p + 1) - 1;
 }
 
+// Grid-stride walk over (position, 16-byte chunk) pairs t = p*nvec + ci without a division per step:
+// one 64-bit division when the thread starts, then p and ci advance by the quotient and remainder of
+// the stride.
+struct PosChunk {
+    int64_t p, dp;
+    int ci, dci, nvec;
+    __device__ __forceinline__ PosChunk(int64_t t0, int64_t stride, int nv) : p(t0 / nv), dp(stride / nv), ci((int)(t0 % nv)), dci((int)(stride % nv)), nvec(nv) {}
+    __device__ __forceinline__ void next() {
+        p += dp;
+        ci += dci;
+        if (ci >= nvec) { ci -= nvec; ++p; }
+    }
+};
+
 // out[k, chunk] = X[idx[k], chunk]; one thread per 16-byte chunk
 __global__ void gather_rows_kernel(const int32_t* __restrict__ idx, int64_t E, const uint4* __restrict__ X,
                                    int nvec, uint4* __restrict__ out) {
     int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * nvec;
-    for (; t < total; t += stride) {
-        const int64_t k = t / nvec;
-        const int ci = (int)(t - k * nvec);
-        out[t] = X[(size_t)idx[k] * nvec + ci];
-    }
+    for (PosChunk q(t, stride, nvec); t < total; t += stride, q.next()) out[t] = X[(size_t)idx[q.p] * nvec + q.ci];
 }
 
 // m[p, f] = e[p, g(f)] * X[col[p], f]   (e == nullptr: plain copy of the source row)
@@ -31,14 +41,21 @@ __global__ void apply_edges_mul_kernel(const int32_t* __restrict__ col, int64_t 
     constexpr int EPC = Chunk<T>::N;
     int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * nvec;
-    for (; t < total; t += stride) {
-        const int64_t p = t / nvec;
-        const int ci = (int)(t - p * nvec);
+    const bool chunk_in_one = feats_per_e % EPC == 0;  // every 16-byte chunk lies under one multiplier
+    for (PosChunk q(t, stride, nvec); t < total; t += stride, q.next()) {
+        const int64_t p = q.p;
+        const int ci = q.ci;
         float x[EPC];
         Chunk<T>::unpack(X[(size_t)col[p] * nvec + ci], x);
         if (e) {
+            if (chunk_in_one) {
+                const float f = e[p * ew + (ci * EPC) / feats_per_e];
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) x[j] *= e[p * ew + (ci * EPC + j) / feats_per_e];
+                for (int j = 0; j < EPC; ++j) x[j] *= f;
+            } else {
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) x[j] *= e[p * ew + (ci * EPC + j) / feats_per_e];
+            }
         }
         m[t] = Chunk<T>::pack(x);
     }
@@ -50,9 +67,9 @@ __global__ void gat_logit_kernel(const int64_t* __restrict__ rowptr, const int32
                                  float slope, float* __restrict__ s) {
     int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * H;
-    for (; t < total; t += stride) {
-        const int64_t p = t / H;
-        const int h = (int)(t - p * H);
+    for (PosChunk q(t, stride, H); t < total; t += stride, q.next()) {
+        const int64_t p = q.p;
+        const int h = q.ci;
         const int i = row_of_position(rowptr, N, p);
         const float z = al[(size_t)col[p] * H + h] + ar[(size_t)i * H + h];
         s[t] = z > 0.f ? z : slope * z;
@@ -67,9 +84,9 @@ __global__ void aggregate_backward_kernel(const int64_t* __restrict__ rowptr, in
     constexpr int EPC = Chunk<T>::N;
     int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * nvec;
-    for (; t < total; t += stride) {
-        const int64_t p = t / nvec;
-        const int ci = (int)(t - p * nvec);
+    for (PosChunk q(t, stride, nvec); t < total; t += stride, q.next()) {
+        const int64_t p = q.p;
+        const int ci = q.ci;
         const int i = row_of_position(rowptr, N, p);
         uint4 raw = dOut[(size_t)i * nvec + ci];
         if (op == GNN_SUM) { dm[t] = raw; continue; }
