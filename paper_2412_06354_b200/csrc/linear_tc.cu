@@ -65,6 +65,23 @@ template <> struct Operand<float> {
     }
 };
 
+// Which 16-byte chunk (row r, chunk c) of a rows x chunks matrix thread-iteration e copies.  Register copies
+// (fp32 input, NS = 3) let eight consecutive threads take the eight rows of one core matrix, so their
+// 16-byte shared-memory stores are contiguous (no bank conflicts) while each still reads a full 32-byte
+// sector; cp.async copies (bf16) keep consecutive threads on consecutive chunks of a row.
+template <int NS>
+__device__ __forceinline__ void tile_coord(int e, int chunks, int* r, int* c) {
+    if (NS == 3) {
+        const int q = e >> 3;
+        const int rg = q / chunks;
+        *c = q - rg * chunks;
+        *r = rg * 8 + (e & 7);
+    } else {
+        *r = e / chunks;
+        *c = e - *r * chunks;
+    }
+}
+
 // products accumulated per k-step: levels (i of A, j of B), small terms first
 template <int NS> __device__ __forceinline__ int num_pairs() { return NS == 1 ? 1 : 6; }
 __device__ __constant__ unsigned char kPairA[6] = {2, 0, 1, 1, 0, 0};
@@ -122,10 +139,11 @@ linear_tc_kernel(const TcParams<T> P) {
         const int rows = P.b_transposed ? M : K, chunks = (P.b_transposed ? K : M) / 8;
 #pragma unroll 4
         for (int e = tid; e < rows * chunks; e += TC_THREADS) {
-            const int r = e / chunks, c = e - r * chunks;
+            int r, c;
+            tile_coord<NS>(e, chunks, &r, &c);
             const uint32_t off = P.b_transposed ? (uint32_t)(r >> 3) * sbo + (uint32_t)c * 128 + (uint32_t)(r & 7) * 16
                                                 : (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16;
-            Op::copy8(b0 + off, b_level, P.W + (size_t)e * 8, true);
+            Op::copy8(b0 + off, b_level, P.W + ((size_t)r * chunks + c) * 8, true);
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -143,7 +161,8 @@ linear_tc_kernel(const TcParams<T> P) {
         // X tile -> canonical K-major layout: chunk kc of row r at (r/8)*sbo + kc*128 + (r%8)*16
 #pragma unroll 4
         for (int e = tid; e < TC_ROWS * kchunks; e += TC_THREADS) {
-            const int r = e / kchunks, kc = e - r * kchunks;
+            int r, kc;
+            tile_coord<NS>(e, kchunks, &r, &kc);
             const bool in = row0 + r < P.N;
             Op::copy8(a0 + (uint32_t)(r >> 3) * sbo + (uint32_t)kc * 128 + (uint32_t)(r & 7) * 16, a_level,
                       P.X + (in ? ((size_t)(row0 + r) * kchunks + kc) * 8 : 0), in);
@@ -299,14 +318,16 @@ linear_tc_dw_kernel(const TcDwParams<T> P) {
         const int64_t row0 = t * TC_ROWS;
 #pragma unroll 4
         for (int e = tid; e < TC_ROWS * kc; e += TC_THREADS2) {
-            const int r = e / kc, c = e - r * kc;
+            int r, c;
+            tile_coord<NS>(e, kc, &r, &c);
             const bool in = row0 + r < P.N;
             Op::copy8(sa0 + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16, a_level,
                       P.X + (in ? ((size_t)(row0 + r) * kc + c) * 8 : 0), in);
         }
 #pragma unroll 4
         for (int e = tid; e < TC_ROWS * mc; e += TC_THREADS2) {
-            const int r = e / mc, c = e - r * mc;
+            int r, c;
+            tile_coord<NS>(e, mc, &r, &c);
             const bool in = row0 + r < P.N;
             Op::copy8(sb0 + (uint32_t)c * sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16, b_level,
                       P.dY + (in ? ((size_t)(row0 + r) * mc + c) * 8 : 0), in);
