@@ -123,6 +123,9 @@ gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int
 bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype);
 gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
                               cudaStream_t st);
+bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype);
+gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
+                                  cudaStream_t st);
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tma_dw_partials(int64_t N);
 gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
@@ -154,6 +157,7 @@ gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn
     cudaStream_t st = as_stream(stream);
     if (cudaMemsetAsync(ws, 0, sizeof(int), st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed (is ws a device pointer?)", who);
     if (linear_tma_supported(N, K, M, 0, dtype)) return linear_tma_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
+    if (linear_tma_f32_supported(N, K, M, dtype)) return linear_tma_f32_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
     if (linear_tc_supported(N, K, M, dtype)) return linear_tc_forward(X, W, N, K, M, 0, dtype, Y, (int*)ws, st);
     if (dtype == GNN_F32)
         launch_simt<float, float, float>((const float*)X, K, 1, (const float*)W, M, 1, (float*)Y, N, M, K, K, 1, 0, st);
@@ -180,6 +184,9 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         // dX[n,k] = sum_m dY[n,m] * W[k,m]
         if (linear_tma_supported(N, M, K, 1, dtype)) {
             gnn_status rc = linear_tma_forward(dY, W, N, M, K, 1, dX, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (linear_tma_f32_supported(N, M, K, dtype)) {
+            gnn_status rc = linear_tma_f32_forward(dY, W, N, M, K, 1, dX, (int*)ws, st);
             if (rc != GNN_OK) return rc;
         } else if (linear_tc_supported(N, M, K, dtype)) {
             gnn_status rc = linear_tc_forward(dY, W, N, M, K, 1, dtype, dX, (int*)ws, st);

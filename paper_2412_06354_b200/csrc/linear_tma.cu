@@ -269,6 +269,252 @@ gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, i
     return GNN_OK;
 }
 
+// ------------------------------------------------------------------ fp32: Y = X * B on the bf16 tensor cores
+// Every fp32 value is split exactly into three bf16 terms (x = x1 + x2 + x3, 8 mantissa bits each) and the
+// six products with i + j <= 4 are accumulated (the dropped ones are below 2^-23 of a product), which keeps
+// the fp32 tolerance.  Roles of the persistent CTA:
+//   warp 0      loader: X arrives as fp32 slices of 128 rows x 32 columns (128-byte rows, 128-byte swizzle)
+//               in a ring of shared-memory slots;
+//   warps 2..9  converters, two groups taking alternate slices: read a slice, split it, and write the three
+//               bf16 levels into the group's operand buffer in the tensor core's canonical no-swizzle
+//               layout (8 rows x 16 bytes per core matrix);
+//   warp 1      MMA issuer: 2 k-steps x 6 level pairs per slice into one of two accumulators;
+//   warps 10..17 epilogue: accumulator -> swizzled staging blocks of 32 rows x 32 columns -> bulk tensor stores to Y.
+// The weight matrix is split once per CTA by all warps before the roles start.
+constexpr int TF_CONV_WARPS = 8, TF_EPI_WARPS = 8;
+constexpr int TF_THREADS = 32 * (2 + TF_CONV_WARPS + TF_EPI_WARPS);
+constexpr int TF_KB = 32;                                  // contraction elements per slice
+constexpr uint32_t TF_SLICE_BYTES = TC_ROWS * TF_KB * 4;   // 16 KB of fp32
+constexpr uint32_t TF_LEVEL_BYTES = TC_ROWS * TF_KB * 2;   // 8 KB: one bf16 level of a slice
+constexpr int TF_MAX_STAGES = 6;
+
+__device__ __constant__ unsigned char kPairA3[6] = {2, 0, 1, 1, 0, 0};  // levels of A and B per product, small terms first
+__device__ __constant__ unsigned char kPairB3[6] = {0, 2, 1, 0, 1, 0};
+
+// 8 fp32 values -> three 16-byte chunks of bf16 (x = x1 + x2 + x3 exactly)
+__device__ __forceinline__ void split8(const float* xin, uint4* lv) {
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = xin[j];
+#pragma unroll
+    for (int l = 0; l < 3; ++l) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            __nv_bfloat162 b = __floats2bfloat162_rn(x[j], x[j + 1]);
+            w[j / 2] = *reinterpret_cast<uint32_t*>(&b);
+            // remainders are exact in fp32: the rounded term shares the leading bits of x
+            x[j] -= __uint_as_float(w[j / 2] << 16);
+            x[j + 1] -= __uint_as_float(w[j / 2] & 0xFFFF0000u);
+        }
+        lv[l] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+__device__ __forceinline__ void st_shared16(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared16(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+struct TmaF32Params {
+    const float* W;  // [Kc,Mo] (b_transposed = 0) or [Mo,Kc] (b_transposed = 1)
+    int64_t N;
+    int Kc, Mo;
+    int b_transposed;
+    int stages;
+    int acc_stride, tmem_cols;
+    int* status;
+};
+
+__global__ void __launch_bounds__(TF_THREADS, 1)
+linear_tma_f32_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY, const TmaF32Params P) {
+    extern __shared__ unsigned char smem_raw[];
+    // f_full[S], f_empty[S], o_full[2], o_empty[2], acc_full[2], acc_empty[2]
+    __shared__ __align__(8) uint64_t bars[2 * TF_MAX_STAGES + 8];
+    __shared__ uint32_t tmem_base_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Kc = P.Kc, Mo = P.Mo, S = P.stages;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int kchunks = Kc / 8;                    // 16-byte chunks of bf16 along the whole contraction
+    const uint32_t b_sbo = (uint32_t)kchunks * 128;  // weight levels: same layout as a whole-K operand
+    const uint32_t b_level = (uint32_t)Mo * Kc * 2;
+    const uint32_t w0 = base, ring0 = base + ((3 * b_level + 1023u) & ~1023u), op0 = ring0 + (uint32_t)S * TF_SLICE_BYTES;
+    const uint32_t stage0 = op0 + 2u * 3u * TF_LEVEL_BYTES;  // per epilogue warp: 32 rows x 32 fp32 columns of Y
+    const int nslices = (Kc + TF_KB - 1) / TF_KB;
+    const uint32_t bar0 = smem_u32(bars);
+    auto f_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto f_empty = [&](int s) { return bar0 + 8u * (uint32_t)(TF_MAX_STAGES + s); };
+    auto o_full = [&](int o) { return bar0 + 8u * (uint32_t)(2 * TF_MAX_STAGES + o); };
+    auto o_empty = [&](int o) { return bar0 + 8u * (uint32_t)(2 * TF_MAX_STAGES + 2 + o); };
+    auto acc_full = [&](int a) { return bar0 + 8u * (uint32_t)(2 * TF_MAX_STAGES + 4 + a); };
+    auto acc_empty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * TF_MAX_STAGES + 6 + a); };
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(f_full(s), 1); mbar_init(f_empty(s), TF_CONV_WARPS / 2); }
+        for (int o = 0; o < 2; ++o) {
+            mbar_init(o_full(o), TF_CONV_WARPS / 2); mbar_init(o_empty(o), 1);
+            mbar_init(acc_full(o), 1); mbar_init(acc_empty(o), TF_EPI_WARPS);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapY)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
+    // weight levels.  16-byte chunk c of stored row r:
+    //   stored [Kc,Mo] (MN-major B): r = k, c = 8 output columns: offset c*sbo + (k/8)*128 + (k%8)*16
+    //   stored [Mo,Kc] (K-major  B): r = n, c = 8 k's:            offset (n/8)*sbo + c*128 + (n%8)*16
+    // eight consecutive threads take the eight rows of one core matrix: contiguous 16-byte stores
+    {
+        const int rows = P.b_transposed ? Mo : Kc, chunks = (P.b_transposed ? Kc : Mo) / 8;
+        for (int e = tid; e < rows * chunks; e += TF_THREADS) {
+            const int q = e >> 3, rg = q / chunks, c = q - rg * chunks, r = rg * 8 + (e & 7);
+            const float4* src = reinterpret_cast<const float4*>(P.W + ((size_t)r * chunks + c) * 8);
+            const float4 lo = __ldg(src), hi = __ldg(src + 1);
+            const float x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            uint4 lv[3];
+            split8(x, lv);
+            const uint32_t off = P.b_transposed ? (uint32_t)(r >> 3) * b_sbo + (uint32_t)c * 128 + (uint32_t)(r & 7) * 16
+                                                : (uint32_t)c * b_sbo + (uint32_t)(r >> 3) * 128 + (uint32_t)(r & 7) * 16;
+#pragma unroll
+            for (int l = 0; l < 3; ++l) st_shared16(w0 + (uint32_t)l * b_level + off, lv[l]);
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const int64_t ntiles = (P.N + TC_ROWS - 1) / TC_ROWS;
+    bool failed = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint64_t stream = policy_evict_first();
+            uint32_t it = 0;
+            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x)
+                for (int j = 0; j < nslices; ++j, ++it) {
+                    const int s = (int)(it % (uint32_t)S);
+                    if (!mbar_wait_bounded(f_empty(s), ((it / (uint32_t)S) & 1u) ^ 1u)) { failed = true; break; }
+                    mbar_arrive_expect_tx(f_full(s), TF_SLICE_BYTES);
+                    tma_load_2d(ring0 + (uint32_t)s * TF_SLICE_BYTES, &mapX, j * TF_KB, (int)(t * TC_ROWS), f_full(s), stream);
+                }
+            if (failed) {
+                const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+                for (uint32_t i = first; i < it; ++i) mbar_wait_bounded(f_full((int)(i % (uint32_t)S)), (i / (uint32_t)S) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(Mo, P.b_transposed ? 0 : 1);
+            uint32_t it = 0, lt = 0;
+            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++lt) {
+                const uint32_t a = lt & 1u;
+                if (!mbar_wait_bounded(acc_empty((int)a), ((lt >> 1) & 1u) ^ 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t dacc = tmem_base + a * (uint32_t)P.acc_stride;
+                for (int j = 0; j < nslices; ++j, ++it) {
+                    const uint32_t o = it & 1u;
+                    if (!mbar_wait_bounded(o_full((int)o), (it >> 1) & 1u)) { failed = true; break; }
+                    tc_fence_after();
+                    const uint32_t abuf = op0 + o * 3u * TF_LEVEL_BYTES;
+                    const int ksteps = (Kc - j * TF_KB) >= TF_KB ? TF_KB / 16 : (Kc - j * TF_KB) / 16;
+                    for (int kk = 0; kk < ksteps; ++kk)
+                        for (int q = 0; q < 6; ++q) {
+                            // A slice: 4 chunks along k, core matrices 128 bytes apart, groups of 8 rows 512 bytes apart
+                            const uint64_t adesc = make_smem_desc(abuf + (uint32_t)kPairA3[q] * TF_LEVEL_BYTES + (uint32_t)kk * 256u, 128, 512);
+                            const uint64_t bdesc = make_smem_desc(w0 + (uint32_t)kPairB3[q] * b_level + (uint32_t)(j * (TF_KB / 16) + kk) * 256u, 128, b_sbo);
+                            mma_bf16_ss(dacc, adesc, bdesc, idesc, (j > 0 || kk > 0 || q > 0) ? 1u : 0u);
+                        }
+                    mma_commit(o_empty((int)o));
+                }
+                if (failed) break;
+                mma_commit(acc_full((int)a));
+            }
+        }
+    } else if (warp < 2 + TF_CONV_WARPS) {
+        // two groups of converter warps take alternate slices, each into its own operand buffer, so that
+        // two slices are being converted while the tensor core works on the ones before
+        constexpr int GT = 32 * TF_CONV_WARPS / 2;  // threads per group
+        const uint32_t grp = (uint32_t)(warp - 2) / (TF_CONV_WARPS / 2);
+        const int ct = (tid - 64) % GT;
+        uint32_t it = 0;
+        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x)
+            for (int j = 0; j < nslices; ++j, ++it) {
+                if ((it & 1u) != grp) continue;
+                const int s = (int)(it % (uint32_t)S);
+                const uint32_t o = grp;
+                if (!mbar_wait_bounded(f_full(s), (it / (uint32_t)S) & 1u)) { failed = true; break; }
+                if (!mbar_wait_bounded(o_empty((int)o), ((it >> 1) & 1u) ^ 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t src = ring0 + (uint32_t)s * TF_SLICE_BYTES, dst = op0 + o * 3u * TF_LEVEL_BYTES;
+#pragma unroll
+                for (int rep = 0; rep < (TC_ROWS * (TF_KB / 8)) / GT; ++rep) {
+                    const int e = ct + rep * GT;
+                    const int q = e >> 3, rg = q >> 2, kc = q & 3, r = rg * 8 + (e & 7);
+                    // fp32 row r: 128 bytes, 16-byte chunk c at position c ^ (r % 8)
+                    const uint4 c0 = ld_shared16(src + (uint32_t)r * 128u + (uint32_t)(((2 * kc) ^ (r & 7)) << 4));
+                    const uint4 c1 = ld_shared16(src + (uint32_t)r * 128u + (uint32_t)(((2 * kc + 1) ^ (r & 7)) << 4));
+                    const float x[8] = {__uint_as_float(c0.x), __uint_as_float(c0.y), __uint_as_float(c0.z), __uint_as_float(c0.w),
+                                        __uint_as_float(c1.x), __uint_as_float(c1.y), __uint_as_float(c1.z), __uint_as_float(c1.w)};
+                    uint4 lv[3];
+                    split8(x, lv);
+                    const uint32_t off = (uint32_t)(r >> 3) * 512u + (uint32_t)kc * 128u + (uint32_t)(r & 7) * 16u;
+#pragma unroll
+                    for (int l = 0; l < 3; ++l) st_shared16(dst + (uint32_t)l * TF_LEVEL_BYTES + off, lv[l]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(f_empty(s)); mbar_arrive(o_full((int)o)); }
+            }
+    } else {
+        const int ew = warp - (2 + TF_CONV_WARPS), quarter = warp & 3, half = ew >> 2;
+        const uint32_t stg = stage0 + (uint32_t)ew * 4096u;
+        uint32_t lt = 0;
+        for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++lt) {
+            const uint32_t a = lt & 1u;
+            if (!mbar_wait_bounded(acc_full((int)a), (lt >> 1) & 1u)) { failed = true; break; }
+            tc_fence_after();
+            const int64_t row0 = t * TC_ROWS + quarter * 32;  // first of this warp's 32 rows
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * (uint32_t)P.acc_stride;
+            for (int cb = half; cb * 32 < Mo; cb += 2) {  // blocks of 32 columns = 128-byte rows
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // staging block free again
+                __syncwarp();
+                const int groups = (Mo - cb * 32 >= 32 ? 32 : Mo - cb * 32) / 16;
+                for (int g16 = 0; g16 < groups; ++g16) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)(cb * 32 + g16 * 16), r);
+                    tmem_ld_wait();
+                    // row = lane, 128 bytes per row; 16-byte chunk c sits at position c ^ (row % 8)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        st_shared16(stg + (uint32_t)lane * 128u + ((uint32_t)((4 * g16 + q) ^ (lane & 7)) << 4),
+                                    make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]));
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && row0 < P.N) {  // rows past N are clipped by the copy engine
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                     reinterpret_cast<uint64_t>(&mapY)),
+                                 "r"(cb * 32), "r"((int)row0), "r"(stg)
+                                 : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty((int)a));
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+    if (failed) atomicExch(P.status, 7);  // GNN_ERR_TIMEOUT
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+}
+
 // ------------------------------------------------------------------ dW = X^T * dY
 // Contraction over the N rows.  A = X^T (features x rows) and B = dY (rows x columns) are both
 // MN-major as stored, so the same 64-column x 64-row swizzled boxes serve: a pipeline slot holds 64
@@ -413,6 +659,52 @@ gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M,
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_dw_kernel, 5, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;
     linear_tma_dw_kernel<<<linear_tma_dw_partials(N), TM_THREADS, 1024 + (size_t)P.stages * slot, st>>>(mapX, mapD, P);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+// row-major fp32 matrix [rows, cols]; box = 32 columns (128 bytes, swizzled) x box_rows rows
+static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+    EncodeTiledFn enc = encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static size_t tf_fixed_bytes(int Kc, int Mo) {
+    return 1024 + (((size_t)3 * Mo * Kc * 2 + 1023) & ~(size_t)1023) + 2 * 3 * (size_t)TF_LEVEL_BYTES + (size_t)TF_EPI_WARPS * 4096;
+}
+
+bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype) {
+    if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
+    if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
+    if (tf_fixed_bytes(Kc, Mo) + 2 * TF_SLICE_BYTES > TM_SMEM_MAX) return false;
+    return encoder() != nullptr;
+}
+
+gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
+                                  cudaStream_t st) {
+    const char* who = "gnn_linear (pipelined fp32 tensor-core path)";
+    GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
+    CUtensorMap mapX, mapY;
+    if (!make_map_f32(&mapX, X, N, Kc, TC_ROWS) || !make_map_f32(&mapY, Y, N, Mo, 32)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    TmaF32Params P;
+    P.W = (const float*)W; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
+    const size_t fixed = tf_fixed_bytes(Kc, Mo);
+    int stages = (int)((TM_SMEM_MAX - fixed) / TF_SLICE_BYTES);
+    P.stages = stages > TF_MAX_STAGES ? TF_MAX_STAGES : stages;
+    P.acc_stride = (Mo + 31) & ~31;
+    int cols = 32;
+    while (cols < 2 * P.acc_stride) cols <<= 1;
+    P.tmem_cols = cols;
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tma_f32_kernel, 6, TM_SMEM_MAX);
+    if (rc != GNN_OK) return rc;
+    const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
+    linear_tma_f32_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TF_THREADS, fixed + (size_t)P.stages * TF_SLICE_BYTES, st>>>(mapX, mapY, P);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
