@@ -48,7 +48,7 @@ TRAFFIC_GB = {
     "64:bf16:e_mul_xj:fwd": 2.59,
     "64:bf16:e_mul_xj:bwd": 2.59,
     "128:bf16:copy_xj:fwd": 6.38,
-    "128:bf16:copy_xj:bwd": 6.38,
+    "128:bf16:copy_xj:bwd": 6.37,
     "128:bf16:e_mul_xj:fwd": 6.89,
     "128:bf16:e_mul_xj:bwd": 6.89,
     "256:bf16:copy_xj:fwd": 19.25,
@@ -72,11 +72,11 @@ TRAFFIC_GB = {
     "128:f32:e_mul_xj:fwd": 19.87,
     "128:f32:e_mul_xj:bwd": 19.83,
     "256:f32:copy_xj:fwd": 38.74,
-    "256:f32:copy_xj:bwd": 38.67,
+    "256:f32:copy_xj:bwd": 38.68,
     "256:f32:e_mul_xj:fwd": 39.77,
     "256:f32:e_mul_xj:bwd": 39.7,
     "512:f32:copy_xj:fwd": 77.53,
-    "512:f32:copy_xj:bwd": 77.37,
+    "512:f32:copy_xj:bwd": 77.36,
     "512:f32:e_mul_xj:fwd": 79.59,
     "512:f32:e_mul_xj:bwd": 79.42,
 }
