@@ -58,7 +58,7 @@ def run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, what):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("H,C", [(4, 16), (8, 32), (1, 64), (2, 8)])
+@pytest.mark.parametrize("H,C", [(4, 16), (8, 32), (1, 64), (2, 8), (16, 8), (32, 8)])
 def test_gat_ragged(gnn, dtype, H, C):
     n, src, dst = ragged_graph(90 + H)
     Wx = synth.normal((n, H * C), dtype, 900 + H, 1)
