@@ -278,8 +278,12 @@ gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_
 /* ------------------------------------------------------------------ dense node-wise transform */
 
 /* Y = X * W (the Dense layer / the weight of a conv layer in the training example): X [N,K],
- * W [K,M], Y [N,M], all row-major and of dtype.  bf16 with K and M multiples of 16 (16..256)
- * runs on the tensor cores with fp32 accumulation; other cases use an fp32 FFMA kernel.
+ * W [K,M], Y [N,M], all row-major and of dtype, 16-byte aligned.  With K and M multiples of 16
+ * (16..256) the product runs on the tensor cores with fp32 accumulation: bf16 directly, fp32 (when
+ * the weight matrix is small enough to sit in shared memory three times, e.g. 128x128) by an exact
+ * three-term bf16 split of every value, which keeps fp32 accuracy.  Other cases use an fp32 FFMA
+ * kernel.  The first call on a device looks up the driver's tensor-map encoder; the calls
+ * themselves allocate nothing.
  * ws: gnn_linear_workspace(N, K, M) bytes; its first 4 bytes are a device status word that the
  * tensor-core path sets to GNN_ERR_TIMEOUT if one of its bounded waits expired (0 otherwise);
  * read it after synchronising if you want to check. */
@@ -288,8 +292,8 @@ gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn
                       void* ws, size_t ws_bytes, gnn_stream stream);
 
 /* dX = dY * W^T ([N,K]) and dW = X^T * dY ([K,M], of dtype); either output may be NULL.  dW sums
- * over the N rows in slabs of 4096 rows whose fp32 partials are added in slab order, so the
- * result is reproducible.  X is needed only for dW, W only for dX. */
+ * over the N rows in fixed slabs (one per thread block) whose fp32 partials are added in a
+ * fixed order, so the result is reproducible.  X is needed only for dW, W only for dX. */
 gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int32_t N, int K, int M,
                                gnn_dtype dtype, void* dX, void* dW, void* ws, size_t ws_bytes,
                                gnn_stream stream);
