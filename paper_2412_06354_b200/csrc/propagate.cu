@@ -4,7 +4,8 @@
 // Work decomposition: the E positions of the sparse form are cut into fixed chunks of PF_CHUNK
 // consecutive edges (256 or 1024), one warp per chunk (merge-path style: perfect balance on power-law rows
 // without any per-graph schedule).  A warp finds its first row by binary search in rowptr and
-// walks the rows that start inside its chunk.  Rows lying wholly inside the chunk are reduced
+// walks the rows that start inside its chunk (runs of rows without edges are jumped over with one
+// search; their zero result comes from a separate row scan).  Rows lying wholly inside the chunk are reduced
 // and written directly.  A row cut by a chunk boundary leaves fp32 partials (one "head" slot and
 // one "tail" slot per chunk) that a second kernel combines in ascending chunk order.  Every
 // accumulation order is a fixed function of (E, F, dtype), so results are bit-reproducible and
@@ -90,6 +91,49 @@ __device__ __forceinline__ bool beats(float cv, int32_t ca, float v, int32_t a) 
     if (a < 0) return true;
     bool better = (MODE == MODE_MAX) ? (cv > v) : (cv < v);
     return better || (cv == v && ca < a);
+}
+
+// Smallest row r in [lo, N) with rowptr[r + 1] > v, or N: the first row at or after lo that has a
+// position beyond v.  Warp-cooperative (every lane must call it with the same arguments): a look at the
+// next 32 rows, then a 32-way search.
+__device__ __forceinline__ int first_row_ending_after(const int64_t* __restrict__ rowptr, int lo, int N, int64_t v, int lane) {
+    {  // the common case, one coalesced load: the row is among the next 32
+        const int r = lo + lane;
+        const unsigned m = __ballot_sync(0xffffffffu, r >= N || rowptr[r + 1] > v);
+        if (m) return min(lo + __ffs(m) - 1, N);
+        lo += 32;
+    }
+    int hi = N;
+    while (hi > lo) {
+        const int step = (hi - lo + 31) / 32;
+        const int idx = lo + lane * step;
+        const bool le = idx < hi && rowptr[idx + 1] <= v;  // true for a prefix of the lanes
+        const int k = __popc(__ballot_sync(0xffffffffu, le));
+        if (k == 0) { hi = lo; break; }
+        const int nlo = lo + (k - 1) * step + 1;
+        hi = min(lo + k * step, hi);
+        lo = nlo;
+    }
+    return lo;
+}
+
+// Rows without edges get their (empty) result from a scan that is independent of the edge chunks:
+// warp c of nchunks takes rows [c*per, (c+1)*per) and calls write_row(r) for each empty one, so a
+// long run of such rows (a bipartite graph's source side, say) is spread over all warps.
+template <class WriteRow>
+__device__ __forceinline__ void scan_empty_rows(const int64_t* __restrict__ rowptr, int N, int64_t c, int64_t nchunks, int lane, WriteRow write_row) {
+    const int64_t per = (N + nchunks - 1) / nchunks;
+    const int64_t b0 = c * per;
+    const int r0 = (int)(b0 < N ? b0 : N), r1 = (int)(b0 + per < N ? b0 + per : N);
+    for (int rb = r0; rb < r1; rb += 32) {
+        const int r = rb + lane;
+        unsigned em = __ballot_sync(0xffffffffu, r < r1 && rowptr[r + 1] == rowptr[r]);
+        while (em) {
+            const int bit = __ffs(em) - 1;
+            em &= em - 1;
+            write_row(rb + bit);
+        }
+    }
 }
 
 // per-warp staging area for one slab of PF_SLAB consecutive positions:
@@ -336,7 +380,8 @@ propagate_chunk_kernel(const PropParams P) {
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
     const int64_t cs = c * P.chunk;
     const int64_t ce = (cs + P.chunk < P.E) ? cs + P.chunk : P.E;
-    const bool last = (c == P.nchunks - 1);
+
+    typename W::A acc;
 
     // cur = the row containing position cs, or the first (possibly empty) row starting at cs
     int cur = lower_bound_i64(P.rowptr, P.N + 1, cs);
@@ -344,9 +389,13 @@ propagate_chunk_kernel(const PropParams P) {
     int64_t pos = cs;
     int64_t sb = cs - PF_SLAB;  // nothing staged yet
     int32_t tail = -1;
-    typename W::A acc;
     while (cur < P.N) {
         const int64_t rs = P.rowptr[cur], re = P.rowptr[cur + 1];
+        if (re == rs) {  // no edges (written by the scan above): jump to the next row that has some
+            cur = first_row_ending_after(P.rowptr, cur + 1, P.N, rs, lane);
+            if (cur >= P.N || P.rowptr[cur] >= ce) break;  // it belongs to a later chunk
+            continue;
+        }
         const int64_t b = re < ce ? re : ce;
         acc.clear();
         const int64_t pos0 = pos;
@@ -366,7 +415,7 @@ propagate_chunk_kernel(const PropParams P) {
             if (started_here) W::write_final(P, cur, re - rs, lane, acc);
             else W::write_partial(P, c, 0, lane, acc);
             ++cur;
-            if (!(re < ce || last)) break;  // the next row starts in the next chunk
+            if (re >= ce) break;  // the next row with edges starts in the next chunk
         } else {  // the row continues in the next chunk
             W::write_partial(P, c, started_here ? 1 : 0, lane, acc);
             if (started_here) tail = cur;
@@ -374,6 +423,11 @@ propagate_chunk_kernel(const PropParams P) {
         }
     }
     if (lane == 0) P.tail_row[c] = tail;
+    // rows without edges, after the walk so that the hot loop's register allocation is undisturbed
+    scan_empty_rows(P.rowptr, P.N, c, P.nchunks, lane, [&](int r) {
+        acc.clear();
+        W::write_final(P, r, 0, lane, acc);
+    });
 }
 
 // second pass: finish the rows that were cut by chunk boundaries, in ascending chunk order
@@ -446,8 +500,8 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
 //   3. rows cut by a run boundary are stitched inside the warp in run order (through shared
 //      memory), rows cut by the chunk boundary leave the same head / tail partials as the
 //      row-walking kernel, so the same fix-up pass finishes them.
-// Empty rows are zero-filled by the chunk after whose last position they come (chunk 0 also takes
-// the leading ones).  All orders are fixed functions of (E, F, dtype).
+// Rows without edges are written by a row scan that is spread over all warps (scan_empty_rows).
+// All orders are fixed functions of (E, F, dtype).
 constexpr int FL_WARPS = 4;
 constexpr int FL_U = 8;
 
@@ -543,35 +597,30 @@ propagate_flat_kernel(const PropParams P) {
     if (lane < 8) { S.hk[lane] = -1; S.hclosed[lane] = 0; S.tk[lane] = -1; }
     __syncwarp();
 
-    // ---- 1c. rows after cur0 that start in (cs, cs+n]: mark non-empty ones, fill empty ones
-    if (c == 0)  // leading empty rows
-        for (int r = 0; r < cur0; ++r) store_empty_row(r);
-    for (int rb = cur0 + 1;; rb += 32) {
+    // ---- 1c. rows after cur0 that start inside the chunk: mark the ones that have edges.  (Rows without
+    // edges are written by the row scan below; a run of them is jumped over with one search.)
+    for (int rb = cur0 + 1; rb < P.N;) {
         const int r = rb + lane;
         int64_t rs = 0, re = 0;
         bool live = false;
         if (r < P.N) {
             rs = P.rowptr[r];
-            live = rs <= cs + n;  // rows starting exactly at the chunk end: only their empty ones are ours
+            live = rs < cs + n;
             if (live) re = P.rowptr[r + 1];
         }
-        const bool empty = live && re == rs;
-        if (live && !empty && rs < cs + n) {
+        if (live && re > rs) {
             const int k = (int)(rs - cs);
             S.srow[k] = r;
             S.send[k] = rel_end(re);
             S.sinv[k] = row_factor(re - rs);
             S.e[k].y = k;
         }
-        unsigned em = __ballot_sync(0xffffffffu, empty);
-        while (em) {
-            const int bit = __ffs(em) - 1;
-            em &= em - 1;
-            store_empty_row(rb + bit);
-        }
         // rowptr is non-decreasing: once a lane is past the chunk (or past the last row) so are all later rows
         if (!__all_sync(0xffffffffu, live)) break;
+        if (__all_sync(0xffffffffu, re == rs)) rb = first_row_ending_after(P.rowptr, rb + 32, P.N, __shfl_sync(0xffffffffu, rs, 0), lane);
+        else rb += 32;
     }
+    scan_empty_rows(P.rowptr, P.N, c, P.nchunks, lane, store_empty_row);
     __syncwarp();
 
     // ---- 1d. prefix maximum of the start marks: lane owns positions 8*lane .. 8*lane+7

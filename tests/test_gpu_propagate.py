@@ -341,3 +341,33 @@ def test_chunk_regimes_with_empty_rows_everywhere(gnn, e, dtype, F):
         dX, _ = gnn.propagate_fused_backward(g, to_dev(R), op, argmax=arg)
         bw = oracle.propagate_backward(op, n, src, dst, X, None, R, arg=a)
         assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, f"{op} backward E={e}")
+
+
+@pytest.mark.parametrize("dtype,F", [("bf16", 64), ("f32", 16), ("bf16", 512)])
+def test_long_runs_of_rows_without_edges(gnn, dtype, F):
+    """A bipartite-like graph: 200000 nodes of which only 2000 in the middle receive edges, with one more
+    run of 40000 empty rows between two of them.  Both the short-row kernel (F*s <= 512 bytes) and the
+    row-walking kernel (wider rows) must jump over the runs and still zero every empty row."""
+    n, e = 200_000, 50_000
+    rng = np.random.default_rng(F)
+    dst = rng.integers(90_000, 92_000, e).astype(np.int32)
+    dst[dst >= 91_000] += 40_000
+    src = rng.integers(0, n, e).astype(np.int32)
+    g = build_graph(gnn, n, src, dst)
+    ref = host_csr(n, src, dst)
+    X = feats((n, F), dtype, 400 + F)
+    Xd = to_dev(X)
+    for op in ("sum", "mean"):
+        out = gnn.propagate_fused(g, Xd, None, op)
+        o, S, _ = oracle.propagate(op, n, src, dst, X)
+        assert_close(to_host64(out), o, S, dtype, f"{op} with long empty runs")
+    out, arg = gnn.propagate_fused(g, Xd, None, "max")
+    o, _, a = oracle.propagate("max", n, src, dst, X)
+    assert np.array_equal(bits(out), f64_to_dtype_bits(o, dtype))
+    ga = arg.cpu().numpy()
+    assert np.array_equal(np.where(ga >= 0, ref["eid"][np.maximum(ga, 0)], -1), a)
+    # the transposed form has the runs elsewhere (sources are spread over all nodes)
+    R = feats((n, F), dtype, 401 + F)
+    dX, _ = gnn.propagate_fused_backward(g, to_dev(R), "sum")
+    bw = oracle.propagate_backward("sum", n, src, dst, X, None, R)
+    assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, "backward with long empty runs")
