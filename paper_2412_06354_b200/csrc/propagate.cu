@@ -891,7 +891,7 @@ sddmm_chunk_kernel(const SddmmParams P) {
     int r = lower_bound_i64(P.rowptr, P.N + 1, cs + 1) - 1;
     int64_t pos = cs;
     while (pos < ce) {
-        while (P.rowptr[r + 1] <= pos) ++r;  // skip rows that end at or before pos
+        r = first_row_ending_after(P.rowptr, r, P.N, pos, lane);  // skip rows that end at or before pos
         const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
         const int64_t b = re < ce ? re : ce;
         float d[VPL][EPC];
@@ -1009,23 +1009,25 @@ sddmm_flat_kernel(const SddmmParams P) {
     for (int i = lane; i < n; i += 32) S.e[i] = make_int2(ld_hint_i32(P.col + cs + i, pol_stream), 0);
     if (lane == 0) { S.srow[0] = cur0; S.sinv[0] = row_factor(P.rowptr[cur0 + 1] - P.rowptr[cur0]); }
     __syncwarp();
-    for (int rb = cur0 + 1;; rb += 32) {  // non-empty rows starting inside the chunk
+    for (int rb = cur0 + 1; rb < P.N;) {  // non-empty rows starting inside the chunk
         const int r = rb + lane;
+        int64_t rs = 0, re = 0;
         bool live = false;
         if (r < P.N) {
-            const int64_t rs = P.rowptr[r];
+            rs = P.rowptr[r];
             live = rs < cs + n;
-            if (live) {
-                const int64_t re = P.rowptr[r + 1];
-                if (re > rs) {
-                    const int k = (int)(rs - cs);
-                    S.srow[k] = r;
-                    S.sinv[k] = row_factor(re - rs);
-                    S.e[k].y = k;
-                }
-            }
+            if (live) re = P.rowptr[r + 1];
+        }
+        if (live && re > rs) {
+            const int k = (int)(rs - cs);
+            S.srow[k] = r;
+            S.sinv[k] = row_factor(re - rs);
+            S.e[k].y = k;
         }
         if (!__all_sync(0xffffffffu, live)) break;
+        // 32 rows without edges: jump over the rest of the run
+        if (__all_sync(0xffffffffu, re == rs)) rb = first_row_ending_after(P.rowptr, rb + 32, P.N, __shfl_sync(0xffffffffu, rs, 0), lane);
+        else rb += 32;
     }
     __syncwarp();
     {  // prefix maximum of the start marks: lane owns positions 8*lane .. 8*lane+7

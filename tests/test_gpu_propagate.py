@@ -371,3 +371,7 @@ def test_long_runs_of_rows_without_edges(gnn, dtype, F):
     dX, _ = gnn.propagate_fused_backward(g, to_dev(R), "sum")
     bw = oracle.propagate_backward("sum", n, src, dst, X, None, R)
     assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, "backward with long empty runs")
+    # edge-weight gradient: one dot product per edge, rows found across the runs
+    _, dW = gnn.propagate_fused_backward(g, to_dev(R), "sum", X=Xd, want_dX=False, want_dW=True)
+    bw = oracle.propagate_backward("sum", n, src, dst, X, np.ones(e, np.float32), R, want_dX=False, want_dw=True)
+    assert_close(to_host64(dW), bw["dw"][ref["eid"]], bw["Sdw"][ref["eid"]], "f32", "dW with long empty runs")
