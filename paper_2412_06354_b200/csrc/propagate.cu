@@ -456,7 +456,27 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
             for (int j = 0; j < EPC; ++j) a[j] = pa[j];
         }
     }
-    for (int64_t cc = c + 1; cc <= c_end; ++cc) {
+    // a hub row is cut into hundreds of chunks: eight chunks' partials are loaded together (independent
+    // loads), then combined in ascending chunk order
+    int64_t cc = c + 1;
+    if (!ARG) {
+        for (; cc + 8 <= c_end + 1; cc += 8) {
+            float4 t[8][EPC / 4];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float4* pv = reinterpret_cast<const float4*>(P.part_val + ((size_t)(cc + u) * 2) * F + (size_t)ci * EPC);
+#pragma unroll
+                for (int q = 0; q < EPC / 4; ++q) t[u][q] = pv[q];
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int q = 0; q < EPC / 4; ++q) {
+                    v[4 * q] += t[u][q].x; v[4 * q + 1] += t[u][q].y; v[4 * q + 2] += t[u][q].z; v[4 * q + 3] += t[u][q].w;
+                }
+        }
+    }
+    for (; cc <= c_end; ++cc) {
         const float* pv = P.part_val + ((size_t)cc * 2) * F + (size_t)ci * EPC;
         if (ARG) {
             const int32_t* pa = P.part_arg + ((size_t)cc * 2) * F + (size_t)ci * EPC;
