@@ -273,7 +273,7 @@ gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, c
     GNN_REQUIRE(g->E == 0 || g->col, GNN_ERR_INVALID_ARG, "%s: null col", who);
     rc = gat_alpha(g, al, ar, slope, H, alpha_csr, st);
     if (rc != GNN_OK) return rc;
-    HeadExtra hx = {alpha_csr, H, nullptr, nullptr, nullptr, nullptr};
+    HeadExtra hx = {alpha_csr, nullptr, H, nullptr, nullptr, nullptr, nullptr};
     return run_chunked(who, MODE_HEADSUM, g->N, g->E, g->rowptr, g->col, nullptr, Wx, out, nullptr, nullptr,
                        nullptr, nullptr, 0, H * C, dtype, w.chunk_ws, w.chunk_bytes, st, &hx);
 }
@@ -327,11 +327,13 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
     gat_da_final_kernel<<<(int)ceil_div(F, 16), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
     GNN_CHECK_LAUNCH(who);
     // dWx[j,h,:] = sum_q alpha[t2f[q],h]*dOut[colT[q],h,:] + dal[j,h]*a_src[h,:] + dar[j,h]*a_dst[h,:]
-    if (g->E > 0) {
+    // the flat kernel reads alpha through t2f; the row-walking one wants it permuted to transposed order first
+    const bool indexed = chunked_is_flat(g->E, F, dtype);
+    if (g->E > 0 && !indexed) {
         rc = gnn_permute_edge_data(g->t2f, g->E, H, 4, alpha_csr, w.alphaT, stream);
         if (rc != GNN_OK) return rc;
     }
-    HeadExtra hx = {w.alphaT, H, w.dal, w.dar, a_src, a_dst};
+    HeadExtra hx = {indexed ? alpha_csr : w.alphaT, indexed ? g->t2f : nullptr, H, w.dal, w.dar, a_src, a_dst};
     return run_chunked(who, MODE_HEADSUM, g->N, g->E, g->rowptrT, g->colT, nullptr, dOut, dWx, nullptr, nullptr,
                        nullptr, nullptr, 0, F, dtype, w.chunk_ws, w.chunk_bytes, st, &hx);
 }

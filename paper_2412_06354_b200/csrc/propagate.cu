@@ -54,6 +54,7 @@ struct PropParams {
     int32_t* part_arg;  // [nchunks][2][F] (MODE_MAX/MIN)
     // MODE_HEADSUM: multiplier per (position, head), features of head h = [h*fph, (h+1)*fph)
     const float* wh;  // [E,H]
+    const int32_t* wh_index;  // flat kernel only: row of wh per position, or nullptr (= the position)
     int H, fph;
     // optional rank-1 epilogue: out[r,f] += epi_l[r,h(f)]*epi_a[f] + epi_r[r,h(f)]*epi_b[f]
     const float *epi_l, *epi_r, *epi_a, *epi_b;
@@ -610,7 +611,9 @@ propagate_flat_kernel(const PropParams P) {
             const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
             w = w / (float)(d > 1 ? d : 1);
         }
-        const int t = (MODE == MODE_ROUTE) ? ld_hint_i32(P.route_pos + cs + i, pol_stream) : 0;
+        int t = 0;
+        if (MODE == MODE_ROUTE) t = ld_hint_i32(P.route_pos + cs + i, pol_stream);
+        if (MODE == MODE_HEADSUM) t = P.wh_index ? ld_hint_i32(P.wh_index + cs + i, pol_stream) : (int)(cs + i);  // E < 2^31 here
         S.e[i] = make_int4(cc, 0, __float_as_int(w), t);
     }
     if (lane == 0) { S.srow[0] = cur0; S.send[0] = rel_end(re0); S.sinv[0] = row_factor(re0 - rs0); }
@@ -709,7 +712,7 @@ propagate_flat_kernel(const PropParams P) {
     };
     const int32_t* const route_l = (MODE == MODE_ROUTE) ? P.route_arg + (size_t)(col_lane ? li : 0) * EPC : nullptr;
     // per-head mode: this lane's head column of the [E,H] multiplier matrix, at the chunk's first position
-    const float* const wh_l = (MODE == MODE_HEADSUM) ? P.wh + (size_t)cs * P.H + ((col_lane ? li : 0) * EPC) / P.fph : nullptr;
+    const float* const wh_l = (MODE == MODE_HEADSUM) ? P.wh + ((col_lane ? li : 0) * EPC) / P.fph : nullptr;
     for (int i = a; i < b; i += U) {
         uint4 buf[U];
         float hw[MODE == MODE_HEADSUM ? U : 1];
@@ -722,7 +725,7 @@ propagate_flat_kernel(const PropParams P) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
-                if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(i + u) * P.H);
+                if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
                 if (MODE == MODE_ROUTE) {
 #pragma unroll
                     for (int q = 0; q < EPC / 4; ++q)
@@ -736,7 +739,7 @@ propagate_flat_kernel(const PropParams P) {
                 if (u < nu) {
                     const int cc = S.e[i + u].x;
                     buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * P.x_ld, pol_keep);
-                    if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(i + u) * P.H);
+                    if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
                     if (MODE == MODE_ROUTE) {
 #pragma unroll
                         for (int q = 0; q < EPC / 4; ++q)
@@ -1221,6 +1224,11 @@ static PfWs pf_carve(void* ws, int64_t E, int F, bool with_arg) {
 
 size_t chunked_workspace(int64_t E, int F, bool with_arg) { return pf_carve(nullptr, E, F, with_arg).bytes; }
 
+bool chunked_is_flat(int64_t E, int F, gnn_dtype dtype) {
+    const int nvec = F * elem_size(dtype) / 16;
+    return E > 0 && chunk_edges(E) <= PF_SLAB && nvec >= 1 && nvec <= 32;
+}
+
 gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const int64_t* rowptr,
                        const int32_t* col, const float* w, const void* X, void* out,
                        int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
@@ -1244,12 +1252,13 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
     P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
-    P.wh = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
+    P.wh = nullptr; P.wh_index = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
     if (hx) {
         const int epc = 16 / s;
         GNN_REQUIRE(mode == MODE_HEADSUM && (hx->wh || E == 0) && hx->H >= 1 && F % hx->H == 0 && (F / hx->H) % epc == 0, GNN_ERR_UNSUPPORTED,
                     "%s: per-head weights need F divisible by H and F/H a multiple of %d elements", who, epc);
-        P.wh = hx->wh; P.H = hx->H; P.fph = F / hx->H;
+        GNN_REQUIRE(!hx->wh_index || chunked_is_flat(E, F, dtype), GNN_ERR_INVALID_ARG, "%s: indexed per-head weights need the flat kernel", who);
+        P.wh = hx->wh; P.wh_index = hx->wh_index; P.H = hx->H; P.fph = F / hx->H;
         P.epi_l = hx->epi_l; P.epi_r = hx->epi_r; P.epi_a = hx->epi_a; P.epi_b = hx->epi_b;
     } else {
         GNN_REQUIRE(mode != MODE_HEADSUM, GNN_ERR_INVALID_ARG, "%s: per-head mode without weights", who);

@@ -13,6 +13,7 @@ enum { MODE_SUM = 0, MODE_MAX = 1, MODE_MIN = 2, MODE_ROUTE = 3, MODE_HEADSUM = 
 //   out[r,f] += epi_l[r,h(f)] * epi_a[f] + epi_r[r,h(f)] * epi_b[f]
 struct HeadExtra {
     const float* wh;  // [E,H]
+    const int32_t* wh_index;  // nullptr: position p uses row p of wh; else row wh_index[p] (only where chunked_is_flat())
     int H;
     const float *epi_l, *epi_r;  // [rows,H] or nullptr
     const float *epi_a, *epi_b;  // [F]
@@ -22,6 +23,9 @@ struct HeadExtra {
 bool pick_shape(int nvec, int* lpr, int* vpl);
 
 size_t chunked_workspace(int64_t E, int F, bool with_arg);
+
+// does run_chunked use the position-first (flat) kernel for this problem?  (It honours HeadExtra::wh_index.)
+bool chunked_is_flat(int64_t E, int F, gnn_dtype dtype);
 
 // out[r,:] = reduce over positions p of row r of  w[p] * X[col[p],:]   (see propagate.cu)
 gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const int64_t* rowptr,
