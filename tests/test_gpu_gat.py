@@ -58,7 +58,7 @@ def run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, what):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("H,C", [(4, 16), (8, 32), (1, 64), (2, 8), (16, 8), (32, 8)])
+@pytest.mark.parametrize("H,C", [(4, 16), (8, 32), (1, 64), (2, 8), (16, 8), (32, 8), (8, 64)])
 def test_gat_ragged(gnn, dtype, H, C):
     n, src, dst = ragged_graph(90 + H)
     Wx = synth.normal((n, H * C), dtype, 900 + H, 1)
@@ -100,5 +100,21 @@ def test_gat_attention_workload_full_size(gnn):
     oracle.set_threads(8)
     try:
         run_case(gnn, wl["N"], wl["src"], wl["dst"], wl["Wx"], wl["a_src"], wl["a_dst"], wl["H"], wl["C"], "bf16", "attention workload")
+    finally:
+        oracle.set_threads(1)
+
+
+def test_gat_more_than_8mi_edges_uses_the_row_walking_kernels(gnn):
+    """8.4 M edges: above the size where the per-head gather, its transposed form (with the permuted
+    coefficients) and the per-head dot products switch from the position-first kernels to the row-walking ones."""
+    n, E, H, C = 200_000, 8_400_000, 4, 8
+    src, dst = synth.rmat(18, n, E, 4321, symmetric=False)
+    Wx = synth.normal_f32((n, H * C), 4322)
+    a = (6.0 / (C + 1)) ** 0.5
+    a_s = synth.uniform_f32((H, C), -a, a, 4323)
+    a_d = synth.uniform_f32((H, C), -a, a, 4324)
+    oracle.set_threads(8)
+    try:
+        run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, "f32", "gat 8.4M edges")
     finally:
         oracle.set_threads(1)
