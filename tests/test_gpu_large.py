@@ -75,3 +75,32 @@ def test_propagate_sampled_rows_full_size(big, dtype, F):
     # properties that hold at any size: isolated targets get exact zeros; column sums match a direct sum
     iso = torch.from_numpy(np.nonzero(deg_in == 0)[0][:5000]).cuda()
     assert torch.count_nonzero(out[iso]) == 0
+
+
+def test_mean_max_and_backward_of_max_full_size(big):
+    """The row-walking kernel's other modes at a size where it (not the position-first kernel) runs:
+    mean on sampled rows, max with winner positions on every row (bit-exact), routing backward on sampled rows."""
+    import torch
+    from util import bits, f64_to_dtype_bits
+    gnn, wl, g = big
+    n, src, dst, seed = wl["N"], wl["src"], wl["dst"], wl["seed"]
+    F = 32
+    X = synth.normal_f32((n, F), seed, 22)
+    R = synth.normal_f32((n, F), seed, 23)
+    Xd, Rd = torch.from_numpy(X).cuda(), torch.from_numpy(R).cuda()
+    rows = sample_rows(np.bincount(dst, minlength=n), 9)
+    out = gnn.propagate_fused(g, Xd, None, "mean")
+    o, S, _ = oracle.propagate("mean", n, src, dst, X, None, rows=rows)
+    assert_close(to_host64(out[torch.from_numpy(rows).cuda()]), o, S, "f32", "mean")
+    out, arg = gnn.propagate_fused(g, Xd, None, "max")
+    o, _, a = oracle.propagate("max", n, src, dst, X)
+    assert np.array_equal(bits(out), f64_to_dtype_bits(o, "f32"))
+    del o
+    eid = g.eid.cpu().numpy()
+    ga = arg.cpu().numpy()
+    assert np.array_equal(np.where(ga >= 0, eid[np.maximum(ga, 0)], -1), a)
+    del eid, ga
+    dX, _ = gnn.propagate_fused_backward(g, Rd, "max", argmax=arg)
+    rows_s = sample_rows(np.bincount(src, minlength=n), 10)
+    bw = oracle.propagate_backward("max", n, src, dst, X, None, R, arg=a, rows=rows_s)
+    assert_close(to_host64(dX[torch.from_numpy(rows_s).cuda()]), bw["dX"], bw["SdX"], "f32", "backward of max")
