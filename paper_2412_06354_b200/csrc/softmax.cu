@@ -119,7 +119,8 @@ struct LongRows {
     int count;
 };
 
-template <bool LONG, int NT, int THRESH = SM_LONG_ROW, class Body>
+// SUB (non-LONG only): threads per row, 32 (a warp) or 8; LO: rows of at most LO positions belong to another kernel.
+template <bool LONG, int NT, int THRESH = SM_LONG_ROW, int SUB = 32, int LO = -1, class Body>
 __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr, int N, LongRows& L, Body body) {
     if (LONG) {
         const int per = (N + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -138,11 +139,11 @@ __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr,
             }
         }
     } else {
-        int row = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-        const int stride = (int)((gridDim.x * (int64_t)blockDim.x) >> 5);
+        int row = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) / SUB);
+        const int stride = (int)((gridDim.x * (int64_t)blockDim.x) / SUB);
         for (; row < N; row += stride) {
             const int64_t a = rowptr[row], b = rowptr[row + 1];
-            if (b - a > THRESH) continue;  // uniform per warp
+            if (b - a > THRESH || b - a <= LO) continue;  // uniform per group of SUB threads
             body(row, a, b);
         }
     }
@@ -212,13 +213,17 @@ gat_alpha_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__
 // ---- position-per-lane layout for H = 4*HV heads: a lane owns whole positions (all heads of an
 // edge as HV float4), so a row of up to 32 edges is one vector load per array per lane, and the
 // per-head reductions run over lanes (warp) or over lanes and warps (block, long rows).
+// NT < 32: the reduction runs over aligned groups of NT lanes, which may have diverged from the other
+// groups of the warp, so the shuffles name only the group's lanes.
 template <int HV, int NT, bool IS_MAX>
 __device__ __forceinline__ void reduce_heads(float (&v)[4 * HV], float* red) {
+    constexpr int W = NT < 32 ? NT : 32;
+    const unsigned mask = W == 32 ? 0xffffffffu : (((1u << W) - 1u) << ((threadIdx.x & 31) / W * W));
 #pragma unroll
     for (int j = 0; j < 4 * HV; ++j) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[j], o);
+        for (int o = W / 2; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(mask, v[j], o);
             v[j] = IS_MAX ? fmaxf(v[j], other) : (((threadIdx.x & o) == 0) ? v[j] + other : other + v[j]);
         }
     }
@@ -248,15 +253,18 @@ __host__ __device__ constexpr int pl_unroll(int HV) { return HV <= 2 ? 4 : (HV =
 // the gathers of a batch (col, then al[col]) are independent.  A row that fits in one batch (the
 // common case) keeps its logits in registers through the max, sum and normalise steps; longer rows
 // park the logits in alpha and re-read them.
-template <int HV, bool LONG>
+template <int HV, bool LONG, int SUB = 32>
 __global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK, LONG ? 1 : (HV <= 2 ? 3 : 2))
 gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                     const float* __restrict__ al, const float* __restrict__ ar, float slope, float* __restrict__ alpha) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : SUB, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
+    // three kernels share the rows: SUB = 8 takes rows that fit one batch of 8 threads, SUB = 32 the rest up to
+    // PL_LONG_ROW, LONG the longer ones
+    constexpr int ROW_MAX = LONG ? PL_LONG_ROW : (SUB == 8 ? 8 * U : PL_LONG_ROW), ROW_LO = (!LONG && SUB == 32) ? 8 * U : -1;
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
-    const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
+    const int tid = LONG ? threadIdx.x : (threadIdx.x & (SUB - 1));
     __shared__ LongRows lrows;
-    for_each_row<LONG, PL_BLOCK, PL_LONG_ROW>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+    for_each_row<LONG, PL_BLOCK, ROW_MAX, SUB, ROW_LO>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) return;
         float arv[H], m[H], zs[H];
 #pragma unroll
@@ -351,18 +359,21 @@ gat_alpha_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restric
 }
 
 // backward rows: d[h] = sum_p alpha*dalpha; dz = alpha*(dalpha - d)*LeakyReLU'(z), written over dalpha; dar = sum_p dz
-template <int HV, bool LONG>
+template <int HV, bool LONG, int SUB = 32>
 __global__ void __launch_bounds__(LONG ? PL_BLOCK : SM_BLOCK, LONG ? 1 : (HV <= 2 ? 3 : 2))
 gat_rows_bwd_pl_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                        const float* __restrict__ alpha, float* __restrict__ dalpha_dz, const float* __restrict__ al,
                        const float* __restrict__ ar, float slope, float* __restrict__ dar) {
-    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : 32, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
+    constexpr int H = 4 * HV, NT = LONG ? PL_BLOCK : SUB, U = LONG ? pl_unroll(HV) : (pl_unroll(HV) > 2 ? 2 : pl_unroll(HV));
+    // three kernels share the rows: SUB = 8 takes rows that fit one batch of 8 threads, SUB = 32 the rest up to
+    // PL_LONG_ROW, LONG the longer ones
+    constexpr int ROW_MAX = LONG ? PL_LONG_ROW : (SUB == 8 ? 8 * U : PL_LONG_ROW), ROW_LO = (!LONG && SUB == 32) ? 8 * U : -1;
     __shared__ float red[LONG ? (PL_BLOCK / 32) * 32 : 1];
-    const int tid = LONG ? threadIdx.x : (threadIdx.x & 31);
+    const int tid = LONG ? threadIdx.x : (threadIdx.x & (SUB - 1));
     __shared__ LongRows lrows;
-    for_each_row<LONG, PL_BLOCK, PL_LONG_ROW>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
+    for_each_row<LONG, PL_BLOCK, ROW_MAX, SUB, ROW_LO>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) {
-            if (tid < H) dar[(size_t)row * H + tid] = 0.f;
+            for (int j = tid; j < H; j += NT) dar[(size_t)row * H + j] = 0.f;
             return;
         }
         float arv[H], d[H], sdz[H];
@@ -442,10 +453,17 @@ static int row_grid_pl(int N, bool is_long) {
     return (int)(want < cap ? (want > 0 ? want : 1) : cap);
 }
 
+// eight threads per row
+static int row_grid_sub(int N) {
+    const int64_t want = ceil_div((int64_t)N * 8, SM_BLOCK), cap = (int64_t)148 * 64;
+    return (int)(want < cap ? (want > 0 ? want : 1) : cap);
+}
+
 gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float slope, int H, float* alpha, cudaStream_t st) {
     if (g->N == 0 || g->E == 0) return GNN_OK;
-    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true);
+    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true), sg = row_grid_sub(g->N);
 #define GNN_GA(HV)                                                                                                    \
+    gat_alpha_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);       \
     gat_alpha_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);          \
     gat_alpha_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);
     if (H == 4) { GNN_GA(1) } else if (H == 8) { GNN_GA(2) } else if (H == 16) { GNN_GA(4) } else if (H == 32) { GNN_GA(8) } else {
@@ -460,8 +478,9 @@ gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float s
 // returns false if H is not handled here (caller falls back to its generic kernel)
 bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz, const float* al, const float* ar,
                           float slope, int H, float* dar, cudaStream_t st) {
-    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true);
+    const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true), sg = row_grid_sub(g->N);
 #define GNN_GB(HV)                                                                                                               \
+    gat_rows_bwd_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar); \
     gat_rows_bwd_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);  \
     gat_rows_bwd_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);
     if (H == 4) { GNN_GB(1) } else if (H == 8) { GNN_GB(2) } else if (H == 16) { GNN_GB(4) } else if (H == 32) { GNN_GB(8) } else return false;
