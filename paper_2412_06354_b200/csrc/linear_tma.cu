@@ -275,9 +275,8 @@ gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, i
 // the fp32 tolerance.  Roles of the persistent CTA:
 //   warp 0      loader: X arrives as fp32 slices of 128 rows x 32 columns (128-byte rows, 128-byte swizzle)
 //               in a ring of shared-memory slots;
-//   warps 2..9  converters, two groups taking alternate slices: read a slice, split it, and write the three
-//               bf16 levels into the group's operand buffer in the tensor core's canonical no-swizzle
-//               layout (8 rows x 16 bytes per core matrix);
+//   warps 2..9  converters: read a slice, split it, and write the three bf16 levels into one of two operand
+//               buffers in the tensor core's canonical no-swizzle layout (8 rows x 16 bytes per core matrix);
 //   warp 1      MMA issuer: 2 k-steps x 6 level pairs per slice into one of two accumulators;
 //   warps 10..17 epilogue: accumulator -> swizzled staging blocks of 32 rows x 32 columns -> bulk tensor stores to Y.
 // The weight matrix is split once per CTA by all warps before the roles start.
@@ -353,9 +352,9 @@ linear_tma_f32_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     auto acc_empty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * TF_MAX_STAGES + 6 + a); };
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(f_full(s), 1); mbar_init(f_empty(s), TF_CONV_WARPS / 2); }
+        for (int s = 0; s < S; ++s) { mbar_init(f_full(s), 1); mbar_init(f_empty(s), TF_CONV_WARPS); }
         for (int o = 0; o < 2; ++o) {
-            mbar_init(o_full(o), TF_CONV_WARPS / 2); mbar_init(o_empty(o), 1);
+            mbar_init(o_full(o), TF_CONV_WARPS); mbar_init(o_empty(o), 1);
             mbar_init(acc_full(o), 1); mbar_init(acc_empty(o), TF_EPI_WARPS);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -435,17 +434,16 @@ linear_tma_f32_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
             }
         }
     } else if (warp < 2 + TF_CONV_WARPS) {
-        // two groups of converter warps take alternate slices, each into its own operand buffer, so that
-        // two slices are being converted while the tensor core works on the ones before
-        constexpr int GT = 32 * TF_CONV_WARPS / 2;  // threads per group
-        const uint32_t grp = (uint32_t)(warp - 2) / (TF_CONV_WARPS / 2);
-        const int ct = (tid - 64) % GT;
+        // Every converter warp works on every slice, in order: a waiter that skipped uses of a slot would
+        // find the parity of an older completed phase and run ahead of the copy (parity waits only tell
+        // the last two phases apart), so the slices are not divided among groups of warps.
+        constexpr int GT = 32 * TF_CONV_WARPS;
+        const int ct = tid - 64;
         uint32_t it = 0;
         for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x)
             for (int j = 0; j < nslices; ++j, ++it) {
-                if ((it & 1u) != grp) continue;
                 const int s = (int)(it % (uint32_t)S);
-                const uint32_t o = grp;
+                const uint32_t o = it & 1u;
                 if (!mbar_wait_bounded(f_full(s), (it / (uint32_t)S) & 1u)) { failed = true; break; }
                 if (!mbar_wait_bounded(o_empty((int)o), ((it >> 1) & 1u) ^ 1u)) { failed = true; break; }
                 tc_fence_after();
@@ -535,7 +533,8 @@ struct TmaDwParams {
 };
 
 __global__ void __launch_bounds__(TM_THREADS, 1)
-linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapD, const TmaDwParams P) {
+linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapD,
+                     const __grid_constant__ CUtensorMap mapP, const TmaDwParams P) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bars[2 * TM_MAX_STAGES + 1];  // full[S], empty[S], acc_full
     __shared__ uint32_t tmem_base_slot;
@@ -555,6 +554,7 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapD)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapP)) : "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
     tc_fence_before();
@@ -608,21 +608,37 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
             failed = true;
         } else {
             tc_fence_after();
-            float* part = P.part + (size_t)blockIdx.x * K * M;
+            // the pipeline slots are idle now (every load was consumed before the last commit): each warp
+            // stages 32 feature rows x 32 columns of fp32 there and sends them with a bulk tensor store
+            const uint32_t stg = base + (uint32_t)ew * 4096u;
             for (int h = 0; h < halves; ++h) {
-                const int krow = h * 128 + quarter * 32 + lane;
+                const int prow0 = (int)blockIdx.x * K + h * 128 + quarter * 32;  // row of the [parts*K, M] partial matrix
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * M);
-                for (int c0 = half * 16; c0 < M; c0 += 32) {
-                    uint32_t r[16];
-                    tmem_ld16(taddr + (uint32_t)c0, r);
-                    tmem_ld_wait();
-                    float4* dst = reinterpret_cast<float4*>(part + (size_t)krow * M + c0);
+                for (int cb = half; cb * 32 < M; cb += 2) {
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+                    const int groups = (M - cb * 32 >= 32 ? 32 : M - cb * 32) / 16;
+                    for (int g16 = 0; g16 < groups; ++g16) {
+                        uint32_t r[16];
+                        tmem_ld16(taddr + (uint32_t)(cb * 32 + g16 * 16), r);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
-                                             __uint_as_float(r[4 * q + 3]));
+                        for (int q = 0; q < 4; ++q)
+                            st_shared16(stg + (uint32_t)lane * 128u + ((uint32_t)((4 * g16 + q) ^ (lane & 7)) << 4),
+                                        make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]));
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                         reinterpret_cast<uint64_t>(&mapP)),
+                                     "r"(cb * 32), "r"(prow0), "r"(stg)
+                                     : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
                 }
             }
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         }
     }
     if (failed) atomicExch(P.status, 7);
@@ -642,12 +658,16 @@ int linear_tma_dw_partials(int64_t N) {
     return (int)(nchunks < 148 ? (nchunks > 0 ? nchunks : 1) : 148);
 }
 
+static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows);
+
 // writes linear_tma_dw_partials(N) fp32 partials [K,M] to part
 gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
     const char* who = "gnn_linear_backward (pipelined tensor-core dW)";
     GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
-    CUtensorMap mapX, mapD;
-    if (!make_map(&mapX, X, N, K, DW_ROWS) || !make_map(&mapD, dY, N, M, DW_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    CUtensorMap mapX, mapD, mapP;
+    if (!make_map(&mapX, X, N, K, DW_ROWS) || !make_map(&mapD, dY, N, M, DW_ROWS) ||
+        !make_map_f32(&mapP, part, (int64_t)linear_tma_dw_partials(N) * K, M, 32))
+        GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaDwParams P;
     P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
     const size_t slot = (size_t)(K / 64 + (M + 63) / 64) * DW_BOX_BYTES;
@@ -658,7 +678,7 @@ gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M,
     P.tmem_cols = cols;
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_dw_kernel, 5, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;
-    linear_tma_dw_kernel<<<linear_tma_dw_partials(N), TM_THREADS, 1024 + (size_t)P.stages * slot, st>>>(mapX, mapD, P);
+    linear_tma_dw_kernel<<<linear_tma_dw_partials(N), TM_THREADS, 1024 + (size_t)P.stages * slot, st>>>(mapX, mapD, mapP, P);
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }

@@ -87,3 +87,25 @@ def test_linear_degenerate(gnn):
     with pytest.raises(gnn.GnnError) as e:
         gnn.linear(torch.zeros((8, 64), device="cuda"), W, ws=torch.empty(8, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_linear_back_to_back_launches_are_bitwise_identical(gnn, dtype):
+    """Forty launches in a row with nothing in between (the pipelines' barrier phases and ring slots are
+    reused at full speed): every result must equal the first one bit for bit, and no wait may expire."""
+    import torch
+    n, K, M = 170_000, 128, 128
+    X = to_dev(synth.normal((n, K), dtype, 1200))
+    W32 = synth.glorot_f32(K, M, 1201)
+    W = to_dev(W32) if dtype == "f32" else torch.from_numpy(W32).to(torch.bfloat16).cuda()
+    dY = to_dev(synth.normal((n, M), dtype, 1202))
+    ws = torch.empty(gnn.load().gnn_linear_workspace(n, K, M), dtype=torch.uint8, device="cuda")
+    Y0 = gnn.linear(X, W, ws=ws).clone()
+    dX0, dW0 = (t.clone() for t in gnn.linear_backward(X, W, dY, ws=ws))
+    for _ in range(40):
+        Y = gnn.linear(X, W, ws=ws)
+        dX, dW = gnn.linear_backward(X, W, dY, ws=ws)
+    torch.cuda.synchronize()
+    assert status_word(ws) == 0
+    assert torch.equal(Y.view(torch.int16 if dtype == "bf16" else torch.int32), Y0.view(torch.int16 if dtype == "bf16" else torch.int32))
+    assert torch.equal(dX.float(), dX0.float()) and torch.equal(dW.float(), dW0.float())
