@@ -178,11 +178,12 @@ def run_reference(args, rank):
 WORKLOAD_NAME = "large sparse aggregation sweep: R-MAT N=2.4M E=123M (a=.57 b=.19 c=.19, symmetrised, relabelled, sorted by dst), F in {32,64,128,256,512} x {bf16,f32}, copy_xj+sum and e_mul_xj+sum, fwd + bwd dX"
 
 
-def cpu_sample(synth, pairs=1_000_000, F=128):
+def cpu_sample(synth, pairs=16_000_000, F=128):
     """A smaller graph of the same family for the CPU checker: R-MAT with the same parameters and
-    the same mean degree (N=39,024, 2,000,000 directed edges), bf16 features of width 128."""
+    the same mean degree (N=624,390, 32,000,000 directed edges), bf16 features of width 128: a few
+    seconds of work per forward + backward pair on 16 cores."""
     n = 2_400_000 * (2 * pairs) // 123_000_000
-    src, dst = synth.rmat(16, n, pairs, synth.BASE_SEED + 5, symmetric=True, relabel=True, sort_by_dst=True)
+    src, dst = synth.rmat(20, n, pairs, synth.BASE_SEED + 5, symmetric=True, relabel=True, sort_by_dst=True)
     return dict(N=n, E=len(src), F=F, src=src, dst=dst, X=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 20),
                 R=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 21), w=synth.uniform_f32((len(src),), 0, 1, synth.BASE_SEED + 5, 13),
                 desc=f"same generator at N={n}, E={2 * pairs} (same mean degree), F={F} bf16, e_mul_xj+sum fwd + bwd dX, fp64")
