@@ -991,8 +991,7 @@ sddmm_chunk_kernel(const SddmmParams P) {
 // Same idea as propagate_flat_kernel: positions first, rows second.  The warp stages the gathered
 // rows of its 256 positions and finds, by marking row starts and a prefix maximum, the row of every
 // position; each lane group then takes a contiguous run and issues, per batch of 4 positions, the
-// independent loads of X[col[p]] and dOut[row(p)] (the latter mostly from L1: neighbouring positions
-// share it).  Every position is independent, so there are no partials and no second pass.
+// independent loads of X[col[p]] and, where the row changes, dOut[row(p)].  Every position is independent, so there are no partials and no second pass.
 constexpr int SF_U = 4;
 
 struct SddmmFlatSmem {
@@ -1086,31 +1085,47 @@ sddmm_flat_kernel(const SddmmParams P) {
     const bool writer = col_lane && (li % span) == 0;
     const int head = P.lph == 0 ? 0 : li / P.lph, wstride = P.lph == 0 ? 1 : P.H;
     const uint32_t row_bytes32 = (uint32_t)row_bytes;
+    int kprev = -1;   // start entry of the position before this batch
+    uint4 dcur = make_uint4(0, 0, 0, 0);  // this lane's chunk of the current row of dOut: reloaded only when the row changes
     for (int i = a; i < a + L; i += U) {  // same trip count in every lane: the shuffles below are warp-wide
         uint4 xb[U], db[U];
         int k[U];
+        bool fresh[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const bool ok = i + u < b;
             const int2 e = S.e[ok ? i + u : 0];
             k[u] = ok ? e.y : -1;
-            if (ok) {
-                xb[u] = ld_hint16(Xl + (size_t)((uint32_t)e.x) * row_bytes32, pol_keep);
-                db[u] = __ldg(reinterpret_cast<const uint4*>(Dl + (size_t)((uint32_t)S.srow[e.y]) * row_bytes32));
-            }
+            fresh[u] = ok && k[u] != (u == 0 ? kprev : k[u - 1]);
+            if (ok) xb[u] = ld_hint16(Xl + (size_t)((uint32_t)e.x) * row_bytes32, pol_keep);
+            if (fresh[u]) db[u] = __ldg(reinterpret_cast<const uint4*>(Dl + (size_t)((uint32_t)S.srow[e.y]) * row_bytes32));
         }
+        kprev = k[U - 1];
+        float res[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
+            if (fresh[u]) dcur = db[u];
             float dot = 0.f;
             if (k[u] >= 0 && col_lane) {
                 float x[EPC], d[EPC];
                 Chunk<T>::unpack(xb[u], x);
-                Chunk<T>::unpack(db[u], d);
+                Chunk<T>::unpack(dcur, d);
 #pragma unroll
                 for (int j = 0; j < EPC; ++j) dot = fmaf(x[j], d[j], dot);
             }
             for (int o = span >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            if (k[u] >= 0 && writer) P.dW[(cs + i + u) * wstride + head] = S.sinv[k[u]] * dot;
+            res[u] = k[u] >= 0 ? S.sinv[k[u]] * dot : 0.f;
+            if (P.lph != 0 && k[u] >= 0 && writer) P.dW[(cs + i + u) * wstride + head] = res[u];  // H values side by side per position
+        }
+        if (P.lph == 0 && writer) {  // one value per position: the batch's U results leave as one 16-byte store
+            static_assert(SF_U == 4, "the vector store below writes four results");
+            if (i + U <= b) {
+                *reinterpret_cast<float4*>(P.dW + cs + i) = make_float4(res[0], res[1], res[2], res[3]);
+            } else {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (k[u] >= 0) P.dW[cs + i + u] = res[u];
+            }
         }
     }
 }
@@ -1175,7 +1190,7 @@ static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStr
 
 template <typename T>
 static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st) {
-    if (vpl == 1 && P.E < (int64_t)8 * 1024 * 1024) {  // short-row regime: positions first
+    if (vpl == 1) {  // positions first
         const int grid = (int)ceil_div(P.nchunks, FL_WARPS);
         switch (lpr) {
             case 4: sddmm_flat_kernel<T, 4><<<grid, FL_WARPS * 32, 0, st>>>(P); break;

@@ -1,11 +1,11 @@
 """Device times of single library calls on the four smaller synthetic workloads.
 
-    python -m paper_2412_06354_b200.microbench [linear] [propagate] [gat] [--plain]
+    python -m paper_2412_06354_b200.microbench [linear] [propagate] [gat] [large] [--plain]
 
 Each call is captured 20 times into one CUDA graph; the reported time is the replay time divided by 20
 (CUDA events on the capturing stream), so launch gaps of the Python binding are not in it.  With
 --plain every call runs three times without graph capture (for a profiler) and nothing is timed.
-The large-graph sweep is bench.py's job, not this tool's.
+The large-graph sweep is bench.py's job; `large` (not run by default) adds the edge-weight gradient on that graph.
 """
 from __future__ import annotations
 
@@ -105,11 +105,30 @@ def bench_gat(plain):
     row("config 4 gat_fused backward", device_time_us(lambda: gnn.gat_fused_backward(g, Wx, a_s, a_d, fwd, Wx, H), plain))
 
 
+def bench_large(plain):
+    """Edge-weight gradient (one dot product per edge) on the large power-law graph, beside the dX pass."""
+    wl = synth.workload_large_graph()
+    g = gnn.coo_to_csr(wl["N"], to_dev(wl["src"]), to_dev(wl["dst"]))
+    n, E = wl["N"], g.E
+    del wl
+    for F, dt in [(32, torch.bfloat16), (128, torch.bfloat16), (128, torch.float32), (512, torch.float32)]:
+        gen = torch.Generator(device="cuda").manual_seed(F)
+        X = torch.randn(n, F, device="cuda", generator=gen).to(dt)
+        R = torch.randn(n, F, device="cuda", generator=gen).to(dt)
+        dW = torch.empty(E, dtype=torch.float32, device="cuda")
+        dX = torch.empty_like(X)
+        ws = torch.empty(gnn.propagate_fused_workspace(E, F, "sum"), dtype=torch.uint8, device="cuda")
+        tag = f"large graph (N={n}, E={E}) F={F} {'bf16' if dt == torch.bfloat16 else 'f32'} backward of sum: "
+        row(tag + "dX", device_time_us(lambda: gnn.propagate_fused_backward(g, R, "sum", dX=dX, ws=ws), plain))
+        row(tag + "edge-weight gradient", device_time_us(lambda: gnn.propagate_fused_backward(g, R, "sum", X=X, want_dX=False, want_dW=True, dW=dW, ws=ws), plain))
+        del X, R, dW, dX, ws
+
+
 def main(argv):
     plain = "--plain" in argv
     which = [a for a in argv if not a.startswith("--")] or ["linear", "propagate", "gat"]
     gnn.load()
-    table = {"linear": bench_linear, "propagate": bench_propagate, "gat": bench_gat}
+    table = {"linear": bench_linear, "propagate": bench_propagate, "gat": bench_gat, "large": bench_large}
     for w in which:
         table[w](plain)
 

@@ -104,3 +104,17 @@ def test_mean_max_and_backward_of_max_full_size(big):
     rows_s = sample_rows(np.bincount(src, minlength=n), 10)
     bw = oracle.propagate_backward("max", n, src, dst, X, None, R, arg=a, rows=rows_s)
     assert_close(to_host64(dX[torch.from_numpy(rows_s).cuda()]), bw["dX"], bw["SdX"], "f32", "backward of max")
+
+
+def test_edge_weight_gradient_full_size(big):
+    """One dot product per edge on all 123 M edges (F = 32, fp32), against the CPU checker."""
+    import torch
+    gnn, wl, g = big
+    n, src, dst, seed = wl["N"], wl["src"], wl["dst"], wl["seed"]
+    F = 32
+    X = synth.normal_f32((n, F), seed, 24)
+    R = synth.normal_f32((n, F), seed, 25)
+    _, dW = gnn.propagate_fused_backward(g, torch.from_numpy(R).cuda(), "sum", X=torch.from_numpy(X).cuda(), want_dX=False, want_dW=True)
+    bw = oracle.propagate_backward("sum", n, src, dst, X, np.ones(len(src), np.float32), R, want_dX=False, want_dw=True)
+    eid = g.eid.cpu().numpy()
+    assert_close(to_host64(dW), bw["dw"][eid], bw["Sdw"][eid], "f32", "edge-weight gradient, all edges")
