@@ -1101,30 +1101,41 @@ sddmm_flat_kernel(const SddmmParams P) {
             if (fresh[u]) db[u] = __ldg(reinterpret_cast<const uint4*>(Dl + (size_t)((uint32_t)S.srow[e.y]) * row_bytes32));
         }
         kprev = k[U - 1];
-        float res[U];
+        static_assert(SF_U == 4, "the reductions below fold four positions at a time");
+        float dot[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (fresh[u]) dcur = db[u];
-            float dot = 0.f;
+            dot[u] = 0.f;
             if (k[u] >= 0 && col_lane) {
                 float x[EPC], d[EPC];
                 Chunk<T>::unpack(xb[u], x);
                 Chunk<T>::unpack(dcur, d);
 #pragma unroll
-                for (int j = 0; j < EPC; ++j) dot = fmaf(x[j], d[j], dot);
+                for (int j = 0; j < EPC; ++j) dot[u] = fmaf(x[j], d[j], dot[u]);
             }
-            for (int o = span >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            res[u] = k[u] >= 0 ? S.sinv[k[u]] * dot : 0.f;
-            if (P.lph != 0 && k[u] >= 0 && writer) P.dW[(cs + i + u) * wstride + head] = res[u];  // H values side by side per position
         }
-        if (P.lph == 0 && writer) {  // one value per position: the batch's U results leave as one 16-byte store
-            static_assert(SF_U == 4, "the vector store below writes four results");
-            if (i + U <= b) {
-                *reinterpret_cast<float4*>(P.dW + cs + i) = make_float4(res[0], res[1], res[2], res[3]);
-            } else {
+        if (span >= 4) {
+            // fold the four positions while reducing over the span lanes: the first two levels halve the values
+            // a lane carries (2 + 1 shuffles), the rest reduce the one left; the quarter of the span a lane
+            // sits in decides which position it ends up with: 6 shuffles for 32 lanes instead of 20
+            const int h1 = span >> 1, h2 = span >> 2;
+            const bool up1 = (li & h1) != 0, up2 = (li & h2) != 0;
+            const float s0 = up1 ? dot[0] : dot[2], s1 = up1 ? dot[1] : dot[3];
+            const float r0 = (up1 ? dot[2] : dot[0]) + __shfl_xor_sync(0xffffffffu, s0, h1);
+            const float r1 = (up1 ? dot[3] : dot[1]) + __shfl_xor_sync(0xffffffffu, s1, h1);
+            float v = (up2 ? r1 : r0) + __shfl_xor_sync(0xffffffffu, up2 ? r0 : r1, h2);
+            for (int o = span >> 3; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            const int mine = (up1 ? 2 : 0) + (up2 ? 1 : 0);  // the position of the batch this lane holds
+            const int km = mine == 0 ? k[0] : mine == 1 ? k[1] : mine == 2 ? k[2] : k[3];
+            // any lane of the span may end up holding a result (with whole-row results also a lane past a narrow row)
+            if ((P.lph == 0 || col_lane) && (li & (h2 - 1)) == 0 && km >= 0) P.dW[(cs + i + mine) * wstride + head] = S.sinv[km] * v;
+        } else {  // heads of one or two 16-byte chunks
 #pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (k[u] >= 0) P.dW[cs + i + u] = res[u];
+            for (int u = 0; u < U; ++u) {
+                float v = dot[u];
+                for (int o = span >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (k[u] >= 0 && writer) P.dW[(cs + i + u) * wstride + head] = S.sinv[k[u]] * v;
             }
         }
     }
