@@ -3,9 +3,12 @@
 //   dX = dY * W^T      dY [N,M]
 //   dW = X^T * dY      reduction over the N rows, split over row slabs and combined in slab order
 //
-// Two paths.  bf16 with K, M multiples of 16 (M <= 256, K <= 256) runs Y and dX on the 5th-generation
-// tensor cores (tcgen05.mma, accumulators in tensor memory); everything else (fp32, odd shapes, dW)
-// runs a shared-memory tiled FFMA kernel with fp32 accumulation.  All sums have a fixed order.
+// This file holds the entry points, their dispatch, and the fallback.  With K and M multiples of 16
+// (16..256) the products run on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
+// memory): the pipelined kernels of linear_tma.cu (bf16: Y, dX, dW; fp32: Y, dX) or the
+// single-buffered ones of linear_tc.cu (fp32 dW, fp32 weights too large for the pipeline, and bf16 when
+// the tensor-map encoder is not available).  Everything else runs the shared-memory tiled FFMA kernel
+// below with fp32 accumulation.  All sums have a fixed order.
 #include "common.cuh"
 
 namespace gnn {

@@ -1,4 +1,6 @@
-// Tensor-core path of the dense node-wise transform: Y[N,M] = X[N,K] * B, bf16 operands, fp32
+// Single-buffered tensor-core kernels of the dense node-wise transform (the pipelined ones are in
+// linear_tma.cu; these serve fp32 dW, fp32 weights too large for the pipeline, and bf16 when no
+// tensor-map encoder is available): Y[N,M] = X[N,K] * B, bf16 operands, fp32
 // accumulation in tensor memory (tcgen05.mma, sm_100a).  fp32 inputs run on the same bf16 MMAs:
 // every value is split exactly into three bf16 terms (x = x1 + x2 + x3, 8 mantissa bits each) while
 // the tile is copied to shared memory, and the six products with i + j <= 4 are accumulated
