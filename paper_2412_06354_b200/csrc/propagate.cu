@@ -1,8 +1,12 @@
 // Fused propagate (Sec. 3 "Message Passing": apply_edges + aggregate_neighbors combined into a
 // generalised sparse x dense product) and its backward passes.
 //
-// Work decomposition: the E positions of the sparse form are cut into fixed chunks of PF_CHUNK
-// consecutive edges (256 or 1024), one warp per chunk (merge-path style: perfect balance on power-law rows
+// Two kernels share one decomposition and one fix-up pass: the row-walking kernel below (graphs of
+// 8 Mi edges and more, and rows wider than 512 bytes) and the position-first kernel further down
+// (propagate_flat_kernel: smaller graphs, whose rows are mostly a handful of edges).
+//
+// Work decomposition: the E positions of the sparse form are cut into fixed chunks of
+// consecutive edges (64 to 1024, by graph size), one warp per chunk (merge-path style: perfect balance on power-law rows
 // without any per-graph schedule).  A warp finds its first row by binary search in rowptr and
 // walks the rows that start inside its chunk (runs of rows without edges are jumped over with one
 // search; their zero result comes from a separate row scan).  Rows lying wholly inside the chunk are reduced
