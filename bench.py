@@ -342,12 +342,13 @@ def main():
     tkey = "%d:%s:%s:fwd" % (dom["F"], dom["dtype"], dom["msg"])
     traffic = TRAFFIC_GB.get(tkey) if shrink == 0 and not args.natural_ids else None
     achieved = comp / dom["fwd_ms"] / 1e6
-    roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel, forward launch of F=%d %s %s (largest share of the step: %.1f %%)"
-                % (dom["F"], dom["dtype"], dom["msg"], 100 * (dom["fwd_ms"] + dom["bwd_ms"]) / tot_ms),
+    nslab = max(1, dom["F"] * sdom // 512)
+    roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel, forward call of F=%d %s %s = %d column-slab launch(es) + fix-up (largest share of the step: %.1f %%); bytes, time and traffic are per call"
+                % (dom["F"], dom["dtype"], dom["msg"], nslab, 100 * (dom["fwd_ms"] + dom["bwd_ms"]) / tot_ms),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if traffic is None else traffic * 1e9,
-                "peak_source": peak_src, "bytes_model": "compulsory bytes per launch: 4E(+4E weights)+8N+2*N*F*s = %d" % comp,
-                "ms_per_launch": dom["fwd_ms"],
+                "peak_source": peak_src, "bytes_model": "compulsory bytes per call: 4E(+4E weights)+8N+2*N*F*s = %d" % comp,
+                "ms_per_call": dom["fwd_ms"], "launches_per_call": 2 * nslab,
                 "dram_traffic_GBs": None if traffic is None else traffic * 1e3 / dom["fwd_ms"],
                 "dram_traffic_frac_of_peak": None if traffic is None else traffic * 1e3 / dom["fwd_ms"] / peak,
                 "gather_upper_bound_GBs": gather_bytes(N, E, dom["F"], sdom, wdom) / dom["fwd_ms"] / 1e6,
