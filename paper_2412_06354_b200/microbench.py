@@ -91,6 +91,10 @@ def bench_propagate(plain):
         row(tag + "copy_xj+mean", device_time_us(lambda: gnn.propagate_fused(g, X, None, "mean"), plain))
         out, arg = gnn.propagate_fused(g, X, None, "max")
         row(tag + "copy_xj+max (+argmax)", device_time_us(lambda: gnn.propagate_fused(g, X, None, "max", out=out, argmax=arg), plain))
+        m = gnn.apply_edges(g, gnn.COPY_XJ, X)  # the E x F message tensor that the fused call never forms
+        row(tag + "UNFUSED apply_edges(copy_xj) + aggregate(mean)",
+            device_time_us(lambda: gnn.aggregate(g, gnn.apply_edges(g, gnn.COPY_XJ, X), "mean"), plain))
+        del m
         row(tag + "backward of mean", device_time_us(lambda: gnn.propagate_fused_backward(g, dO, "mean"), plain))
         row(tag + "backward of max", device_time_us(lambda: gnn.propagate_fused_backward(g, dO, "max", argmax=arg), plain))
 
