@@ -424,7 +424,6 @@ def run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, de
     s_bwd.wait_stream(s_fwd)
     step()
     join()
-    step()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t0.record(s_fwd)
