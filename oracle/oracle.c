@@ -27,7 +27,7 @@
  * list and keeps only its own rows, so the per-row accumulation order is the edge order
  * whatever the thread count.
  *
- * Parity pins: every function below is pinned by tests/test_oracle_*.py (closed forms on
+ * Parity pins: every function below is pinned by tests/test_oracle_pins.py (closed forms on
  * star/path graphs, dense A^T X brute force, invariants, fp64 finite differences).
  */
 #include <math.h>
@@ -164,8 +164,7 @@ void oracle_apply_edges(int msg, int64_t E, const int32_t* src, const int32_t* d
  *              among equal values (strict comparison while scanning in edge order, so +0 and
  *              -0 tie); empty -> value 0, arg -1.
  * S (optional) = sum over the same edges of |m| (divided like the mean). m is fp64 [E,F] in
- * the original edge order; rows given by `rows` only if rows != NULL (nrows of them; out/S/arg
- * are then [nrows,F]). */
+ * the original edge order. */
 void oracle_aggregate(int op, int32_t N, int64_t E, const int32_t* dst, const double* m, int F,
                       double* out, double* S, int64_t* arg) {
     int T = g_threads;
@@ -210,7 +209,11 @@ void oracle_aggregate(int op, int32_t N, int64_t E, const int32_t* dst, const do
 /* propagate(message, g, op) written directly (no E x F tensor): message COPY_XJ (w == NULL)
  * or E_MUL_XJ with one scalar w[k] per edge.  By definition equal to
  * aggregate(op, apply_edges(message)).  If slot != NULL only the rows i with slot[i] >= 0 are
- * computed, into row slot[i] of out/S/arg (sampled checking of large graphs); else slot[i] = i. */
+ * computed, into row slot[i] of out/S/arg (sampled checking of large graphs); else slot[i] = i.
+ * Reading for max/min over weighted messages of stored (fp32 / bf16) features: the winner is an
+ * integer decided by floating point, so the comparison is made on the message as a device holds
+ * it, w[k]*x rounded once to fp32 (the fp64 product of two fp32 values is exact, so the cast
+ * below is that single rounding); fp64 features are compared unrounded. */
 void oracle_propagate(int op, int32_t N, int64_t E, const int32_t* src, const int32_t* dst,
                       const void* X, int dt, const float* w, int F, const int32_t* slot,
                       int32_t nslots, double* out, double* S, int64_t* arg) {
@@ -234,8 +237,10 @@ void oracle_propagate(int op, int32_t N, int64_t E, const int32_t* src, const in
             int64_t j = src[k];
             double wk = w ? (double)w[k] : 1.0;
             int first = (cnt[r]++ == 0);
+            int as_f32 = (op == OP_MAX || op == OP_MIN) && w && dt != DT_F64;
             for (int f = 0; f < F; ++f) {
                 double v = wk * ld(X, dt, j * F + f);
+                if (as_f32) v = (double)(float)v;
                 int64_t o = r * F + f;
                 if (op == OP_SUM || op == OP_MEAN) {
                     out[o] += v;

@@ -272,6 +272,72 @@ def test_propagate_row_subset_matches_full():
             assert np.array_equal(a[rows], b)
 
 
+def test_propagate_backward_source_row_subset_matches_full():
+    """The rows= path of the backward (a slot per SOURCE row) against the full result, which the finite
+    differences below pin; rows unsorted, first and last row included, directed graph so that a slot
+    looked up through the wrong endpoint lands in another row."""
+    n, e, F = 50, 700, 6
+    src, dst = rand_graph(n, e)
+    X = synth.normal_f32((n, F), 5)
+    R = synth.normal_f32((n, F), 6)
+    w = RNG.random(e).astype(np.float32)
+    rows = np.array([49, 0, 31, 7, 23])
+    outdeg = np.bincount(src, minlength=n)
+    assert (outdeg[rows] > 0).all() and len(set(src[:20]) - set(dst[:20])) > 0
+    for op in ("sum", "mean", "max", "min"):
+        arg = oracle.propagate(op, n, src, dst, X, w)[2] if op in ("max", "min") else None
+        full = oracle.propagate_backward(op, n, src, dst, X, w, R, arg=arg)
+        part = oracle.propagate_backward(op, n, src, dst, X, w, R, arg=arg, rows=rows)
+        assert part["dX"].shape == (len(rows), F)
+        assert np.array_equal(full["dX"][rows], part["dX"]) and np.array_equal(full["SdX"][rows], part["SdX"])
+        assert np.abs(part["dX"]).sum() > 0
+    # and against the definition written out for the subset: dX[j] = sum over edges out of j
+    part = oracle.propagate_backward("mean", n, src, dst, X, w, R, rows=rows)
+    indeg = np.bincount(dst, minlength=n)
+    for t, j in enumerate(rows):
+        ref = np.zeros(F)
+        for k in np.nonzero(src == j)[0]:
+            ref += float(w[k]) / indeg[dst[k]] * R[dst[k]].astype(np.float64)
+        assert np.allclose(part["dX"][t], ref, rtol=1e-13, atol=1e-15)
+
+
+def test_weighted_max_compares_messages_rounded_to_f32():
+    """Stored (fp32) features: the winner is decided on w*x rounded once to fp32, the precision a
+    device compares in; two exact products that differ below fp32 resolution tie and the first
+    edge wins.  fp64 features are compared exactly."""
+    u = 2.0 ** -23
+    X32 = np.array([[1.0 + 2 * u], [1.0 + u], [0.0]], np.float32)   # nodes 0, 1 feed node 2
+    w = np.array([1.0, 1.0 + u], np.float32)
+    src, dst = np.array([0, 1], np.int32), np.array([2, 2], np.int32)
+    p0, p1 = float(w[0]) * float(X32[0, 0]), float(w[1]) * float(X32[1, 0])
+    assert p1 > p0 and np.float32(p1) == np.float32(p0)
+    v, _, a = oracle.propagate("max", 3, src, dst, X32, w)
+    assert a[2, 0] == 0 and v[2, 0] == float(np.float32(p0))
+    v, _, a = oracle.propagate("max", 3, src, dst, X32.astype(np.float64), w)
+    assert a[2, 0] == 1 and v[2, 0] == p1
+    v, _, a = oracle.propagate("min", 3, src[::-1].copy(), dst, X32, w[::-1].copy())
+    assert a[2, 0] == 0   # the same tie under min, other edge first
+
+
+@pytest.mark.parametrize("op", ["max", "min"])
+def test_weighted_max_backward_finite_differences(op):
+    n, e, F = 20, 150, 4
+    src, dst = rand_graph(n, e)
+    X = RNG.standard_normal((n, F))
+    w = (RNG.random(e) + 0.5).astype(np.float32) * np.where(RNG.random(e) < 0.3, -1, 1).astype(np.float32)
+    R = RNG.standard_normal((n, F))
+    arg = oracle.propagate(op, n, src, dst, X, w)[2]
+    bw = oracle.propagate_backward(op, n, src, dst, X, w, R, arg=arg)
+    loss = lambda: (oracle.propagate(op, n, src, dst, X, w)[0] * R).sum()
+    ids = RNG.choice(X.size, 60, replace=False)
+    assert np.allclose(fd(loss, X, ids, h=1e-7), bw["dX"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    # fused == apply_edges + aggregate for the weighted message
+    m = oracle.apply_edges(oracle.E_MUL_XJ, src, dst, X, e=w)
+    v2, _, a2 = oracle.aggregate(op, n, dst, m)
+    v1, _, a1 = oracle.propagate(op, n, src, dst, X, w)
+    assert np.array_equal(v1, v2) and np.array_equal(a1, a2)
+
+
 def test_thread_count_does_not_change_results():
     n, e, F = 64, 2000, 8
     src, dst = rand_graph(n, e)
