@@ -35,9 +35,13 @@ ALL_CASES = [(F, dt) for dt in ("bf16", "f32") for F in (32, 64, 128, 256, 512)]
 FMAX = 512
 
 # DRAM bytes (read + write, GB) of one gnn_propagate_fused / _backward call (all its propagate_chunk_kernel
-# launches: wide rows run as 512-byte column slabs) at full size, from the single-pass ncu
-# capture summarised in profiles/propagate_sweep_full_size_dram_bytes.md.  Valid for the kernel as committed
-# with that capture; set an entry to None when the kernel changes.
+# launches: wide rows run as 512-byte column slabs) at full size, taken once with the hardware counters
+# dram__bytes_read.sum + dram__bytes_write.sum.  The numbers belong to the kernel sources whose digest is
+# TRAFFIC_KERNEL_SHA256; with any other sources the line reports traffic = null.
+TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none (single pass) over one step of this "
+                  "sweep at full size, row-walking and fix-up kernels as of commit 8f9365f (unchanged up to the digest below); per-call sums in the summary of the full-size DRAM-byte capture under profiles/")
+TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
+TRAFFIC_KERNEL_SHA256 = "c23bd6af0c3f8a9b1bc495d55dedf585f3abe630dbae8a92d4ff992552f83415"
 TRAFFIC_GB = {
     "32:bf16:copy_xj:fwd": 1.48,
     "32:bf16:copy_xj:bwd": 1.48,
@@ -90,6 +94,16 @@ def parse_cases(s):
         f, dt = tok.split(":")
         out.append((int(f), dt))
     return out
+
+
+def kernel_sources_digest():
+    """sha256 over the sources of the propagate kernels, in the order of TRAFFIC_KERNEL_FILES."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_KERNEL_FILES:
+        with open(os.path.join(ROOT, "paper_2412_06354_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 
 
 def measured_peak():
@@ -169,7 +183,9 @@ def run_reference(args, rank):
     val = sample["E"] * sample["F"] / (ms * 1e-3)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD_NAME},
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "bounded sample for the CPU checker: " + sample["desc"], "N": sample["N"], "E": sample["E"], "cases": ["%d:bf16" % sample["F"]],
+                       "sample_of": WORKLOAD_NAME},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample["desc"]},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -178,12 +194,12 @@ def run_reference(args, rank):
 WORKLOAD_NAME = "large sparse aggregation sweep: R-MAT N=2.4M E=123M (a=.57 b=.19 c=.19, symmetrised, relabelled, sorted by dst), F in {32,64,128,256,512} x {bf16,f32}, copy_xj+sum and e_mul_xj+sum, fwd + bwd dX"
 
 
-def cpu_sample(synth, pairs=16_000_000, F=128):
+def cpu_sample(synth, pairs=16_000_000, F=128, scale=20):
     """A smaller graph of the same family for the CPU checker: R-MAT with the same parameters and
     the same mean degree (N=624,390, 32,000,000 directed edges), bf16 features of width 128: a few
     seconds of work per forward + backward pair on 16 cores."""
     n = 2_400_000 * (2 * pairs) // 123_000_000
-    src, dst = synth.rmat(20, n, pairs, synth.BASE_SEED + 5, symmetric=True, relabel=True, sort_by_dst=True)
+    src, dst = synth.rmat(scale, n, pairs, synth.BASE_SEED + 5, symmetric=True, relabel=True, sort_by_dst=True)
     return dict(N=n, E=len(src), F=F, src=src, dst=dst, X=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 20),
                 R=synth.normal_bf16((n, F), synth.BASE_SEED + 5, 21), w=synth.uniform_f32((len(src),), 0, 1, synth.BASE_SEED + 5, 13),
                 desc=f"same generator at N={n}, E={2 * pairs} (same mean degree), F={F} bf16, e_mul_xj+sum fwd + bwd dX, fp64")
@@ -212,6 +228,38 @@ def whole_job_value(work_per_rank, ms_per_step_max, world):
     return world * work_per_rank / (ms_per_step_max * 1e-3)
 
 
+# ----------------------------------------------------------------------------- smaller workloads
+SMALL_WORKLOADS = {
+    1: "GCN layer: Erdos-Renyi N=2000, 10000 directed edges + self-loops, F=64 f32, normalised sum",
+    2: "batched small graphs: 512 graphs of 10-40 nodes, F=128 f32, mean aggregation + per-graph mean pooling",
+    3: "power-law graph: preferential attachment N=170000, m=4, F=128 f32 and bf16, mean / max / normalised sum",
+    4: "attention: R-MAT N=100000, 1.6M directed edges, 8 heads x 32 features bf16, fused GAT core",
+}
+
+
+def run_small_config(args, rank, local):
+    """Layer-level calls of one of the smaller workloads: per call the warm device time (20 calls replayed as one
+    CUDA graph) and the time after an L2 flush (256 MB written before every call, CUDA events, median of 20)."""
+    if rank != 0:
+        return
+    import torch
+    import microbench
+    from paper_2412_06354_b200 import build, gnn
+    build.build()
+    gnn.load()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    microbench.measure.to_stderr = True
+    sampler = ClockSampler(local)
+    sampler.start()
+    rows = microbench.measure(microbench.TABLE["config%d" % args.config](), flush=True)
+    clocks = sampler.stop()
+    line = {"metric": "device time per call", "unit": "us", "value": sum(r["us_warm"] for r in rows), "n_gpus": 1, "higher_is_better": False,
+            "data": "synthetic", "config": {"workload": SMALL_WORKLOADS[args.config], "l2": "us_warm: inputs resident in L2 (graph replay); us_flushed: 256 MB written before every call"},
+            "value_note": "sum of the warm per-call times", "clocks": clocks, "calls": rows}
+    print(json.dumps(line), flush=True)
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -222,6 +270,9 @@ def main():
     ap.add_argument("--cases", default="sweep")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-dw", action="store_true", help="skip the separate timing of the edge-weight gradient")
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5],
+                    help="5 (default): the large sweep.  1-4: device times of the layer-level calls of the smaller workloads, warm and after an L2 flush")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--natural-ids", action="store_true",
                     help="keep the generator's vertex ids (hubs at low ids) instead of the random relabelling of the headline workload")
@@ -233,6 +284,8 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         return run_reference(args, rank)
+    if args.config != 5:
+        return run_small_config(args, rank, local)
     assert args.warmup >= 3 or os.environ.get("GNN_BENCH_ALLOW_SHORT"), "use at least 3 warm-up steps"
 
     import torch
@@ -320,6 +373,25 @@ def main():
     work = sum(E * F for F, _, _, _ in plan)  # edges*features per step (each fwd+bwd pair counted once)
     value = whole_job_value(work, ms_per_step, world)
 
+    # ---- edge-weight gradient of the e_mul_xj cases (one dot product per edge), timed after the step and
+    # reported per case beside the dX time; it is not part of `value`
+    dw_ms = {}
+    if not args.no_dw:
+        dWbuf = torch.empty(E, dtype=torch.float32, device=dev)
+        for F, dt, weighted, (X, R, out, dX) in plan:
+            if not weighted:
+                continue
+            for _ in range(2):
+                gnn.propagate_fused_backward(g, R, "sum", X=X, want_dX=False, want_dW=True, dW=dWbuf, ws=ws)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(3):
+                gnn.propagate_fused_backward(g, R, "sum", X=X, want_dX=False, want_dW=True, dW=dWbuf, ws=ws)
+            b.record(stream)
+            torch.cuda.synchronize()
+            dw_ms[(F, dt)] = a.elapsed_time(b) / 3
+        del dWbuf
+
     # ---- per-case breakdown and the roofline of the chunked propagate kernel
     peak, peak_src = measured_peak()
     per_case, tot_ms, tot_comp, tot_gath = [], 0.0, 0.0, 0.0
@@ -333,29 +405,35 @@ def main():
         tot_gath += 2 * gath
         per_case.append({"F": F, "dtype": dt, "msg": "e_mul_xj" if weighted else "copy_xj", "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
                          "edges_feat_per_s": E * F / ((f_ms + b_ms) * 1e-3), "compulsory_GBs_fwd": comp / f_ms / 1e6,
-                         "gather_GBs_fwd": gath / f_ms / 1e6, "compulsory_frac_fwd": comp / f_ms / 1e6 / peak})
+                         "l2_side_model_GBs_fwd": gath / f_ms / 1e6, "compulsory_frac_fwd": comp / f_ms / 1e6 / peak})
+        if weighted and (F, dt) in dw_ms:
+            per_case[-1]["bwd_dW_ms"] = round(dw_ms[(F, dt)], 4)
     # dominant kernel instance = the case with the largest share of the step
     dom = max(per_case, key=lambda c: c["fwd_ms"] + c["bwd_ms"])
     sdom = 2 if dom["dtype"] == "bf16" else 4
     wdom = dom["msg"] == "e_mul_xj"
     comp = compulsory_bytes(N, E, dom["F"], sdom, wdom)
     tkey = "%d:%s:%s:fwd" % (dom["F"], dom["dtype"], dom["msg"])
-    traffic = TRAFFIC_GB.get(tkey) if shrink == 0 and not args.natural_ids else None
+    traffic_valid = shrink == 0 and not args.natural_ids and kernel_sources_digest() == TRAFFIC_KERNEL_SHA256
+    traffic = TRAFFIC_GB.get(tkey) if traffic_valid else None
     achieved = comp / dom["fwd_ms"] / 1e6
     nslab = max(1, dom["F"] * sdom // 512)
     roofline = {"bound": "hbm", "kernel": "propagate_chunk_kernel, forward call of F=%d %s %s = %d column-slab launch(es) + fix-up (largest share of the step: %.1f %%); bytes, time and traffic are per call"
                 % (dom["F"], dom["dtype"], dom["msg"], nslab, 100 * (dom["fwd_ms"] + dom["bwd_ms"]) / tot_ms),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if traffic is None else traffic * 1e9,
+                "traffic_source": (TRAFFIC_SOURCE + "; kernel sources sha256 " + TRAFFIC_KERNEL_SHA256[:16]) if traffic is not None else
+                                  "null: the kernel sources differ from the ones the counters were taken with, or this is not the full-size relabelled workload",
                 "peak_source": peak_src, "bytes_model": "compulsory bytes per call: 4E(+4E weights)+8N+2*N*F*s = %d" % comp,
                 "ms_per_call": dom["fwd_ms"], "launches_per_call": 2 * nslab,
                 "dram_traffic_GBs": None if traffic is None else traffic * 1e3 / dom["fwd_ms"],
                 "dram_traffic_frac_of_peak": None if traffic is None else traffic * 1e3 / dom["fwd_ms"] / peak,
-                "gather_upper_bound_GBs": gather_bytes(N, E, dom["F"], sdom, wdom) / dom["fwd_ms"] / 1e6,
+                "l2_side_model_GBs": gather_bytes(N, E, dom["F"], sdom, wdom) / dom["fwd_ms"] / 1e6,
+                "l2_side_model_note": "bytes if every edge fetched its row with no reuse, over time: a rate on the L2 -> SM side (it can exceed any HBM peak), not DRAM bandwidth",
                 "all_launches": {"compulsory_GBs": tot_comp / tot_ms / 1e6, "frac": tot_comp / tot_ms / 1e6 / peak,
-                                 "gather_upper_bound_GBs": tot_gath / tot_ms / 1e6,
+                                 "l2_side_model_GBs": tot_gath / tot_ms / 1e6,
                                  "dram_traffic_GBs": (sum(TRAFFIC_GB["%d:%s:%s:%s" % (c["F"], c["dtype"], c["msg"], d)] for c in per_case for d in ("fwd", "bwd")) * 1e3 / tot_ms
-                                                      if shrink == 0 and not args.natural_ids and all(TRAFFIC_GB.get("%d:%s:%s:fwd" % (c["F"], c["dtype"], c["msg"])) for c in per_case) else None)}}
+                                                      if traffic_valid and all(TRAFFIC_GB.get("%d:%s:%s:fwd" % (c["F"], c["dtype"], c["msg"])) for c in per_case) else None)}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -376,6 +454,11 @@ def main():
         cpu_step(oracle, sample)
         t = min(cpu_step(oracle, sample) for _ in range(2))
         line["cpu_baseline"] = {"value": sample["E"] * sample["F"] / t, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample["desc"]}
+        del sample
+        oracle.set_threads(1)  # the same checker on one thread, on a sample an eighth of the size
+        small = cpu_sample(synth, pairs=2_000_000, scale=17)
+        t1 = min(cpu_step(oracle, small) for _ in range(2))
+        line["cpu_baseline"].update({"value_1thread": small["E"] * small["F"] / t1, "sample_1thread": small["desc"]})
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -237,8 +237,10 @@ gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, con
  *   s[p,h]  = LeakyReLU_slope(al[col[p],h] + ar[i,h]),  alpha = edge softmax of s per row and head
  *   out[i,h,:] = sum over p in row i of alpha[p,h] * Wx[col[p],h,:]      (heads concatenated)
  * No self-loops are added; a node without incoming edges gets 0.  Saved for the backward call:
- * alpha_csr float [E,H] (CSR order), al, ar float [N,H].  H must be a power of two <= 32 and
- * C*sizeof(element) a multiple of 16 bytes.  The E x F message tensor is never formed.
+ * alpha_csr float [E,H] (CSR order), al, ar float [N,H].  H must be a power of two <= 32 and a
+ * head must span a power-of-two number (1..32) of 16-byte chunks (C = 4, 8, 16, ... for float,
+ * 8, 16, 32, ... for bf16); other shapes return GNN_ERR_UNSUPPORTED from the forward and the
+ * backward call alike.  The E x F message tensor is never formed.
  * ws: gnn_gat_fused_workspace(N, E, H, C, backward) bytes. */
 size_t gnn_gat_fused_workspace(int32_t N, int64_t E, int H, int C, int backward);
 gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, const float* a_dst,

@@ -224,6 +224,10 @@ static gnn_status gat_check(const char* who, const gnn_csr* g, int H, int C, gnn
     const int epc = 16 / elem_size(dtype);
     GNN_REQUIRE(C >= epc && C % epc == 0, GNN_ERR_UNSUPPORTED,
                 "%s: features per head must be a multiple of %d (C=%d)", who, epc, C);
+    // the per-head dot products of the backward pass reduce over a power-of-two number of lanes: the forward
+    // call refuses the same shapes, so that a layer never runs forward and then fails backward
+    GNN_REQUIRE(pow2_le32(C / epc), GNN_ERR_UNSUPPORTED,
+                "%s: a head must span a power-of-two number (<= 32) of 16-byte chunks (C=%d)", who, C);
     return GNN_OK;
 }
 

@@ -37,23 +37,31 @@ def run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, what):
     R = synth.normal((n, F), dtype, 4242, 3)
     bw = gnn.gat_fused_backward(g, to_dev(Wx), to_dev(a_s), to_dev(a_d), fwd, to_dev(R), H)
     rb = oracle.gat_backward(n, src, dst, Wx, a_s, a_d, H, C, ref, R)
-    # LeakyReLU'(z) is decided by the sign of z; where |z| is below fp32 resolution of its terms the
-    # two precisions may decide differently, so nodes touching such an edge are left out
+    # LeakyReLU'(z) is decided by the sign of z.  Where |z| is below the fp32 resolution of its terms the
+    # two precisions may decide differently: such an edge moves dz[k,h] by at most |ds[k,h]|*(1-slope), which
+    # reaches dal[src], dar[dst] and, through them, three outputs.  The allowance is accumulated from the
+    # checker's own intermediates and added to the bound of exactly the elements it can reach.
+    slope = 0.2
     z = ref["al"][src] + ref["ar"][dst]
     risky = np.abs(z) < 2e-6 * (Sal[src] + Sar[dst])
-    skip = np.zeros(n, bool)
-    skip[src[risky.any(axis=1)]] = True
-    skip[dst[risky.any(axis=1)]] = True
-    assert skip.mean() < 0.05
-    keep = ~skip
-    assert_close(to_host64(bw["dWx"])[keep], rb["dWx"][keep], rb["SdWx"][keep], dtype, what + " dWx")
-    if not skip.any():
-        assert_close(to_host64(bw["da_src"]), rb["da_src"], rb["Sda_src"], "f32", what + " da_src")
-        assert_close(to_host64(bw["da_dst"]), rb["da_dst"], rb["Sda_dst"], "f32", what + " da_dst")
-    else:  # the attention-vector gradients sum over every node: compare norm-wise only
-        for k in ("da_src", "da_dst"):
-            err = np.abs(to_host64(bw[k]) - rb[k]).max() / np.abs(rb[k]).max()
-            assert err < 1e-3, (k, err)
+    assert risky.mean() < 0.01, risky.mean()
+    r64 = synth.to_f64(R).reshape(n, H, C)
+    dalpha = np.empty((len(src), H))
+    for h in range(H):
+        dalpha[:, h] = (r64[dst, h, :] * x64[src, h, :]).sum(axis=1)
+    ds, _ = oracle.edge_softmax_backward(n, dst, ref["alpha"], dalpha) if len(src) else (np.zeros((0, H)), None)
+    slack = np.where(risky, np.abs(ds) * (1.0 - slope), 0.0)
+    sl_al, sl_ar = np.zeros((n, H)), np.zeros((n, H))
+    for h in range(H):
+        sl_al[:, h] = np.bincount(src, weights=slack[:, h], minlength=n)
+        sl_ar[:, h] = np.bincount(dst, weights=slack[:, h], minlength=n)
+    as64, ad64 = np.abs(a_s.astype(np.float64)), np.abs(a_d.astype(np.float64))
+    extra_dWx = (sl_al[:, :, None] * as64[None] + sl_ar[:, :, None] * ad64[None]).reshape(n, F)
+    extra_src = np.einsum("nh,nhc->hc", sl_al, np.abs(x64))
+    extra_dst = np.einsum("nh,nhc->hc", sl_ar, np.abs(x64))
+    assert_close(to_host64(bw["dWx"]), rb["dWx"], rb["SdWx"], dtype, what + " dWx", extra=extra_dWx)
+    assert_close(to_host64(bw["da_src"]), rb["da_src"], rb["Sda_src"], "f32", what + " da_src", extra=extra_src)
+    assert_close(to_host64(bw["da_dst"]), rb["da_dst"], rb["Sda_dst"], "f32", what + " da_dst", extra=extra_dst)
     return g, fwd
 
 
@@ -91,6 +99,12 @@ def test_gat_degenerate(gnn):
     assert torch.count_nonzero(bw["dWx"]) == 0 and torch.count_nonzero(bw["da_src"]) == 0
     with pytest.raises(gnn.GnnError) as e:  # three heads
         gnn.gat_fused(g, to_dev(synth.normal_f32((4, 24), 3)), a_s, a_s, 3)
+    assert e.value.status == 5
+    # a head of 24 bf16 values (three 16-byte chunks) is refused by the forward and the backward call alike
+    Wx3 = to_dev(synth.normal_bf16((4, 48), 4))
+    a3 = to_dev(synth.normal_f32((2, 24), 5))
+    with pytest.raises(gnn.GnnError) as e:
+        gnn.gat_fused(g, Wx3, a3, a3, 2)
     assert e.value.status == 5
 
 

@@ -44,8 +44,10 @@ def test_csr_bit_exact_full_size(big):
     assert np.array_equal(g.t2f.cpu().numpy(), oracle.t2f(eid, eidT))
 
 
-@pytest.mark.parametrize("dtype,F", [("bf16", 128), ("f32", 32), ("f32", 512)])
+@pytest.mark.parametrize("dtype,F", [("bf16", 128), ("f32", 32), ("f32", 512), ("bf16", 512), ("f32", 256), ("bf16", 64), ("bf16", 256)])
 def test_propagate_sampled_rows_full_size(big, dtype, F):
+    """Every launch shape the benchmark times at this size: narrow and 512-byte rows on the row-walking kernel,
+    and the column-slab passes (two for 1024-byte rows: bf16 F=512, f32 F=256; four for f32 F=512)."""
     import torch
     gnn, wl, g = big
     n, src, dst, w, seed = wl["N"], wl["src"], wl["dst"], wl["w"], wl["seed"]

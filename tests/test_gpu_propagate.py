@@ -158,6 +158,28 @@ def test_propagate_max_min_bit_exact(gnn, dtype, F, op):
     assert np.array_equal(eid_of, a), "winner differs"
 
 
+@pytest.mark.parametrize("dtype,F", [("f32", 64), ("f32", 512), ("bf16", 32), ("bf16", 128), ("bf16", 1024)])
+@pytest.mark.parametrize("op", ["max", "min"])
+def test_propagate_weighted_max_min(gnn, dtype, F, op):
+    """e_mul_xj with max/min: the message w*x is rounded once to fp32 and compared in fp32 (the checker does
+    the same), so values and winners are bit-exact; signed weights, both kernels (rows up to 512 bytes take the
+    position-first kernel here, wider rows the row-walking one); then the routing backward with the weights."""
+    n, src, dst = ragged_graph(50 + F)
+    g = build_graph(gnn, n, src, dst)
+    ref = host_csr(n, src, dst)
+    X = feats((n, F), dtype, 500 + F)
+    R = feats((n, F), dtype, 501 + F, stream=1)
+    w = synth.uniform_f32((len(src),), -1.0, 1.0, 12)
+    out, arg = gnn.propagate_fused(g, to_dev(X), to_dev(w[ref["eid"]]), op)
+    o, _, a = oracle.propagate(op, n, src, dst, X, w)
+    assert np.array_equal(bits(out), f64_to_dtype_bits(o, dtype)), "values differ"
+    got_arg = arg.cpu().numpy()
+    assert np.array_equal(np.where(got_arg >= 0, ref["eid"][np.maximum(got_arg, 0)], -1), a), "winner differs"
+    dX, _ = gnn.propagate_fused_backward(g, to_dev(R), op, w_csrT=to_dev(w[ref["eidT"]]), argmax=arg)
+    bw = oracle.propagate_backward(op, n, src, dst, X, w, R, arg=a)
+    assert_close(to_host64(dX), bw["dX"], bw["SdX"], dtype, f"weighted dX {op}")
+
+
 # ---------------------------------------------------------------- backward
 @pytest.mark.parametrize("dtype,F", [("f32", 16), ("f32", 64), ("f32", 128), ("f32", 512), ("bf16", 32), ("bf16", 64), ("bf16", 128), ("bf16", 512)])
 @pytest.mark.parametrize("op", ["sum", "mean"])

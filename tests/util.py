@@ -51,9 +51,11 @@ def f64_to_dtype_bits(x64, dtype):
     return t.to(torch.float32).view(torch.int32).numpy()
 
 
-def assert_close(got, ref, S, dtype, what=""):
+def assert_close(got, ref, S, dtype, what="", extra=None):
     """Element-wise: f32 |got-ref| <= 1e-5*S ; bf16 |got-ref| <= 2e-2*|ref| + 1e-5*S, where S is the
-    sum of |terms| of the element (S >= |ref|).  Plus the norm-wise bound on the whole tensor."""
+    sum of |terms| of the element (S >= |ref|).  Plus the norm-wise bound on the whole tensor.
+    extra (optional, same shape): an absolute allowance per element that the caller derives for
+    elements reached by a floating-point branch decision (zero elsewhere); it widens both bounds."""
     got = np.asarray(got, np.float64)
     ref = np.asarray(ref, np.float64)
     S = np.asarray(S, np.float64)
@@ -61,6 +63,10 @@ def assert_close(got, ref, S, dtype, what=""):
     assert np.isfinite(got).all(), f"{what}: non-finite output"
     err = np.abs(got - ref)
     bound = 1e-5 * S if dtype == "f32" else 2e-2 * np.abs(ref) + 1e-5 * S
+    if extra is not None:
+        extra = np.asarray(extra, np.float64)
+        assert extra.shape == ref.shape and (extra >= 0).all()
+        bound = bound + extra
     bad = err > bound
     if bad.any():
         i = np.unravel_index(np.argmax(err - bound), err.shape)
@@ -68,4 +74,5 @@ def assert_close(got, ref, S, dtype, what=""):
                              f"got {got[i]!r} ref {ref[i]!r} S {S[i]!r} err {err[i]:.3e} bound {bound[i]:.3e}")
     den = np.abs(ref).max() if ref.size else 0.0
     if den > 0:
-        assert err.max() / den <= TOL[dtype], f"{what}: norm-wise error {err.max() / den:.3e}"
+        nerr = err if extra is None else np.maximum(err - extra, 0.0)
+        assert nerr.max() / den <= TOL[dtype], f"{what}: norm-wise error {nerr.max() / den:.3e}"
