@@ -21,7 +21,7 @@ _LIB_PATH = os.path.join(_HERE, "liboracle.so")
 _lib = None
 
 SUM, MEAN, MAX, MIN = 0, 1, 2, 3
-COPY_XJ, E_MUL_XJ, GAT_LOGIT = 0, 1, 2
+COPY_XJ, E_MUL_XJ, GAT_LOGIT, XI_SUB_XJ, XI_DOT_XJ = 0, 1, 2, 3, 4
 OPS = {"sum": SUM, "mean": MEAN, "max": MAX, "min": MIN}
 
 
@@ -129,7 +129,9 @@ def gather(idx, X):
     return out
 
 
-def apply_edges(msg, src, dst, X, Y=None, e=None, slope=0.2):
+def apply_edges(msg, src, dst, X, Y=None, e=None, slope=0.2, H=1):
+    """Per-edge messages, original edge order.  X: source-side node array (x_j; al for GAT_LOGIT); Y: target-side
+    node array (x_i for XI_SUB_XJ / XI_DOT_XJ, ar for GAT_LOGIT).  XI_DOT_XJ returns [E,H] (one dot product per head)."""
     src, dst, X = _i32(src), _i32(dst), _c(X)
     E, F = src.shape[0], X.shape[1]
     Y = None if Y is None else _c(Y)
@@ -139,12 +141,40 @@ def apply_edges(msg, src, dst, X, Y=None, e=None, slope=0.2):
         if e.ndim == 1:
             e = e.reshape(-1, 1)
         ew = e.shape[1]
-    m = np.empty((E, F), np.float64)
+    if msg == XI_DOT_XJ:
+        ew = H
+    m = np.empty((E, H if msg == XI_DOT_XJ else F), np.float64)
     _L().oracle_apply_edges(C.c_int(msg), C.c_int64(E), _ptr(src), _ptr(dst), _ptr(X), C.c_int(_dt(X)),
                             _ptr(Y), C.c_int(_dt(Y) if Y is not None else 0),
                             _ptr(e), C.c_int(_dt(e) if e is not None else 0), C.c_int(ew), C.c_int(F),
                             C.c_double(slope), _ptr(m))
     return m
+
+
+def apply_edges_backward(msg, N, src, dst, X, dm, Y=None, e=None, H=1, want=("dXj",)):
+    """Backward of apply_edges for dL/dm = dm -> dict with the wanted ones of dXj, dXi [N,F], de [E,ew]
+    and their magnitude sums SXj, SXi, Se."""
+    src, dst, X = _i32(src), _i32(dst), _c(X)
+    E, F = src.shape[0], X.shape[1]
+    Y = None if Y is None else _c(Y)
+    dm = _c(dm, np.float64)
+    ew = 0
+    if e is not None:
+        e = _c(e)
+        if e.ndim == 1:
+            e = e.reshape(-1, 1)
+        ew = e.shape[1]
+    if msg == XI_DOT_XJ:
+        ew = H
+    o = {}
+    for k, shape in (("dXj", (N, F)), ("dXi", (N, F)), ("de", (E, max(ew, 1)))):
+        o[k] = np.empty(shape, np.float64) if k in want else None
+        o["S" + k[1:]] = np.empty(shape, np.float64) if k in want else None
+    _L().oracle_apply_edges_backward(C.c_int(msg), C.c_int32(N), C.c_int64(E), _ptr(src), _ptr(dst), _ptr(X), C.c_int(_dt(X)),
+                                     _ptr(Y), C.c_int(_dt(Y) if Y is not None else 0), _ptr(e), C.c_int(_dt(e) if e is not None else 0),
+                                     C.c_int(ew), C.c_int(F), _ptr(dm), _ptr(o["dXj"]), _ptr(o["SXj"]), _ptr(o["dXi"]), _ptr(o["SXi"]),
+                                     _ptr(o["de"]), _ptr(o["Se"]))
+    return o
 
 
 def aggregate(op, N, dst, m):
@@ -305,3 +335,68 @@ def matmul(A, B, ta=False, tb=False):
     _L().oracle_matmul(_ptr(A), C.c_int(_dt(A)), C.c_int(int(ta)), _ptr(B), C.c_int(_dt(B)), C.c_int(int(tb)),
                        C.c_int64(n), C.c_int64(k), C.c_int64(m), _ptr(Y), _ptr(S))
     return Y, S
+
+
+# ------------------------------------------------------------------ compositions of the primitives above
+# (Sec. 3 "Message Passing": propagate = apply_edges followed by aggregate_neighbors; Sec. 3 "Graph
+# Convolutional Layers" names GINConv; Sec. 3 "Graph Data Structures" names heterogeneous and temporal graphs.)
+def propagate_msg(msg, op, N, src, dst, Xj, Xi=None, e=None, H=1):
+    """aggregate(op, apply_edges(msg)) for any message -> (out, S, arg)."""
+    return aggregate(op, N, dst, apply_edges(msg, src, dst, Xj, Y=Xi, e=e, H=H))
+
+
+def propagate_msg_backward(msg, op, N, src, dst, Xj, R, Xi=None, e=None, H=1, arg=None, want=("dXj",)):
+    """Backward of propagate_msg for dL/dout = R: aggregate_backward, then apply_edges_backward."""
+    dm = aggregate_backward(op, N, dst, R, arg)
+    return apply_edges_backward(msg, N, src, dst, Xj, dm, Y=Xi, e=e, H=H, want=want)
+
+
+def gin(N, src, dst, X, eps):
+    """GIN aggregation: out[i,:] = (1 + eps) * x_i + sum over incoming edges of x_j -> (out, S)."""
+    o, S, _ = propagate("sum", N, src, dst, X)
+    from_self = (1.0 + float(eps)) * _to64(X)
+    return from_self + o, np.abs(from_self) + S
+
+
+def gin_backward(N, src, dst, X, eps, R):
+    """-> dict(dX, SdX, deps): dX = (1+eps) * R + sum over outgoing edges of R[target]; deps = <R, X>."""
+    bw = propagate_backward("sum", N, src, dst, None, None, R)
+    R64 = _to64(R)
+    return dict(dX=(1.0 + float(eps)) * R64 + bw["dX"], SdX=np.abs((1.0 + float(eps)) * R64) + bw["SdX"],
+                deps=float((R64 * _to64(X)).sum()), Sdeps=float(np.abs(R64 * _to64(X)).sum()))
+
+
+def hetero_propagate(N_dst, relations):
+    """Heterogeneous graph: relations = list of dict(src, dst, X, w (or None), op ('sum' | 'mean')); every
+    relation sends from its own source node set (rows of its X) to the same target node set; the results are
+    summed over relations in list order -> (out [N_dst,F], S)."""
+    out = S = None
+    for r in relations:
+        n_src = r["X"].shape[0]
+        n = max(N_dst, n_src)
+        Xp = r["X"]
+        if n_src < n:  # the edge-list routine takes one node count: pad the source side with unused rows
+            Xp = np.concatenate([Xp, np.zeros((n - n_src, Xp.shape[1]), Xp.dtype)])
+        o, s, _ = propagate(r["op"], n, r["src"], r["dst"], Xp, r.get("w"))
+        out = o[:N_dst] if out is None else out + o[:N_dst]
+        S = s[:N_dst] if S is None else S + s[:N_dst]
+    return out, S
+
+
+def epilogue(Z, bias=None, act=None):
+    """Element-wise tail of a layer: Z + bias (per feature), then ReLU if act == 'relu' (float64 in, float64 out)."""
+    Y = np.asarray(Z, np.float64) + (0.0 if bias is None else np.asarray(bias, np.float64)[None, :])
+    return np.maximum(Y, 0.0) if act == "relu" else Y
+
+
+def epilogue_backward(Y, R, act=None):
+    """For Y = epilogue(Z): dZ = R * [Y > 0] (ReLU) or R; dbias = column sums of dZ -> (dZ, dbias, Sdbias)."""
+    dZ = _to64(R) * ((np.asarray(Y) > 0) if act == "relu" else 1.0)
+    return dZ, dZ.sum(axis=0), np.abs(dZ).sum(axis=0)
+
+
+def _to64(a):
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)

@@ -40,7 +40,7 @@
 
 enum { DT_F64 = 0, DT_F32 = 1, DT_BF16 = 2 };
 enum { OP_SUM = 0, OP_MEAN = 1, OP_MAX = 2, OP_MIN = 3 };
-enum { MSG_COPY_XJ = 0, MSG_E_MUL_XJ = 1, MSG_GAT_LOGIT = 2 };
+enum { MSG_COPY_XJ = 0, MSG_E_MUL_XJ = 1, MSG_GAT_LOGIT = 2, MSG_XI_SUB_XJ = 3, MSG_XI_DOT_XJ = 4 };
 
 static inline double ld(const void* p, int dt, int64_t i) {
     if (dt == DT_F64) return ((const double*)p)[i];
@@ -127,16 +127,33 @@ void oracle_gather(int64_t E, const int32_t* idx, const void* X, int dt, int F, 
         for (int f = 0; f < F; ++f) out[k * F + f] = ld(X, dt, (int64_t)idx[k] * F + f);
 }
 
-/* apply_edges, the per-edge message m_k of edge j -> i:
+/* apply_edges, the per-edge message m_k of edge j -> i (Sec. 3 "Message Passing": a message function of
+ * the target features xi, the source features xj and the edge features eji):
  *   COPY_XJ    m_k[f] = x_j[f]
  *   E_MUL_XJ   m_k[f] = e_k[g(f)] * x_j[f], e of width 1 (one scalar per edge), H (one per head,
  *              head of feature f is f / (F/H)) or F (element-wise)
  *   GAT_LOGIT  m_k[h] = LeakyReLU_slope(al[j,h] + ar[i,h]), F = H here; LeakyReLU(x) = x for
  *              x > 0, slope*x otherwise
- * X is the node array (for GAT_LOGIT: al), Y the second node array (ar) or NULL. */
+ *   XI_SUB_XJ  m_k[f] = x_i[f] - x_j[f]
+ *   XI_DOT_XJ  m_k[h] = sum_c x_i[h*C+c] * x_j[h*C+c], one value per head; ew = H here (number of heads,
+ *              C = F/H) and m is [E,H]
+ * X holds the source features x_j (for GAT_LOGIT: al); Y the second node array: ar for GAT_LOGIT, the
+ * target features x_i for XI_SUB_XJ / XI_DOT_XJ, NULL otherwise. */
 void oracle_apply_edges(int msg, int64_t E, const int32_t* src, const int32_t* dst, const void* X,
                         int dtx, const void* Y, int dty, const void* e, int dte, int ew, int F,
                         double slope, double* m) {
+    if (msg == MSG_XI_DOT_XJ) {
+        int H = ew, C = F / H;
+        for (int64_t k = 0; k < E; ++k) {
+            int64_t j = src[k], i = dst[k];
+            for (int h = 0; h < H; ++h) {
+                double a = 0.0;
+                for (int c = 0; c < C; ++c) a += ld(Y, dty, i * F + h * C + c) * ld(X, dtx, j * F + h * C + c);
+                m[k * H + h] = a;
+            }
+        }
+        return;
+    }
     for (int64_t k = 0; k < E; ++k) {
         int64_t j = src[k], i = dst[k];
         for (int f = 0; f < F; ++f) {
@@ -146,11 +163,71 @@ void oracle_apply_edges(int msg, int64_t E, const int32_t* src, const int32_t* d
             } else if (msg == MSG_E_MUL_XJ) {
                 int g = (ew == 1) ? 0 : (ew == F ? f : f / (F / ew));
                 v = ld(e, dte, k * ew + g) * ld(X, dtx, j * F + f);
+            } else if (msg == MSG_XI_SUB_XJ) {
+                v = ld(Y, dty, i * F + f) - ld(X, dtx, j * F + f);
             } else {
                 double s = ld(X, dtx, j * F + f) + ld(Y, dty, i * F + f);
                 v = s > 0.0 ? s : slope * s;
             }
             m[k * F + f] = v;
+        }
+    }
+}
+
+/* backward of apply_edges for dL/dm = dm (fp64; [E,F], or [E,H] for XI_DOT_XJ), original edge order:
+ *   COPY_XJ    dXj[j,:] += dm[k,:]
+ *   E_MUL_XJ   dXj[j,f] += e_k[g(f)] * dm[k,f];  de[k,g] = sum over the features f of group g of x_j[f]*dm[k,f]
+ *   XI_SUB_XJ  dXi[i,:] += dm[k,:];  dXj[j,:] -= dm[k,:]
+ *   XI_DOT_XJ  dXi[i,h,:] += dm[k,h] * x_j[h,:];  dXj[j,h,:] += dm[k,h] * x_i[h,:]
+ * dXj, dXi [N,F] and de [E,ew] are optional (NULL: not wanted); SXj, SXi, Se hold the sums of |terms|. */
+void oracle_apply_edges_backward(int msg, int32_t N, int64_t E, const int32_t* src, const int32_t* dst,
+                                 const void* X, int dtx, const void* Y, int dty, const void* e, int dte,
+                                 int ew, int F, const double* dm, double* dXj, double* SXj, double* dXi,
+                                 double* SXi, double* de, double* Se) {
+    for (int64_t x = 0; x < (int64_t)N * F; ++x) {
+        if (dXj) dXj[x] = 0.0;
+        if (SXj) SXj[x] = 0.0;
+        if (dXi) dXi[x] = 0.0;
+        if (SXi) SXi[x] = 0.0;
+    }
+    if (de) for (int64_t x = 0; x < E * ew; ++x) { de[x] = 0.0; if (Se) Se[x] = 0.0; }
+    for (int64_t k = 0; k < E; ++k) {
+        int64_t j = src[k], i = dst[k];
+        for (int f = 0; f < F; ++f) {
+            if (msg == MSG_COPY_XJ) {
+                double g = dm[k * F + f];
+                if (dXj) { dXj[j * F + f] += g; if (SXj) SXj[j * F + f] += fabs(g); }
+            } else if (msg == MSG_E_MUL_XJ) {
+                int g = (ew == 1) ? 0 : (ew == F ? f : f / (F / ew));
+                double d = dm[k * F + f];
+                if (dXj) {
+                    double t = ld(e, dte, k * ew + g) * d;
+                    dXj[j * F + f] += t;
+                    if (SXj) SXj[j * F + f] += fabs(t);
+                }
+                if (de) {
+                    double t = ld(X, dtx, j * F + f) * d;
+                    de[k * ew + g] += t;
+                    if (Se) Se[k * ew + g] += fabs(t);
+                }
+            } else if (msg == MSG_XI_SUB_XJ) {
+                double g = dm[k * F + f];
+                if (dXi) { dXi[i * F + f] += g; if (SXi) SXi[i * F + f] += fabs(g); }
+                if (dXj) { dXj[j * F + f] -= g; if (SXj) SXj[j * F + f] += fabs(g); }
+            } else if (msg == MSG_XI_DOT_XJ) {
+                int H = ew, C = F / H;
+                double g = dm[k * H + f / C];
+                if (dXi) {
+                    double t = g * ld(X, dtx, j * F + f);
+                    dXi[i * F + f] += t;
+                    if (SXi) SXi[i * F + f] += fabs(t);
+                }
+                if (dXj) {
+                    double t = g * ld(Y, dty, i * F + f);
+                    dXj[j * F + f] += t;
+                    if (SXj) SXj[j * F + f] += fabs(t);
+                }
+            }
         }
     }
 }

@@ -586,3 +586,107 @@ def test_bf16_and_f32_inputs_are_widened_exactly():
     Xb = np.array([[0x3FC0, 0xC000], [0x3F81, 0x0000]], np.uint16)
     out, _, _ = oracle.propagate("sum", 2, [0, 1], [1, 1], Xb)
     assert out[1].tolist() == [1.5 + 1.0078125, -2.0]
+
+
+# ---------------------------------------------------------------- further messages, GIN, heterogeneous sums
+def test_xi_sub_xj_and_xi_dot_xj_messages_against_dense_algebra():
+    n, e, H, Cw = 23, 140, 2, 3
+    F = H * Cw
+    src, dst = rand_graph(n, e)
+    Xj, Xi = RNG.standard_normal((n, F)), RNG.standard_normal((n, F))
+    A = dense_adj(n, src, dst)                       # A[j, i] = multiplicity of j -> i
+    deg = A.sum(axis=0)
+    o, _, _ = oracle.propagate_msg(oracle.XI_SUB_XJ, "sum", n, src, dst, Xj, Xi=Xi)
+    assert np.allclose(o, deg[:, None] * Xi - A.T @ Xj, atol=1e-12)
+    m = oracle.apply_edges(oracle.XI_DOT_XJ, src, dst, Xj, Y=Xi, H=H)
+    for h in range(H):
+        G = Xi[:, h * Cw:(h + 1) * Cw] @ Xj[:, h * Cw:(h + 1) * Cw].T      # G[i, j]
+        assert np.allclose(m[:, h], G[dst, src], atol=1e-12)
+    # direction: on the single edge 0 -> 1 the message is x_i - x_j with i = 1, j = 0
+    m = oracle.apply_edges(oracle.XI_SUB_XJ, [0], [1], Xj, Y=Xi)
+    assert np.array_equal(m[0], Xi[1] - Xj[0])
+    # max over x_i - x_j is x_i minus the smallest x_j
+    o, _, a = oracle.propagate_msg(oracle.XI_SUB_XJ, "max", n, src, dst, Xj, Xi=Xi)
+    mn, _, amn = oracle.propagate("min", n, src, dst, Xj)
+    has = deg > 0
+    assert np.allclose(o[has], (Xi - mn)[has], atol=1e-12) and np.array_equal(a, amn)
+
+
+@pytest.mark.parametrize("msg", ["copy", "emul1", "emulH", "emulF", "sub", "dot"])
+def test_apply_edges_backward_finite_differences(msg):
+    n, e, H, Cw = 15, 70, 2, 4
+    F = H * Cw
+    src, dst = rand_graph(n, e)
+    Xj, Xi = RNG.standard_normal((n, F)), RNG.standard_normal((n, F))
+    code = {"copy": oracle.COPY_XJ, "emul1": oracle.E_MUL_XJ, "emulH": oracle.E_MUL_XJ, "emulF": oracle.E_MUL_XJ,
+            "sub": oracle.XI_SUB_XJ, "dot": oracle.XI_DOT_XJ}[msg]
+    ev = {"emul1": RNG.standard_normal((e, 1)), "emulH": RNG.standard_normal((e, H)), "emulF": RNG.standard_normal((e, F))}.get(msg)
+    Y = Xi if msg in ("sub", "dot") else None
+    dm = RNG.standard_normal((e, H if msg == "dot" else F))
+    loss = lambda: (oracle.apply_edges(code, src, dst, Xj, Y=Y, e=ev, H=H) * dm).sum()
+    want = ("dXj",) + (("dXi",) if Y is not None else ()) + (("de",) if ev is not None else ())
+    bw = oracle.apply_edges_backward(code, n, src, dst, Xj, dm, Y=Y, e=ev, H=H, want=want)
+    ids = RNG.choice(Xj.size, 40, replace=False)
+    assert np.allclose(fd(loss, Xj, ids), bw["dXj"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    if Y is not None:
+        assert np.allclose(fd(loss, Xi, ids), bw["dXi"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    if ev is not None:
+        ide = RNG.choice(ev.size, 40, replace=False)
+        assert np.allclose(fd(loss, ev, ide), bw["de"].reshape(-1)[ide], rtol=1e-6, atol=1e-8)
+    # magnitude sums bound the results
+    assert (np.abs(bw["dXj"]) <= bw["SXj"] + 1e-15).all()
+
+
+def test_gin_closed_form_dense_form_and_gradient():
+    # star with hub 0 and n-1 leaves, all features 1: hub = (1+eps) + (n-1), leaf = (1+eps) + 1
+    n, eps = 6, 0.25
+    src, dst = undirected([(0, k) for k in range(1, n)])
+    o, S = oracle.gin(n, src, dst, np.ones((n, 2)), eps)
+    assert np.allclose(o[0], 1 + eps + n - 1) and np.allclose(o[1:], 1 + eps + 1) and np.allclose(S, o)
+    n, e, F = 30, 200, 4
+    src, dst = rand_graph(n, e)
+    X, R = RNG.standard_normal((n, F)), RNG.standard_normal((n, F))
+    o, _ = oracle.gin(n, src, dst, X, eps)
+    assert np.allclose(o, (dense_adj(n, src, dst).T + (1 + eps) * np.eye(n)) @ X, atol=1e-12)
+    bw = oracle.gin_backward(n, src, dst, X, eps, R)
+    ids = RNG.choice(X.size, 50, replace=False)
+    assert np.allclose(fd(lambda: (oracle.gin(n, src, dst, X, eps)[0] * R).sum(), X, ids), bw["dX"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    h = 1e-6
+    num = ((oracle.gin(n, src, dst, X, eps + h)[0] * R).sum() - (oracle.gin(n, src, dst, X, eps - h)[0] * R).sum()) / (2 * h)
+    assert abs(num - bw["deps"]) < 1e-6 * max(1.0, abs(num))
+
+
+def test_hetero_sum_equals_one_propagate_over_the_merged_graph():
+    """Three relations from three source node sets into one target set: the sum over relations equals one
+    propagate over the union graph whose sources index the stacked feature matrix (mean as 1/deg weights)."""
+    nd, F = 12, 3
+    sizes = [7, 12, 20]
+    rels, off, ms, md, mw, Xs = [], 0, [], [], [], []
+    for t, ns in enumerate(sizes):
+        e = 30 + 10 * t
+        s = RNG.integers(0, ns, e).astype(np.int32)
+        d = RNG.integers(0, nd, e).astype(np.int32)
+        X = RNG.standard_normal((ns, F))
+        op = "mean" if t == 1 else "sum"
+        w = RNG.random(e).astype(np.float32) if t == 2 else None
+        rels.append(dict(src=s, dst=d, X=X, w=w, op=op))
+        deg = np.bincount(d, minlength=nd)
+        ms.append(s + off); md.append(d); Xs.append(X)
+        mw.append(1.0 / deg[d] if op == "mean" else (w.astype(np.float64) if w is not None else np.ones(e)))
+        off += ns
+    o, S = oracle.hetero_propagate(nd, rels)
+    A = np.zeros((off, nd))
+    np.add.at(A, (np.concatenate(ms), np.concatenate(md)), np.concatenate(mw))
+    assert np.allclose(o, A.T @ np.concatenate(Xs), atol=1e-12) and (np.abs(o) <= S + 1e-15).all()
+
+
+def test_epilogue_bias_relu_and_its_backward():
+    Z = RNG.standard_normal((9, 5))
+    b = RNG.standard_normal(5)
+    R = RNG.standard_normal((9, 5))
+    Y = oracle.epilogue(Z, b, "relu")
+    assert (Y >= 0).all() and np.array_equal(Y[Y > 0], (Z + b)[Y > 0]) and np.array_equal(oracle.epilogue(Z, None, None), Z)
+    dZ, db, _ = oracle.epilogue_backward(Y, R, "relu")
+    ids = RNG.choice(Z.size, 30, replace=False)
+    assert np.allclose(fd(lambda: (oracle.epilogue(Z, b, "relu") * R).sum(), Z, ids, h=1e-7), dZ.reshape(-1)[ids], atol=1e-6)
+    assert np.allclose(fd(lambda: (oracle.epilogue(Z, b, "relu") * R).sum(), b, np.arange(5), h=1e-7), db, atol=1e-6)
