@@ -54,7 +54,15 @@ typedef enum {
 
 typedef enum { GNN_F32 = 0, GNN_BF16 = 1 } gnn_dtype;
 typedef enum { GNN_SUM = 0, GNN_MEAN = 1, GNN_MAX = 2, GNN_MIN = 3 } gnn_op;
-typedef enum { GNN_MSG_COPY_XJ = 0, GNN_MSG_E_MUL_XJ = 1, GNN_MSG_GAT_LOGIT = 2 } gnn_msg;
+typedef enum {
+    GNN_MSG_COPY_XJ = 0,   /* m = x_j */
+    GNN_MSG_E_MUL_XJ = 1,  /* m = e_ji * x_j */
+    GNN_MSG_GAT_LOGIT = 2, /* m = LeakyReLU(al_j + ar_i), per head */
+    GNN_MSG_XI_SUB_XJ = 3, /* m = x_i - x_j */
+    GNN_MSG_XI_DOT_XJ = 4  /* m = <x_i, x_j>, per head */
+} gnn_msg;
+/* which multiple c(i) of its self term a row i receives in a gnn_row_epilogue */
+typedef enum { GNN_SELF_ALWAYS = 0, GNN_SELF_TIMES_DEGREE = 1, GNN_SELF_IF_NONEMPTY = 2 } gnn_self_mode;
 
 /* Sparse form of a graph (Sec. 3 "Graph Data Structures": the sparse adjacency encoding the
  * fused operations run on).  Host struct, device arrays, all caller-owned.
@@ -169,6 +177,136 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
                                         const void* dOut, const void* X, const float* w_csrT,
                                         const int32_t* argmax, int F, gnn_dtype dtype, void* dX,
                                         float* dW, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* ------------------------------------------------------------------ more fused (message, op) pairs */
+
+/* Element-wise tail of a layer, applied to each finished row of a fused call in fp32 before its
+ * single rounding (the bias / relu of the conv layers in the training example; the self term of the
+ * GIN layer named in Sec. 3 "Graph Convolutional Layers"):
+ *   z[i,f]  = agg[i,f] + self_coef * c(i) * Xself[i,f] + bias[f]
+ *   out[i,f] = relu ? max(z[i,f], 0) : z[i,f]
+ * c(i) = 1 (GNN_SELF_ALWAYS), the number of incoming edges of i (GNN_SELF_TIMES_DEGREE), or 1 if i
+ * has an incoming edge and 0 otherwise (GNN_SELF_IF_NONEMPTY).  Xself: [N,F] of the call's dtype or
+ * NULL (no self term); bias: float [F] or NULL.  Host struct of device pointers. */
+typedef struct {
+    const void* Xself;
+    float self_coef;
+    int self_mode; /* gnn_self_mode */
+    const float* bias;
+    int relu;
+} gnn_row_epilogue;
+
+/* propagate for further "specific message functions and aggregation operations" (Sec. 3 "Message
+ * Passing"), still without materialising the E x F message tensor:
+ *   out[i,:] = epilogue( op over p in row i of m[p,:] )
+ *   COPY_XJ    m[p,:] = Xj[col[p],:]
+ *   E_MUL_XJ   m[p,f] = e[p, f / (F / e_width)] * Xj[col[p],f]; e_csr float [E,e_width] in CSR
+ *              order, e_width = 1 (any op), or H dividing F with F/H a multiple of 16 bytes worth
+ *              of elements, or F (one factor per edge and feature; e rows 16-byte aligned); widths
+ *              above 1 take SUM or MEAN only
+ *   XI_SUB_XJ  m[p,:] = Xi[i,:] - Xj[col[p],:] for p in row i; Xi [N,F] of dtype.  Computed as
+ *              c(i) * Xi[i,:] - (op' over the row of Xj[col[p],:]) with op' = op for SUM / MEAN and
+ *              the opposite extremum for MAX / MIN (the difference falls as x_j grows, and rounding
+ *              keeps that order); argmax is the position of the winning edge, the smallest among
+ *              equal x_j.  epi->Xself must be NULL for this message (the self slot is taken).
+ * epi: NULL or an epilogue.  A node with no incoming edge gets epilogue(0) and argmax -1.
+ * GIN: COPY_XJ, SUM, epi = {X, 1 + eps, GNN_SELF_ALWAYS}.  ws as for gnn_propagate_fused. */
+gnn_status gnn_propagate_msg(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* Xj, const void* Xi,
+                             const float* e_csr, int e_width, int F, gnn_dtype dtype,
+                             const gnn_row_epilogue* epi, void* out, int32_t* argmax, void* ws,
+                             size_t ws_bytes, gnn_stream stream);
+
+/* Backward of gnn_propagate_msg for dL/d(op result) = dOut [N,F] (run gnn_row_epilogue_backward
+ * first if the forward call had a bias or relu).  Each output may be NULL (skipped):
+ *   dXj [N,F]  gradient that reaches Xj through the messages, reduced over the outgoing edges of
+ *              each node in the transposed form (E_MUL_XJ: e_csrT = e in transposed-CSR order,
+ *              see gnn_permute_edge_data(t2f); MAX/MIN: argmax of the forward call), plus, if
+ *              self_grad is given, self_coef * c(j) * self_grad->Xself[j,:] in the same pass (c(j)
+ *              counts the INCOMING edges of j, as in the forward call).  Use it for the self term of
+ *              GIN (Xself = dOut, 1 + eps, GNN_SELF_ALWAYS) or when Xi and Xj of XI_SUB_XJ are one
+ *              tensor (Xself = dOut, 1, GNN_SELF_TIMES_DEGREE for SUM, GNN_SELF_IF_NONEMPTY else).
+ *              self_grad->bias must be NULL and relu 0.
+ *   dXi [N,F]  XI_SUB_XJ only: c(i) * dOut[i,:]
+ *   de_csr     E_MUL_XJ with SUM / MEAN only: float [E,e_width] in CSR order,
+ *              de[p,k] = scale(i) * sum over the features f under factor k of Xj[col[p],f]*dOut[i,f]
+ * ws as for the forward call. */
+gnn_status gnn_propagate_msg_backward(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* dOut,
+                                      const void* Xj, const float* e_csrT, int e_width,
+                                      const int32_t* argmax, int F, gnn_dtype dtype,
+                                      const gnn_row_epilogue* self_grad, void* dXj, void* dXi,
+                                      float* de_csr, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* Backward of a gnn_row_epilogue's bias and relu for Y = the forward output [N,F]:
+ *   dZ[i,f] = dY[i,f] if (!relu or Y[i,f] > 0) else 0   (dZ may alias dY)
+ *   dbias[f] = sum over i of dZ[i,f]  (float [F], may be NULL; fixed-order two-stage sum)
+ * The gradient of the self term is self_coef * c(i) * dZ[i,:] (see self_grad above).
+ * ws: gnn_row_epilogue_backward_workspace(N, F) bytes (needed only with dbias). */
+size_t gnn_row_epilogue_backward_workspace(int32_t N, int F);
+gnn_status gnn_row_epilogue_backward(const void* Y, const void* dY, int32_t N, int F, gnn_dtype dtype,
+                                     int relu, void* dZ, float* dbias, void* ws, size_t ws_bytes,
+                                     gnn_stream stream);
+
+/* GIN aggregation (the GINConv layer named in Sec. 3 "Graph Convolutional Layers"):
+ *   out[i,:] = (1 + eps) * X[i,:] + sum over incoming edges of X[j,:]       (one pass, one rounding)
+ * Backward for dL/dout = dOut: dX[j,:] = (1 + eps) * dOut[j,:] + sum over outgoing edges of
+ * dOut[target,:]; deps (device float[1], may be NULL; needs X) = <dOut, X>, a fixed-order sum.
+ * ws: gnn_gin_workspace(E, F) bytes for both calls. */
+size_t gnn_gin_workspace(int64_t E, int F);
+gnn_status gnn_gin(const gnn_csr* g, const void* X, float eps, int F, gnn_dtype dtype, void* out,
+                   void* ws, size_t ws_bytes, gnn_stream stream);
+gnn_status gnn_gin_backward(const gnn_csr* g, const void* dOut, const void* X, float eps, int F,
+                            gnn_dtype dtype, void* dX, float* deps, void* ws, size_t ws_bytes,
+                            gnn_stream stream);
+
+/* XI_DOT_XJ message (Sec. 3 "Message Passing": apply_edges with the target and source features):
+ *   s[p,h] = <Xi[i,h,:], Xj[col[p],h,:]> for p in row i, float [E,H] in CSR order; Xi, Xj [N,H,C]
+ * of dtype, H = 1 or a head spanning a power-of-two number (1..32) of 16-byte chunks.
+ * Backward for ds_csr float [E,H] (CSR order):
+ *   dXi[i,h,:] = sum over p in row i of ds[p,h] * Xj[col[p],h,:]
+ *   dXj[j,h,:] = sum over the outgoing edges of j of ds[.,h] * Xi[target,h,:]
+ * (either may be NULL).  ws: gnn_edge_dot_backward_workspace(E, H, C) bytes. */
+gnn_status gnn_edge_dot(const gnn_csr* g, const void* Xj, const void* Xi, int H, int C,
+                        gnn_dtype dtype, float* s_csr, gnn_stream stream);
+size_t gnn_edge_dot_backward_workspace(int64_t E, int H, int C);
+gnn_status gnn_edge_dot_backward(const gnn_csr* g, const void* Xj, const void* Xi,
+                                 const float* ds_csr, int H, int C, gnn_dtype dtype, void* dXj,
+                                 void* dXi, void* ws, size_t ws_bytes, gnn_stream stream);
+
+/* ------------------------------------------------------------------ heterogeneous and temporal graphs */
+
+/* A heterogeneous graph (Sec. 3 "Graph Data Structures": several node and edge types) or a sequence
+ * of temporal snapshots is run as ONE sparse form: the edge lists of the relations (snapshots) are
+ * concatenated, each with its own offsets into a common numbering of source rows and target rows.
+ *   relations    : source nodes of type t start at src_offset = first row of type t in the stacked
+ *                  feature matrix; all relations into one target type share dst_offset
+ *   snapshots    : dst_offset = t * N (every snapshot owns its block of output rows); src_offset =
+ *                  t * N for per-snapshot features or 0 for static features, which then stay
+ *                  resident in L2 across the snapshots
+ * gnn_merge_edge_lists writes the merged COO list (segment by segment, edges in their given order)
+ * and seg_out[k] = segment of merged edge k.  Build the sparse form with gnn_coo_to_csr over
+ * max(rows, columns) nodes; inside a row the positions are then ordered by segment, so the sum over
+ * relations is taken in relation order, deterministically, by the one launch of the fused
+ * propagate.  segs: HOST array of host structs holding device pointers. */
+typedef struct {
+    int64_t E;
+    const int32_t* src;
+    const int32_t* dst;
+    int32_t src_offset;
+    int32_t dst_offset;
+} gnn_edge_segment;
+gnn_status gnn_merge_edge_lists(const gnn_edge_segment* segs, int S, int32_t* src_out,
+                                int32_t* dst_out, int32_t* seg_out, gnn_stream stream);
+
+/* Per-position multipliers that give every segment its own reduction inside the merged form:
+ *   coef[p] = w[p] / max(1, number of positions of row i that belong to the segment of p)
+ * if seg_is_mean[segment] != 0, else w[p] (w == NULL: 1).  seg_csr: int32 [E], the segment of each
+ * CSR position (gnn_permute_edge_data(eid) of seg_out); seg_is_mean: device int32 [S].
+ * coef_csr / coef_csrT: float [E] in CSR / transposed-CSR order (either may be NULL).  Then
+ *   forward : gnn_propagate_fused(g, E_MUL_XJ, SUM, Xstacked, coef_csr, ...)
+ *   backward: gnn_propagate_fused_backward(g, E_MUL_XJ, SUM, dOut, ..., coef_csrT, ...) */
+gnn_status gnn_segment_coef(const gnn_csr* g, const int32_t* seg_csr, const float* w_csr,
+                            const int32_t* seg_is_mean, int S, float* coef_csr, float* coef_csrT,
+                            gnn_stream stream);
 
 /* ------------------------------------------------------------------ unfused primitives ------ */
 

@@ -235,7 +235,7 @@ gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float s
 bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz, const float* al, const float* ar,
                           float slope, int H, float* dar, cudaStream_t st);
 gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const void* dOut, int H, int C,
-                       gnn_dtype dtype, float* dW_EH, cudaStream_t st);
+                       gnn_dtype dtype, float* dW_EH, cudaStream_t st, int mean);
 
 }  // namespace gnn
 
@@ -303,7 +303,7 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
         return GNN_OK;
     }
     // dalpha[p,h] = <dOut[i,h,:], Wx[col[p],h,:]>  -> w.dz
-    rc = sddmm_heads(who, g, Wx, dOut, H, C, dtype, w.dz, st);
+    rc = sddmm_heads(who, g, Wx, dOut, H, C, dtype, w.dz, st, 0);
     if (rc != GNN_OK) return rc;
     // softmax and LeakyReLU derivatives, dz over dalpha, dar per row
     if (!gat_rows_backward_pl(g, alpha_csr, w.dz, al, ar, slope, H, w.dar, st)) {

@@ -62,7 +62,51 @@ struct PropParams {
     int H, fph;
     // optional rank-1 epilogue: out[r,f] += epi_l[r,h(f)]*epi_a[f] + epi_r[r,h(f)]*epi_b[f]
     const float *epi_l, *epi_r, *epi_a, *epi_b;
+    // MODE_EFSUM: multiplier per (position, feature), fp32 [E, ef_ld]
+    const float* ef;
+    int ef_ld;
+    // optional row epilogue (has_epi), applied in fp32 to a finished row before its single rounding:
+    //   v = agg_c * v + self_c * c(r) * self_X[r,f] + bias[f], then max(v, 0) if relu
+    // c(r) = 1 (GNN_SELF_ALWAYS), the length of row r in self_rowptr (GNN_SELF_TIMES_DEGREE), or 1 if that
+    // length is positive else 0 (GNN_SELF_IF_NONEMPTY)
+    int has_epi;
+    float agg_c, self_c;
+    int self_mode, relu;
+    const void* self_X;
+    uint32_t self_ld;  // bytes between rows of self_X
+    const int64_t* self_rowptr;
+    const float* bias;  // [F] or nullptr
 };
+
+// the row epilogue of PropParams on the 16-byte column ci of finished row `row`
+template <typename T>
+__device__ __forceinline__ void row_epilogue(const PropParams& P, int64_t row, int ci, float* v) {
+    constexpr int EPC = Chunk<T>::N;
+    if (!P.has_epi) return;
+    if (P.agg_c != 1.0f) {
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] *= P.agg_c;
+    }
+    if (P.self_X) {
+        float c = P.self_c;
+        if (P.self_mode != GNN_SELF_ALWAYS) {
+            const int64_t d = P.self_rowptr[row + 1] - P.self_rowptr[row];
+            c = (P.self_mode == GNN_SELF_TIMES_DEGREE) ? c * (float)d : (d > 0 ? c : 0.f);
+        }
+        float x[EPC];
+        Chunk<T>::unpack(__ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(P.self_X) + (size_t)row * P.self_ld + (size_t)ci * 16)), x);
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] = fmaf(c, x[j], v[j]);
+    }
+    if (P.bias) {
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] += P.bias[ci * EPC + j];
+    }
+    if (P.relu) {
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) v[j] = fmaxf(v[j], 0.f);
+    }
+}
 
 // d.xy += w.xy * x.xy as one packed fp32x2 FMA (each half is an IEEE fused multiply-add)
 __device__ __forceinline__ void fma2(float& a0, float& a1, float x0, float x1, float w0, float w1) {
@@ -155,9 +199,28 @@ struct Walker {
     static constexpr bool BATCH_TAIL = (MODE == MODE_MAX || MODE == MODE_MIN);
     static constexpr int EPC = Chunk<T>::N;
     static constexpr int NG = 32 / LPR;
-    static constexpr int U = (LPR >= 16) ? (PF_U_WIDE / VPL) : PF_U_NARROW;
+    static constexpr bool EF = (MODE == MODE_EFSUM);  // one multiplier per (position, feature)
+    // the per-feature mode also streams EPC multipliers per gathered chunk: half as many gathers in flight
+    static constexpr int U = (LPR >= 16) ? (EF ? (PF_U_WIDE / VPL > 1 ? PF_U_WIDE / VPL / 2 : 1) : PF_U_WIDE / VPL) : PF_U_NARROW;
+    static constexpr int MW = EF ? EPC : 1;  // multipliers a lane holds per gathered 16-byte chunk
     static constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
     using A = Acc<T, VPL, MODE>;
+
+    // multipliers of one position for this lane's chunk v: per head (MODE_HEADSUM) or per feature (MODE_EFSUM)
+    __device__ __forceinline__ static void load_mul(const PropParams& P, const float* base, size_t rel, float* dst) {
+        if (MODE == MODE_HEADSUM) {
+            dst[0] = __ldg(base + rel * P.H);
+        } else if (EF) {
+            const float4* q = reinterpret_cast<const float4*>(base + rel * P.ef_ld);
+#pragma unroll
+            for (int t = 0; t < MW / 4; ++t) {
+                const float4 a = __ldcs(q + t);
+                dst[4 * t] = a.x; dst[4 * t + 1] = a.y; dst[4 * t + 2] = a.z; dst[4 * t + 3] = a.w;
+            }
+        } else {
+            dst[0] = 0.f;
+        }
+    }
 
     // copy indices and multipliers of positions [sb, se) into shared memory (one round trip)
     __device__ __forceinline__ static void stage(const PropParams& P, int64_t sb, int64_t se, int lane,
@@ -185,8 +248,13 @@ struct Walker {
             float x[EPC];
             Chunk<T>::unpack(buf[v], x);
             if (MODE == MODE_HEADSUM) {
+                const float m = hw[v] * w0;  // w0 = 1 unless the gathered rows are rescaled (backward of the mean)
 #pragma unroll
-                for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], hw[v], hw[v]);
+                for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], m, m);
+            } else if (EF) {
+#pragma unroll
+                for (int j = 0; j < EPC; j += 2)
+                    fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], hw[v * MW + j] * w0, hw[v * MW + j + 1] * w0);
             } else if (MODE == MODE_SUM) {
 #pragma unroll
                 for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], w0, w1);
@@ -230,17 +298,18 @@ struct Walker {
             Xl[v] = reinterpret_cast<const char*>(P.X) + (size_t)c0[v] * 16;
         }
         const int lane_chunk0 = (li < P.nvec) ? li : 0;  // VPL > 1 only with full rows of 32 lanes
-        const float* whl[VPL];  // MODE_HEADSUM: this lane's head column of the multiplier matrix
+        const float* whl[VPL];  // this lane's head column (MODE_HEADSUM) or feature columns (MODE_EFSUM) of the multipliers
 #pragma unroll
         for (int v = 0; v < VPL; ++v)
-            whl[v] = (MODE == MODE_HEADSUM) ? P.wh + (size_t)sb * P.H + (c0[v] * EPC) / P.fph : nullptr;
+            whl[v] = (MODE == MODE_HEADSUM) ? P.wh + (size_t)sb * P.H + (c0[v] * EPC) / P.fph
+                     : EF ? P.ef + (size_t)sb * P.ef_ld + (size_t)c0[v] * EPC : nullptr;
         const int i1 = (int)(e1 - sb);
         int i = (int)(p0 - sb) + g;
         // full groups of U positions per lane group: no predicates
         for (; i + (U - 1) * NG < i1; i += NG * U) {
             int4 e[U];
             uint4 buf[U][VPL];
-            float hw[U][VPL];
+            float hw[U][VPL * MW];
 #pragma unroll
             for (int u = 0; u < U; ++u) e[u] = S.e[i + u * NG];
 #pragma unroll
@@ -248,7 +317,7 @@ struct Walker {
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     buf[u][v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e[u].x * row_bytes, pol_keep);
-                    hw[u][v] = (MODE == MODE_HEADSUM) ? __ldg(whl[v] + (size_t)(i + u * NG) * P.H) : 0.f;
+                    load_mul(P, whl[v], (size_t)(i + u * NG), &hw[u][v * MW]);
                 }
 #pragma unroll
             for (int u = 0; u < U; ++u) consume(P, e[u], buf[u], hw[u], (int32_t)(sb + i + u * NG), lane_chunk0, acc);
@@ -259,7 +328,7 @@ struct Walker {
                 const int cnt = (i1 - i + NG - 1) / NG;
                 int4 e[U];
                 uint4 buf[U][VPL];
-                float hw[U][VPL];
+                float hw[U][VPL * MW];
 #pragma unroll
                 for (int u = 0; u < U - 1; ++u)
                     if (u < cnt) {
@@ -267,7 +336,7 @@ struct Walker {
 #pragma unroll
                         for (int v = 0; v < VPL; ++v) {
                             buf[u][v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e[u].x * row_bytes, pol_keep);
-                            hw[u][v] = (MODE == MODE_HEADSUM) ? __ldg(whl[v] + (size_t)(i + u * NG) * P.H) : 0.f;
+                            load_mul(P, whl[v], (size_t)(i + u * NG), &hw[u][v * MW]);
                         }
                     }
 #pragma unroll
@@ -279,11 +348,11 @@ struct Walker {
             for (; i < i1; i += NG) {
                 const int4 e = S.e[i];
                 uint4 buf[VPL];
-                float hw[VPL];
+                float hw[VPL * MW];
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     buf[v] = ld_hint16(Xl[v] + (size_t)(uint32_t)e.x * row_bytes, pol_keep);
-                    hw[v] = (MODE == MODE_HEADSUM) ? __ldg(whl[v] + (size_t)i * P.H) : 0.f;
+                    load_mul(P, whl[v], (size_t)i, &hw[v * MW]);
                 }
                 consume(P, e, buf, hw, (int32_t)(sb + i), lane_chunk0, acc);
             }
@@ -336,6 +405,7 @@ struct Walker {
                 for (int j = 0; j < EPC; ++j) acc.v[v][j] = acc.v[v][j] / d;
             }
             if (MODE == MODE_HEADSUM) epilogue(P, row, ci, acc.v[v]);
+            row_epilogue<T>(P, row, ci, acc.v[v]);
             st_stream16(ob + (size_t)ci * 16, Chunk<T>::pack(acc.v[v]));
             if (ARG && P.argmax) {
                 int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
@@ -504,6 +574,7 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
 #pragma unroll
         for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
     }
+    row_epilogue<T>(P, r, ci, v);
     char* ob = reinterpret_cast<char*>(P.out) + (size_t)r * P.out_ld + (size_t)ci * 16;
     *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
     if (ARG && P.argmax) {
@@ -549,7 +620,9 @@ struct FlatSmem {
 template <typename T, int LPR, int MODE>
 __global__ void __launch_bounds__(FL_WARPS * 32, (MODE == MODE_SUM || MODE == MODE_HEADSUM) ? 6 : 4)
 propagate_flat_kernel(const PropParams P) {
-    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = MODE == MODE_ROUTE ? FL_U / 2 : FL_U;
+    constexpr bool EF = MODE == MODE_EFSUM;  // one multiplier per (position, feature)
+    constexpr int EPC = Chunk<T>::N, NG = 32 / LPR, U = (MODE == MODE_ROUTE || EF) ? FL_U / 2 : FL_U;
+    constexpr int MW = EF ? EPC : 1;
     constexpr bool ARG = MODE == MODE_MAX || MODE == MODE_MIN;
     const int L = P.chunk / NG;  // positions per lane group; P.chunk is 64, 128 or 256 here
     __shared__ FlatSmem<EPC, ARG> s_all[FL_WARPS];
@@ -572,6 +645,7 @@ propagate_flat_kernel(const PropParams P) {
 #pragma unroll
             for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
         }
+        row_epilogue<T>(P, row, ci, v);
         st_stream16(outb + (size_t)row * P.out_ld + (size_t)ci * 16, Chunk<T>::pack(v));
         if (ARG && P.argmax) {
             int32_t* ap = P.argmax + (size_t)row * P.F + (size_t)ci * EPC;
@@ -717,9 +791,19 @@ propagate_flat_kernel(const PropParams P) {
     const int32_t* const route_l = (MODE == MODE_ROUTE) ? P.route_arg + (size_t)(col_lane ? li : 0) * EPC : nullptr;
     // per-head mode: this lane's head column of the [E,H] multiplier matrix, at the chunk's first position
     const float* const wh_l = (MODE == MODE_HEADSUM) ? P.wh + ((col_lane ? li : 0) * EPC) / P.fph : nullptr;
+    // per-feature mode: this lane's feature columns of the [E,F] multiplier matrix, at the chunk's first position
+    const float* const ef_l = EF ? P.ef + (size_t)cs * P.ef_ld + (size_t)(col_lane ? li : 0) * EPC : nullptr;
+    auto load_ef = [&](int pos_in_chunk, float* dst) {
+        const float4* q = reinterpret_cast<const float4*>(ef_l + (size_t)pos_in_chunk * P.ef_ld);
+#pragma unroll
+        for (int t = 0; t < MW / 4; ++t) {
+            const float4 a4 = __ldcs(q + t);
+            dst[4 * t] = a4.x; dst[4 * t + 1] = a4.y; dst[4 * t + 2] = a4.z; dst[4 * t + 3] = a4.w;
+        }
+    };
     for (int i = a; i < b; i += U) {
         uint4 buf[U];
-        float hw[MODE == MODE_HEADSUM ? U : 1];
+        float hw[(MODE == MODE_HEADSUM || EF) ? U : 1][MW];
         int4 win[MODE == MODE_ROUTE ? U : 1][MODE == MODE_ROUTE ? EPC / 4 : 1];
         const int nu = min(U, b - i);  // U except at the ragged end of the last chunk
         if (nu == U) {
@@ -729,7 +813,8 @@ propagate_flat_kernel(const PropParams P) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
-                if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
+                if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0][0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
+                if (EF) load_ef(i + u, hw[EF ? u : 0]);
                 if (MODE == MODE_ROUTE) {
 #pragma unroll
                     for (int q = 0; q < EPC / 4; ++q)
@@ -743,7 +828,8 @@ propagate_flat_kernel(const PropParams P) {
                 if (u < nu) {
                     const int cc = S.e[i + u].x;
                     buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * P.x_ld, pol_keep);
-                    if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
+                    if (MODE == MODE_HEADSUM) hw[MODE == MODE_HEADSUM ? u : 0][0] = __ldg(wh_l + (size_t)(uint32_t)S.e[i + u].w * P.H);
+                    if (EF) load_ef(i + u, hw[EF ? u : 0]);
                     if (MODE == MODE_ROUTE) {
 #pragma unroll
                         for (int q = 0; q < EPC / 4; ++q)
@@ -782,8 +868,13 @@ propagate_flat_kernel(const PropParams P) {
                     if (t.z == e.w) acc[4 * q + 2] = fmaf(w, x[4 * q + 2], acc[4 * q + 2]);
                     if (t.w == e.w) acc[4 * q + 3] = fmaf(w, x[4 * q + 3], acc[4 * q + 3]);
                 }
+            } else if (EF) {
+#pragma unroll
+                for (int j = 0; j < EPC; j += 2)
+                    fma2(acc[j], acc[j + 1], x[j], x[j + 1], hw[EF ? u : 0][EF ? j : 0] * w, hw[EF ? u : 0][EF ? j + 1 : 0] * w);
             } else {
-                const float m = (MODE == MODE_HEADSUM) ? hw[MODE == MODE_HEADSUM ? u : 0] : w;
+                // w = 1 in the per-head mode unless the gathered rows are rescaled (backward of the mean)
+                const float m = (MODE == MODE_HEADSUM) ? hw[MODE == MODE_HEADSUM ? u : 0][0] * w : w;
 #pragma unroll
                 for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], m, m);
             }
@@ -1189,6 +1280,7 @@ static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStr
     if (vpl == 1 && P.chunk <= PF_SLAB && P.E > 0) {
         if (mode == MODE_SUM) launch_flat<T, MODE_SUM>(P, lpr, st);
         else if (mode == MODE_HEADSUM) launch_flat<T, MODE_HEADSUM>(P, lpr, st);
+        else if (mode == MODE_EFSUM) launch_flat<T, MODE_EFSUM>(P, lpr, st);
         else if (mode == MODE_MAX) launch_flat<T, MODE_MAX>(P, lpr, st);
         else if (mode == MODE_MIN) launch_flat<T, MODE_MIN>(P, lpr, st);
         else launch_flat<T, MODE_ROUTE>(P, lpr, st);
@@ -1199,6 +1291,7 @@ static void launch_mode(const PropParams& P, int mode, int lpr, int vpl, cudaStr
         case MODE_MAX: launch_chunks<T, MODE_MAX>(P, lpr, vpl, st); break;
         case MODE_MIN: launch_chunks<T, MODE_MIN>(P, lpr, vpl, st); break;
         case MODE_HEADSUM: launch_chunks<T, MODE_HEADSUM>(P, lpr, vpl, st); break;
+        case MODE_EFSUM: launch_chunks<T, MODE_EFSUM>(P, lpr, vpl, st); break;
         default: launch_chunks<T, MODE_ROUTE>(P, lpr, vpl, st); break;
     }
 }
@@ -1263,7 +1356,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
                        const int32_t* col, const float* w, const void* X, void* out,
                        int32_t* argmax, const int64_t* gscale_rowptr, const int32_t* route_arg,
                        const int32_t* route_pos, int mean, int F, gnn_dtype dtype, void* ws,
-                       size_t ws_bytes, cudaStream_t st, const HeadExtra* hx) {
+                       size_t ws_bytes, cudaStream_t st, const HeadExtra* hx, const RowExtra* rx) {
     const int s = elem_size(dtype);
     GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED,
                 "%s: F*sizeof(element) = %d must be a multiple of 16 bytes", who, F * s);
@@ -1294,6 +1387,23 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
         GNN_REQUIRE(mode != MODE_HEADSUM, GNN_ERR_INVALID_ARG, "%s: per-head mode without weights", who);
     }
     P.x_ld = P.out_ld = (uint32_t)nvec * 16;
+    P.ef = nullptr; P.ef_ld = 0; P.has_epi = 0; P.agg_c = 1.0f; P.self_c = 0.f; P.self_mode = GNN_SELF_ALWAYS; P.relu = 0;
+    P.self_X = nullptr; P.self_ld = (uint32_t)nvec * 16; P.self_rowptr = rowptr; P.bias = nullptr;
+    if (rx) {
+        GNN_REQUIRE(mode == MODE_EFSUM ? (rx->ef != nullptr || E == 0) : rx->ef == nullptr, GNN_ERR_INVALID_ARG,
+                    "%s: per-feature multipliers and mode disagree", who);
+        GNN_REQUIRE(!rx->ef || (rx->ef_ld >= F && rx->ef_ld % 4 == 0 && aligned16(rx->ef)), GNN_ERR_INVALID_ARG,
+                    "%s: per-feature multipliers must be 16-byte aligned rows of at least F floats", who);
+        GNN_REQUIRE(!rx->self_X || aligned16(rx->self_X), GNN_ERR_INVALID_ARG, "%s: the self-term matrix must be 16-byte aligned", who);
+        GNN_REQUIRE(rx->self_mode >= GNN_SELF_ALWAYS && rx->self_mode <= GNN_SELF_IF_NONEMPTY, GNN_ERR_INVALID_ARG, "%s: bad self mode", who);
+        P.ef = rx->ef; P.ef_ld = rx->ef_ld;
+        P.agg_c = rx->agg_c; P.self_X = rx->self_X; P.self_c = rx->self_c; P.self_mode = rx->self_mode;
+        if (rx->self_rowptr) P.self_rowptr = rx->self_rowptr;
+        P.bias = rx->bias; P.relu = rx->relu;
+        P.has_epi = (rx->agg_c != 1.0f || rx->self_X || rx->bias || rx->relu) ? 1 : 0;
+    } else {
+        GNN_REQUIRE(mode != MODE_EFSUM, GNN_ERR_INVALID_ARG, "%s: per-feature mode without multipliers", who);
+    }
     // Column slabs: when rows are wider than 512 bytes and the gathered matrix is far larger than L2,
     // sum reductions run one 512-byte column slab at a time.  Each pass re-reads the index stream but
     // gathers from a 4x (2x) narrower matrix, of which 4x (2x) more rows stay in L2: fewer DRAM
@@ -1305,6 +1415,8 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
         for (int sl = 0; sl < nslab; ++sl) {
             P.X = (const char*)X + (size_t)sl * 512;
             P.out = (char*)out + (size_t)sl * 512;
+            if (rx && rx->self_X) P.self_X = (const char*)rx->self_X + (size_t)sl * 512;
+            if (rx && rx->bias) P.bias = rx->bias + (size_t)sl * fslab;
             if (dtype == GNN_F32) launch_mode<float>(P, mode, 32, 1, st);
             else launch_mode<__nv_bfloat16>(P, mode, 32, 1, st);
         }
@@ -1317,7 +1429,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
 // dW[p,h] = <X[col[p],h,:], dOut[i,h,:]> for p in row i: the per-head edge dot products of the
 // attention backward pass
 gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const void* dOut, int H, int C,
-                       gnn_dtype dtype, float* dW_EH, cudaStream_t st) {
+                       gnn_dtype dtype, float* dW_EH, cudaStream_t st, int mean) {
     const int s = elem_size(dtype), F = H * C;
     GNN_REQUIRE(((size_t)C * s) % 16 == 0, GNN_ERR_UNSUPPORTED, "%s: a head must be a multiple of 16 bytes wide", who);
     const int lph = C * s / 16;
@@ -1330,7 +1442,28 @@ gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const v
     if (g->E == 0) return GNN_OK;
     SddmmParams S;
     S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW_EH;
-    S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = 0; S.nchunks = num_slabs(g->E); S.H = H; S.lph = lph;
+    S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = mean; S.nchunks = num_slabs(g->E); S.H = H; S.lph = lph;
+    if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
+    else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
+// one dot product per edge (H == 1; scaled by 1 / row length if mean) or per edge and head
+gnn_status run_sddmm(const char* who, const gnn_csr* g, const void* X, const void* D, int H, int C, int mean,
+                     gnn_dtype dtype, float* dW, cudaStream_t st) {
+    if (H > 1) {
+        return sddmm_heads(who, g, X, D, H, C, dtype, dW, st, mean);
+    }
+    const int s = elem_size(dtype), F = C;
+    GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED, "%s: F*sizeof(element) must be a multiple of 16 bytes", who);
+    int lpr, vpl;
+    GNN_REQUIRE(pick_shape(F * s / 16, &lpr, &vpl), GNN_ERR_UNSUPPORTED, "%s: feature rows wider than 2048 bytes", who);
+    GNN_REQUIRE(aligned16(X) && aligned16(D), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
+    if (g->E == 0) return GNN_OK;
+    SddmmParams S;
+    S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = D; S.dW = dW;
+    S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = mean; S.nchunks = num_slabs(g->E); S.H = 1; S.lph = 0;
     if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
     else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
     GNN_CHECK_LAUNCH(who);
@@ -1429,19 +1562,8 @@ gnn_status gnn_propagate_fused_backward(const gnn_csr* g, gnn_msg msg, gnn_op op
     if (dW) {
         GNN_REQUIRE(!mm, GNN_ERR_UNSUPPORTED, "%s: dW is defined for SUM/MEAN only", who);
         GNN_REQUIRE(X, GNN_ERR_INVALID_ARG, "%s: dW needs X", who);
-        const int s = elem_size(dtype);
-        GNN_REQUIRE(F > 0 && ((size_t)F * s) % 16 == 0, GNN_ERR_UNSUPPORTED, "%s: F*sizeof(element) must be a multiple of 16 bytes", who);
-        int lpr, vpl;
-        GNN_REQUIRE(pick_shape(F * s / 16, &lpr, &vpl), GNN_ERR_UNSUPPORTED, "%s: feature rows wider than 2048 bytes", who);
-        GNN_REQUIRE(aligned16(X) && aligned16(dOut), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
-        if (g->E > 0) {
-            SddmmParams S;
-            S.rowptr = g->rowptr; S.col = g->col; S.X = X; S.dOut = dOut; S.dW = dW;
-            S.N = g->N; S.E = g->E; S.nvec = F * s / 16; S.mean = (op == GNN_MEAN); S.nchunks = num_slabs(g->E); S.H = 1; S.lph = 0;
-            if (dtype == GNN_F32) launch_sddmm<float>(S, lpr, vpl, st);
-            else launch_sddmm<__nv_bfloat16>(S, lpr, vpl, st);
-            GNN_CHECK_LAUNCH(who);
-        }
+        gnn_status rc = run_sddmm(who, g, X, dOut, 1, F, op == GNN_MEAN, dtype, dW, st);
+        if (rc != GNN_OK) return rc;
     }
     return GNN_OK;
 }

@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libgnn_b200.so")
 _lib = None
 
 SUM, MEAN, MAX, MIN = 0, 1, 2, 3
-COPY_XJ, E_MUL_XJ, GAT_LOGIT = 0, 1, 2
+COPY_XJ, E_MUL_XJ, GAT_LOGIT, XI_SUB_XJ, XI_DOT_XJ = 0, 1, 2, 3, 4
+SELF_ALWAYS, SELF_TIMES_DEGREE, SELF_IF_NONEMPTY = 0, 1, 2
 F32, BF16 = 0, 1
 OPS = {"sum": SUM, "mean": MEAN, "max": MAX, "min": MIN}
 STATUS_NAMES = ["OK", "INVALID_ARG", "INDEX_OUT_OF_RANGE", "NOT_SORTED", "WORKSPACE_TOO_SMALL", "UNSUPPORTED", "CUDA", "TIMEOUT"]
@@ -34,8 +35,18 @@ class CsrStruct(C.Structure):
                 ("rowptrT", C.c_void_p), ("colT", C.c_void_p), ("eidT", C.c_void_p), ("t2f", C.c_void_p)]
 
 
+class RowEpilogueStruct(C.Structure):
+    _fields_ = [("Xself", C.c_void_p), ("self_coef", C.c_float), ("self_mode", C.c_int), ("bias", C.c_void_p), ("relu", C.c_int)]
+
+
+class EdgeSegmentStruct(C.Structure):
+    _fields_ = [("E", C.c_int64), ("src", C.c_void_p), ("dst", C.c_void_p), ("src_offset", C.c_int32), ("dst_offset", C.c_int32)]
+
+
 _VP, _I32, _I64, _INT, _SZ, _F = C.c_void_p, C.c_int32, C.c_int64, C.c_int, C.c_size_t, C.c_float
 _CSR = C.POINTER(CsrStruct)
+_EPI = C.POINTER(RowEpilogueStruct)
+_SEG = C.POINTER(EdgeSegmentStruct)
 
 # name -> (restype, argtypes); mirrors include/gnn.h
 SIGNATURES = {
@@ -53,6 +64,18 @@ SIGNATURES = {
     "gnn_propagate_fused_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_static_max_bytes": (_SZ, []),
     "gnn_propagate_fused_static": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP]),
+    "gnn_propagate_msg": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _EPI, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_msg_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _VP, _INT, _INT, _EPI, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_row_epilogue_backward_workspace": (_SZ, [_I32, _INT]),
+    "gnn_row_epilogue_backward": (_INT, [_VP, _VP, _I32, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_gin_workspace": (_SZ, [_I64, _INT]),
+    "gnn_gin": (_INT, [_CSR, _VP, _F, _INT, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_gin_backward": (_INT, [_CSR, _VP, _VP, _F, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_edge_dot": (_INT, [_CSR, _VP, _VP, _INT, _INT, _INT, _VP, _VP]),
+    "gnn_edge_dot_backward_workspace": (_SZ, [_I64, _INT, _INT]),
+    "gnn_edge_dot_backward": (_INT, [_CSR, _VP, _VP, _VP, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_merge_edge_lists": (_INT, [_SEG, _INT, _VP, _VP, _VP, _VP]),
+    "gnn_segment_coef": (_INT, [_CSR, _VP, _VP, _VP, _INT, _VP, _VP, _VP]),
     "gnn_gather": (_INT, [_VP, _I64, _VP, _I32, _INT, _INT, _VP, _VP]),
     "gnn_gather_backward": (_INT, [_CSR, _INT, _VP, _INT, _INT, _VP, _VP, _SZ, _VP]),
     "gnn_apply_edges": (_INT, [_CSR, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP]),
@@ -256,6 +279,137 @@ def propagate_fused_backward_host(g: Graph, h_dOut, op, w_csrT, h_dX, d_in, d_ou
     _check(load().gnn_propagate_fused_backward_host(g.ref, msg, _op(op), _p(h_dOut), _pf32(w_csrT, "w_csrT"), _pi(argmax, torch.int32, "argmax"), F, _dtype(h_dOut),
                                                     _p(h_dX), _p(d_in), _p(d_out), _p(ws), ws.numel(), _stream()))
     return h_dX
+
+
+# ------------------------------------------------------------------ more (message, op) pairs, GIN, XI_DOT_XJ
+def _epi(epi):
+    """dict(Xself=, self_coef=, self_mode=, bias=, relu=) -> (struct or None, the tensors it points to)."""
+    if epi is None:
+        return None, ()
+    xs, b = epi.get("Xself"), epi.get("bias")
+    st = RowEpilogueStruct(xs.data_ptr() if xs is not None else None, float(epi.get("self_coef", 0.0)),
+                           int(epi.get("self_mode", SELF_ALWAYS)), _pf32(b, "bias").value if b is not None else None,
+                           int(bool(epi.get("relu", False))))
+    return C.byref(st), (st, xs, b)
+
+
+def propagate_msg(g: Graph, msg, Xj, Xi=None, e_csr=None, op="sum", epi=None, out=None, argmax=None, ws=None):
+    """gnn_propagate_msg -> out, or (out, argmax) for max/min.  e_csr: float32 [E] or [E,width] in CSR order."""
+    Xj = _dev(Xj)
+    F = Xj.shape[1]
+    opc = _op(op)
+    ew = 0 if e_csr is None else (1 if e_csr.dim() == 1 else e_csr.shape[1])
+    if out is None:
+        out = torch.empty((g.N, F), dtype=Xj.dtype, device=Xj.device)
+    if opc in (MAX, MIN) and argmax is None:
+        argmax = torch.empty((g.N, F), dtype=torch.int32, device=Xj.device)
+    ws = _ws(g.E, F, opc, Xj.device, ws)
+    ep, keep = _epi(epi)
+    _check(load().gnn_propagate_msg(g.ref, msg, opc, _p(Xj), _p(Xi), _pf32(e_csr, "e_csr"), ew, F, _dtype(Xj), ep, _p(out),
+                                    _pi(argmax, torch.int32, "argmax"), _p(ws), ws.numel(), _stream()))
+    del keep
+    return (out, argmax) if opc in (MAX, MIN) else out
+
+
+def propagate_msg_backward(g: Graph, msg, dOut, op="sum", Xj=None, e_csrT=None, e_width=0, argmax=None, self_grad=None,
+                           want_dXj=True, want_dXi=False, want_de=False, ws=None):
+    """gnn_propagate_msg_backward -> dict(dXj, dXi, de) with None for the outputs not asked for."""
+    dOut = _dev(dOut)
+    F = dOut.shape[1]
+    opc = _op(op)
+    ew = e_width or (0 if e_csrT is None else (1 if e_csrT.dim() == 1 else e_csrT.shape[1]))
+    dev = dOut.device
+    dXj = torch.empty((g.N, F), dtype=dOut.dtype, device=dev) if want_dXj else None
+    dXi = torch.empty((g.N, F), dtype=dOut.dtype, device=dev) if want_dXi else None
+    de = torch.empty((max(g.E, 1), max(ew, 1)), dtype=torch.float32, device=dev) if want_de else None
+    ws = _ws(g.E, F, opc, dev, ws)
+    sg, keep = _epi(self_grad)
+    _check(load().gnn_propagate_msg_backward(g.ref, msg, opc, _p(dOut), _p(Xj), _pf32(e_csrT, "e_csrT"), ew, _pi(argmax, torch.int32, "argmax"),
+                                             F, _dtype(dOut), sg, _p(dXj), _p(dXi), _p(de), _p(ws), ws.numel(), _stream()))
+    del keep
+    return dict(dXj=dXj, dXi=dXi, de=None if de is None else de[:g.E])
+
+
+def row_epilogue_backward(Y, dY, relu=True, want_dbias=True, dZ=None, ws=None):
+    """-> (dZ, dbias or None)"""
+    dY = _dev(dY)
+    N, F = dY.shape
+    if dZ is None:
+        dZ = torch.empty_like(dY)
+    dbias = torch.empty(F, dtype=torch.float32, device=dY.device) if want_dbias else None
+    if ws is None:
+        ws = torch.empty(load().gnn_row_epilogue_backward_workspace(N, F), dtype=torch.uint8, device=dY.device)
+    _check(load().gnn_row_epilogue_backward(_p(Y), _p(dY), N, F, _dtype(dY), int(bool(relu)), _p(dZ), _p(dbias), _p(ws), ws.numel(), _stream()))
+    return dZ, dbias
+
+
+def gin(g: Graph, X, eps, out=None, ws=None):
+    X = _dev(X)
+    F = X.shape[1]
+    if out is None:
+        out = torch.empty((g.N, F), dtype=X.dtype, device=X.device)
+    if ws is None:
+        ws = torch.empty(load().gnn_gin_workspace(g.E, F), dtype=torch.uint8, device=X.device)
+    _check(load().gnn_gin(g.ref, _p(X), float(eps), F, _dtype(X), _p(out), _p(ws), ws.numel(), _stream()))
+    return out
+
+
+def gin_backward(g: Graph, dOut, eps, X=None, want_deps=False, ws=None):
+    """-> (dX, deps as a float32 device tensor of one element, or None)"""
+    dOut = _dev(dOut)
+    F = dOut.shape[1]
+    dX = torch.empty((g.N, F), dtype=dOut.dtype, device=dOut.device)
+    deps = torch.empty(1, dtype=torch.float32, device=dOut.device) if want_deps else None
+    if ws is None:
+        ws = torch.empty(load().gnn_gin_workspace(g.E, F), dtype=torch.uint8, device=dOut.device)
+    _check(load().gnn_gin_backward(g.ref, _p(dOut), _p(X), float(eps), F, _dtype(dOut), _p(dX), _p(deps), _p(ws), ws.numel(), _stream()))
+    return dX, deps
+
+
+def edge_dot(g: Graph, Xj, Xi, H=1):
+    """s[p,h] = <Xi[row(p),h,:], Xj[col[p],h,:]> -> float32 [E,H], CSR order."""
+    Xj, Xi = _dev(Xj), _dev(Xi)
+    F = Xj.shape[1]
+    s = torch.empty((max(g.E, 1), H), dtype=torch.float32, device=Xj.device)
+    _check(load().gnn_edge_dot(g.ref, _p(Xj), _p(Xi), H, F // H, _dtype(Xj), _p(s), _stream()))
+    return s[:g.E]
+
+
+def edge_dot_backward(g: Graph, Xj, Xi, ds_csr, H=1, want_dXj=True, want_dXi=True, ws=None):
+    Xj, Xi = _dev(Xj), _dev(Xi)
+    N, F = Xj.shape
+    dXj = torch.empty_like(Xj) if want_dXj else None
+    dXi = torch.empty_like(Xi) if want_dXi else None
+    if ws is None:
+        ws = torch.empty(load().gnn_edge_dot_backward_workspace(g.E, H, F // H), dtype=torch.uint8, device=Xj.device)
+    _check(load().gnn_edge_dot_backward(g.ref, _p(Xj), _p(Xi), _pf32(ds_csr, "ds_csr"), H, F // H, _dtype(Xj), _p(dXj), _p(dXi), _p(ws), ws.numel(), _stream()))
+    return dXj, dXi
+
+
+# ------------------------------------------------------------------ heterogeneous / temporal graphs
+def merge_edge_lists(segments):
+    """segments: list of (src, dst, src_offset, dst_offset) with int32 device tensors -> (src, dst, seg) of the merged list."""
+    S = len(segments)
+    arr = (EdgeSegmentStruct * S)()
+    total = 0
+    for k, (src, dst, so, do) in enumerate(segments):
+        arr[k] = EdgeSegmentStruct(src.numel(), _pi(src, torch.int32, "src").value if src.numel() else None,
+                                   _pi(dst, torch.int32, "dst").value if dst.numel() else None, int(so), int(do))
+        total += src.numel()
+    dev = segments[0][0].device
+    so_, do_, sg_ = (torch.empty(max(total, 1), dtype=torch.int32, device=dev) for _ in range(3))
+    _check(load().gnn_merge_edge_lists(arr, S, _p(so_), _p(do_), _p(sg_), _stream()))
+    return so_[:total], do_[:total], sg_[:total]
+
+
+def segment_coef(g: Graph, seg_csr, seg_is_mean, w_csr=None, want_T=True):
+    """-> (coef_csr, coef_csrT or None): per-position multipliers of a merged multi-relation / multi-snapshot form."""
+    dev = g.rowptr.device
+    coef = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev)
+    coefT = torch.empty(max(g.E, 1), dtype=torch.float32, device=dev) if want_T else None
+    _check(load().gnn_segment_coef(g.ref, _pi(seg_csr, torch.int32, "seg_csr"), _pf32(w_csr, "w_csr"), _pi(seg_is_mean, torch.int32, "seg_is_mean"),
+                                   seg_is_mean.numel(), _p(coef), _p(coefT), _stream()))
+    return coef[:g.E], (coefT[:g.E] if want_T else None)
 
 
 # ------------------------------------------------------------------ unfused primitives
