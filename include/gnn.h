@@ -431,12 +431,46 @@ size_t gnn_linear_workspace(int32_t N, int K, int M);
 gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype, void* Y,
                       void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* Y = act(X * W + bias): gnn_linear with the element-wise tail of a conv / Dense layer in the training
+ * example (bias float [M] or NULL; relu != 0: max(., 0)) applied to the fp32 accumulator before the single
+ * rounding, inside the epilogue of the product kernel (no extra pass over Y).  Backward:
+ * gnn_row_epilogue_backward(Y, dY, ...) gives dZ and dbias, then gnn_linear_backward on dZ. */
+gnn_status gnn_linear_bias_act(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype,
+                               const float* bias, int relu, void* Y, void* ws, size_t ws_bytes,
+                               gnn_stream stream);
+
 /* dX = dY * W^T ([N,K]) and dW = X^T * dY ([K,M], of dtype); either output may be NULL.  dW sums
  * over the N rows in fixed slabs (one per thread block) whose fp32 partials are added in a
  * fixed order, so the result is reproducible.  X is needed only for dW, W only for dX. */
 gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int32_t N, int K, int M,
                                gnn_dtype dtype, void* dX, void* dW, void* ws, size_t ws_bytes,
                                gnn_stream stream);
+
+/* ------------------------------------------------------------------ aggregate -> transform fusion */
+
+/* Y = act( (op over p in row i of w[p] * X[col[p],:]) * W + bias ): the fused propagate followed by the
+ * weight of a conv layer (Sec. 3 "Message Passing": operations fused "for efficiency"; the GCNConv of
+ * the training example) in ONE kernel.  The aggregated [N,K] matrix is never written: a thread block
+ * reduces 128 target rows into a shared-memory operand tile (bf16; fp32 input is split exactly into
+ * three bf16 terms, which keeps fp32 accuracy) that the tensor cores multiply with the resident W.
+ * msg COPY_XJ / E_MUL_XJ (w_csr float [E], CSR order); op SUM or MEAN; X [N,K], W [K,M], Y [N,M] of
+ * dtype; bias float [M] or NULL.  Fused for K, M multiples of 16 up to 256 with K*sizeof(element) <= 512
+ * and W small enough for shared memory (bf16: up to 256 x 256; fp32: up to 128 x 128); other shapes run
+ * aggregate and transform one after the other through the workspace, with the same results.
+ * For bf16 the aggregated row is rounded to bf16 once before the product, as the unfused sequence does
+ * when it stores it.  ws: gnn_propagate_linear_workspace(N, E, K, M) bytes; its first 4 bytes are the
+ * status word of the tensor-core kernels (see gnn_linear).
+ * Backward for dL/dY = dY [N,M] (run gnn_row_epilogue_backward first if bias / relu were used):
+ *   dX = (A^T dY) * W^T, dW = X^T * (A^T dY), A the weighted adjacency of the forward call.
+ * With dW == NULL the same fused kernel runs on the transposed form; with dW the transposed aggregate
+ * is needed in memory anyway and goes through the workspace.  w_csrT: transposed-CSR order. */
+size_t gnn_propagate_linear_workspace(int32_t N, int64_t E, int K, int M);
+gnn_status gnn_propagate_linear(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* X, const float* w_csr,
+                                const void* W, int K, int M, gnn_dtype dtype, const float* bias, int relu,
+                                void* Y, void* ws, size_t ws_bytes, gnn_stream stream);
+gnn_status gnn_propagate_linear_backward(const gnn_csr* g, gnn_msg msg, gnn_op op, const void* dY, const void* X,
+                                         const float* w_csrT, const void* W, int K, int M, gnn_dtype dtype,
+                                         void* dX, void* dW, void* ws, size_t ws_bytes, gnn_stream stream);
 
 /* Host-buffer variants for callers whose features live in host memory (one call = copy in,
  * compute, copy out; no counterpart in the paper beyond its "transfer the batch to the gpu"

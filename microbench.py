@@ -1,6 +1,6 @@
 """Device times of single library calls on the four smaller synthetic workloads.
 
-    python microbench.py [linear] [config1] [config2] [config3] [config4] [large] [--plain] [--flush]
+    python microbench.py [linear] [fused] [config1] [config2] [config3] [config4] [large] [--plain] [--flush]
 
 Each call is captured 20 times into one CUDA graph; the reported time is the replay time divided by 20
 (CUDA events on the capturing stream), so launch gaps of the Python binding are not in it and the inputs
@@ -179,7 +179,40 @@ def large_calls():
     return calls
 
 
-TABLE = {"linear": linear_calls, "config1": config1_calls, "config2": config2_calls, "config3": config3_calls,
+def fused_calls():
+    """Aggregate -> transform: the fused call beside the two calls it replaces (configs 1, 3 and 4 shapes)."""
+    lib = gnn.load()
+    calls = []
+    cases = []
+    wl = synth.workload_gcn_small()
+    src, dst = synth.with_self_loops(wl["N"], wl["src"], wl["dst"])
+    cases.append(("config 1 GCN 64x64 f32", wl["N"], src, dst, to_dev(wl["X"]), 64, True))
+    for dtype in ("bf16", "f32"):
+        wl = synth.workload_powerlaw(dtype=dtype)
+        cases.append((f"config 3 128x128 {dtype}", wl["N"], wl["src"], wl["dst"], to_dev(wl["X"]), 128, False))
+    wl = synth.workload_attention()
+    cases.append(("config 4 graph 256x256 bf16", wl["N"], wl["src"], wl["dst"], to_dev(wl["Wx"]), 256, False))
+    for tag, n, src, dst, X, M, gcn in cases:
+        g = gnn.coo_to_csr(n, to_dev(src), to_dev(dst))
+        K = X.shape[1]
+        gen = torch.Generator(device="cuda").manual_seed(K + M)
+        W = (torch.randn(K, M, device="cuda", generator=gen) * (2.0 / (K + M)) ** 0.5).to(X.dtype)
+        w = gnn.gcn_norm(g)[1] if gcn else None
+        op = "sum" if gcn else "mean"
+        wsf = torch.empty(lib.gnn_propagate_linear_workspace(n, g.E, K, M), dtype=torch.uint8, device="cuda")
+        wsp = torch.empty(gnn.propagate_fused_workspace(g.E, K, op), dtype=torch.uint8, device="cuda")
+        wsl = torch.empty(lib.gnn_linear_workspace(n, K, M), dtype=torch.uint8, device="cuda")
+        H = torch.empty_like(X)
+        calls.append((f"{tag} (N={n}, E={g.E}) FUSED propagate+linear", lambda g=g, X=X, W=W, w=w, op=op, wsf=wsf: gnn.propagate_linear(g, X, W, w_csr=w, op=op, ws=wsf), None))
+        calls.append((f"{tag} propagate, then linear (two calls)",
+                      lambda g=g, X=X, W=W, w=w, op=op, H=H, wsp=wsp, wsl=wsl: gnn.linear(gnn.propagate_fused(g, X, w, op, out=H, ws=wsp), W, ws=wsl), None))
+        dY = torch.randn(n, M, device="cuda", generator=gen).to(X.dtype)
+        calls.append((f"{tag} FUSED backward dX", lambda g=g, X=X, W=W, w=w, op=op, dY=dY, wsf=wsf: gnn.propagate_linear_backward(g, dY, X, W, w_csrT=w, op=op, want_dW=False, ws=wsf), None))
+        calls.append((f"{tag} backward dX + dW", lambda g=g, X=X, W=W, w=w, op=op, dY=dY, wsf=wsf: gnn.propagate_linear_backward(g, dY, X, W, w_csrT=w, op=op, ws=wsf), None))
+    return calls
+
+
+TABLE = {"linear": linear_calls, "fused": fused_calls, "config1": config1_calls, "config2": config2_calls, "config3": config3_calls,
          "config4": config4_calls, "large": large_calls,
          # older names: the propagate calls of configs 1-3 together, the attention calls of config 4
          "propagate": lambda: config1_calls() + config2_calls() + config3_calls(), "gat": config4_calls}

@@ -30,7 +30,7 @@ template <typename TA, typename TB, typename TC>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* __restrict__ B, int64_t sbk,
                  int64_t sbn, TC* __restrict__ C, int64_t Mr, int64_t Nc, int64_t Kd, int64_t k_per_slab,
-                 int64_t slab_stride) {
+                 int64_t slab_stride, const float* __restrict__ bias, int relu) {
     __shared__ float As[SG_K][SG_TILE + 1];
     __shared__ float Bs[SG_K][SG_TILE + 1];
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
@@ -77,7 +77,12 @@ gemm_simt_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* _
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int64_t n = n0 + tx * 4 + j;
-            if (n < Nc) Cz[m * Nc + n] = from_f32<TC>(acc[i][j]);
+            if (n < Nc) {
+                float y = acc[i][j];
+                if (bias) y += bias[n];  // the element-wise tail of a layer, before the single rounding
+                if (relu) y = fmaxf(y, 0.f);
+                Cz[m * Nc + n] = from_f32<TC>(y);
+            }
         }
     }
 }
@@ -110,9 +115,9 @@ slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __rest
 template <typename TA, typename TB, typename TC>
 static void launch_simt(const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbk, int64_t sbn, TC* C,
                         int64_t Mr, int64_t Nc, int64_t Kd, int64_t k_per_slab, int slabs, int64_t slab_stride,
-                        cudaStream_t st) {
+                        cudaStream_t st, const float* bias = nullptr, int relu = 0) {
     dim3 grid((unsigned)ceil_div(Nc, SG_TILE), (unsigned)ceil_div(Mr, SG_TILE), (unsigned)slabs);
-    gemm_simt_kernel<TA, TB, TC><<<grid, 256, 0, st>>>(A, sam, sak, B, sbk, sbn, C, Mr, Nc, Kd, k_per_slab, slab_stride);
+    gemm_simt_kernel<TA, TB, TC><<<grid, 256, 0, st>>>(A, sam, sak, B, sbk, sbn, C, Mr, Nc, Kd, k_per_slab, slab_stride, bias, relu);
 }
 
 // FFMA dW: rows of X / dY per partial.  128 rows while that gives at most 148 partials (small inputs
@@ -125,10 +130,10 @@ gnn_status linear_tc_forward(const void* X, const void* W, int64_t N, int K, int
                              void* Y, int* d_flag, cudaStream_t st);
 bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype);
 gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
-                              cudaStream_t st);
+                              cudaStream_t st, const float* bias = nullptr, int relu = 0);
 bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype);
 gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
-                                  cudaStream_t st);
+                                  cudaStream_t st, const float* bias = nullptr, int relu = 0);
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tma_dw_partials(int64_t N);
 gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
@@ -151,6 +156,12 @@ size_t gnn_linear_workspace(int32_t N, int K, int M) {
 
 gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype, void* Y,
                       void* ws, size_t ws_bytes, gnn_stream stream) {
+    return gnn_linear_bias_act(X, W, N, K, M, dtype, nullptr, 0, Y, ws, ws_bytes, stream);
+}
+
+gnn_status gnn_linear_bias_act(const void* X, const void* W, int32_t N, int K, int M, gnn_dtype dtype,
+                               const float* bias, int relu, void* Y, void* ws, size_t ws_bytes,
+                               gnn_stream stream) {
     const char* who = "gnn_linear";
     GNN_REQUIRE(N >= 0 && K > 0 && M > 0, GNN_ERR_INVALID_ARG, "%s: bad shape", who);
     GNN_REQUIRE(dtype == GNN_F32 || dtype == GNN_BF16, GNN_ERR_INVALID_ARG, "%s: bad dtype", who);
@@ -159,14 +170,17 @@ gnn_status gnn_linear(const void* X, const void* W, int32_t N, int K, int M, gnn
     GNN_REQUIRE(ws && ws_bytes >= 256, GNN_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes needed", who, gnn_linear_workspace(N, K, M));
     cudaStream_t st = as_stream(stream);
     if (cudaMemsetAsync(ws, 0, sizeof(int), st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "%s: memset failed (is ws a device pointer?)", who);
-    if (linear_tma_supported(N, K, M, 0, dtype)) return linear_tma_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
-    if (linear_tma_f32_supported(N, K, M, dtype)) return linear_tma_f32_forward(X, W, N, K, M, 0, Y, (int*)ws, st);
-    if (linear_tc_supported(N, K, M, dtype)) return linear_tc_forward(X, W, N, K, M, 0, dtype, Y, (int*)ws, st);
-    if (dtype == GNN_F32)
-        launch_simt<float, float, float>((const float*)X, K, 1, (const float*)W, M, 1, (float*)Y, N, M, K, K, 1, 0, st);
-    else
+    if (linear_tma_supported(N, K, M, 0, dtype)) return linear_tma_forward(X, W, N, K, M, 0, Y, (int*)ws, st, bias, relu);
+    if (linear_tma_f32_supported(N, K, M, dtype)) return linear_tma_f32_forward(X, W, N, K, M, 0, Y, (int*)ws, st, bias, relu);
+    // fp32 with weights too large for the pipelined kernel runs the single-buffered tensor-core kernel; with a
+    // bias or relu it takes the FFMA kernel instead, whose epilogue applies them before the single rounding
+    if (!bias && !relu && linear_tc_supported(N, K, M, dtype)) return linear_tc_forward(X, W, N, K, M, 0, dtype, Y, (int*)ws, st);
+    if (dtype == GNN_F32) {
+        launch_simt<float, float, float>((const float*)X, K, 1, (const float*)W, M, 1, (float*)Y, N, M, K, K, 1, 0, st, bias, relu);
+    } else {
         launch_simt<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>((const __nv_bfloat16*)X, K, 1, (const __nv_bfloat16*)W, M, 1,
-                                                               (__nv_bfloat16*)Y, N, M, K, K, 1, 0, st);
+                                                               (__nv_bfloat16*)Y, N, M, K, K, 1, 0, st, bias, relu);
+    }
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }

@@ -52,6 +52,8 @@ struct TmaParams {
     int acc_stride;    // tensor-memory columns between the two accumulators
     int tmem_cols;
     int* status;
+    const float* bias;  // [Mo] added to every output row, or nullptr
+    int relu;           // max(y, 0) after the bias
 };
 
 __global__ void __launch_bounds__(TM_THREADS, 1)
@@ -169,7 +171,11 @@ linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     tmem_ld_wait();
                     float f[16];
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) f[q] = __uint_as_float(r[q]);
+                    for (int q = 0; q < 16; ++q) {
+                        f[q] = __uint_as_float(r[q]);
+                        if (P.bias) f[q] += __ldg(P.bias + cb * 64 + g * 16 + q);
+                        if (P.relu) f[q] = fmaxf(f[q], 0.f);
+                    }
                     // row = lane, 128 bytes per row; 16-byte chunk c sits at position c ^ (row % 8)
 #pragma unroll
                     for (int h2 = 0; h2 < 2; ++h2) {
@@ -219,7 +225,9 @@ static EncodeTiledFn encoder() {
 }
 
 // row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes, swizzled) x box_rows rows; out-of-range reads give zeros
-static bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+bool tensor_map_encoder_available() { return encoder() != nullptr; }
+
+bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
     EncodeTiledFn enc = encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -242,7 +250,7 @@ bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype
 }
 
 gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
-                              cudaStream_t st) {
+                              cudaStream_t st, const float* bias, int relu) {
     const char* who = "gnn_linear (pipelined tensor-core path)";
     GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
     CUtensorMap mapX, mapW, mapY;
@@ -251,7 +259,7 @@ gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, i
         !make_map(&mapY, Y, N, Mo, 32))
         GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaParams P;
-    P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
+    P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag; P.bias = bias; P.relu = relu;
     const size_t wbytes = tma_w_bytes(Kc, Mo, b_transposed);
     const size_t fixed = 1024 + wbytes + (size_t)TM_EPI_WARPS * TM_STAGING_BYTES;
     int stages = (int)((TM_SMEM_MAX - fixed) / TM_SLICE_BYTES);
@@ -326,6 +334,8 @@ struct TmaF32Params {
     int stages;
     int acc_stride, tmem_cols;
     int* status;
+    const float* bias;  // [Mo] added to every output row, or nullptr
+    int relu;           // max(y, 0) after the bias
 };
 
 __global__ void __launch_bounds__(TF_THREADS, 1)
@@ -485,6 +495,15 @@ linear_tma_f32_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
                     uint32_t r[16];
                     tmem_ld16(taddr + (uint32_t)(cb * 32 + g16 * 16), r);
                     tmem_ld_wait();
+                    if (P.bias || P.relu) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            float y = __uint_as_float(r[q]);
+                            if (P.bias) y += __ldg(P.bias + cb * 32 + g16 * 16 + q);
+                            if (P.relu) y = fmaxf(y, 0.f);
+                            r[q] = __float_as_uint(y);
+                        }
+                    }
                     // row = lane, 128 bytes per row; 16-byte chunk c sits at position c ^ (row % 8)
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
@@ -658,7 +677,7 @@ int linear_tma_dw_partials(int64_t N) {
     return (int)(nchunks < 148 ? (nchunks > 0 ? nchunks : 1) : 148);
 }
 
-static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows);
+bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows);
 
 // writes linear_tma_dw_partials(N) fp32 partials [K,M] to part
 gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
@@ -684,7 +703,7 @@ gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M,
 }
 
 // row-major fp32 matrix [rows, cols]; box = 32 columns (128 bytes, swizzled) x box_rows rows
-static bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
     EncodeTiledFn enc = encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -707,13 +726,13 @@ bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype) {
 }
 
 gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, const float* bias, int relu) {
     const char* who = "gnn_linear (pipelined fp32 tensor-core path)";
     GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
     CUtensorMap mapX, mapY;
     if (!make_map_f32(&mapX, X, N, Kc, TC_ROWS) || !make_map_f32(&mapY, Y, N, Mo, 32)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaF32Params P;
-    P.W = (const float*)W; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag;
+    P.W = (const float*)W; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag; P.bias = bias; P.relu = relu;
     const size_t fixed = tf_fixed_bytes(Kc, Mo);
     int stages = (int)((TM_SMEM_MAX - fixed) / TF_SLICE_BYTES);
     P.stages = stages > TF_MAX_STAGES ? TF_MAX_STAGES : stages;

@@ -103,7 +103,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // raise a kernel's dynamic shared memory limit, once per (device, kernel slot)
 inline gnn_status allow_big_smem(const char* who, const void* kernel, int which, size_t bytes = TC_SMEM_LIMIT) {
-    static std::atomic<unsigned char> done[64][8];
+    static std::atomic<unsigned char> done[64][16];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
     if (dev >= 0 && done[dev][which].load()) return GNN_OK;

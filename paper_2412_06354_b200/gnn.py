@@ -92,6 +92,10 @@ SIGNATURES = {
     "gnn_reduce_nodes_backward": (_INT, [_VP, _I32, _I32, _INT, _VP, _VP, _INT, _INT, _VP, _VP]),
     "gnn_linear_workspace": (_SZ, [_I32, _INT, _INT]),
     "gnn_linear": (_INT, [_VP, _VP, _I32, _INT, _INT, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_linear_bias_act": (_INT, [_VP, _VP, _I32, _INT, _INT, _INT, _VP, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_linear_workspace": (_SZ, [_I32, _I64, _INT, _INT]),
+    "gnn_propagate_linear": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _INT, _VP, _INT, _VP, _VP, _SZ, _VP]),
+    "gnn_propagate_linear_backward": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _VP, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_linear_backward": (_INT, [_VP, _VP, _VP, _I32, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_propagate_fused_backward_host": (_INT, [_CSR, _INT, _INT, _VP, _VP, _VP, _INT, _INT, _VP, _VP, _VP, _VP, _SZ, _VP]),
@@ -571,6 +575,44 @@ def linear(X, W, ws=None, return_ws=False):
         ws = torch.empty(load().gnn_linear_workspace(N, K, M), dtype=torch.uint8, device=X.device)
     _check(load().gnn_linear(_p(X), _p(W), N, K, M, _dtype(X), _p(Y), _p(ws), ws.numel(), _stream()))
     return (Y, ws) if return_ws else Y
+
+
+def linear_bias_act(X, W, bias=None, relu=False, ws=None):
+    """Y = act(X W + bias) with the tail inside the product kernel's epilogue."""
+    X, W = _dev(X), _dev(W)
+    (N, K), M = X.shape, W.shape[1]
+    Y = torch.empty((N, M), dtype=X.dtype, device=X.device)
+    if ws is None:
+        ws = torch.empty(load().gnn_linear_workspace(N, K, M), dtype=torch.uint8, device=X.device)
+    _check(load().gnn_linear_bias_act(_p(X), _p(W), N, K, M, _dtype(X), _pf32(bias, "bias"), int(bool(relu)), _p(Y), _p(ws), ws.numel(), _stream()))
+    return Y
+
+
+def propagate_linear(g: Graph, X, W, w_csr=None, op="sum", bias=None, relu=False, ws=None, return_ws=False):
+    """Y = act((op over incoming edges of w * X[source]) W + bias) in one kernel."""
+    X, W = _dev(X), _dev(W)
+    K, M = W.shape
+    Y = torch.empty((g.N, M), dtype=X.dtype, device=X.device)
+    if ws is None:
+        ws = torch.empty(load().gnn_propagate_linear_workspace(g.N, g.E, K, M), dtype=torch.uint8, device=X.device)
+    msg = COPY_XJ if w_csr is None else E_MUL_XJ
+    _check(load().gnn_propagate_linear(g.ref, msg, _op(op), _p(X), _pf32(w_csr, "w_csr"), _p(W), K, M, _dtype(X), _pf32(bias, "bias"),
+                                       int(bool(relu)), _p(Y), _p(ws), ws.numel(), _stream()))
+    return (Y, ws) if return_ws else Y
+
+
+def propagate_linear_backward(g: Graph, dY, X, W, w_csrT=None, op="sum", want_dX=True, want_dW=True, ws=None):
+    """-> (dX or None, dW or None)"""
+    dY, W = _dev(dY), _dev(W)
+    K, M = W.shape
+    dX = torch.empty((g.N, K), dtype=dY.dtype, device=dY.device) if want_dX else None
+    dW = torch.empty((K, M), dtype=dY.dtype, device=dY.device) if want_dW else None
+    if ws is None:
+        ws = torch.empty(load().gnn_propagate_linear_workspace(g.N, g.E, K, M), dtype=torch.uint8, device=dY.device)
+    msg = COPY_XJ if w_csrT is None else E_MUL_XJ
+    _check(load().gnn_propagate_linear_backward(g.ref, msg, _op(op), _p(dY), _p(X), _pf32(w_csrT, "w_csrT"), _p(W), K, M, _dtype(dY),
+                                                _p(dX), _p(dW), _p(ws), ws.numel(), _stream()))
+    return dX, dW
 
 
 def linear_backward(X, W, dY, want_dX=True, want_dW=True, ws=None, return_ws=False):
