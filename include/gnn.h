@@ -135,7 +135,9 @@ gnn_status gnn_permute_edge_data(const int32_t* perm, int64_t E, int width, int 
  * scalar per edge, CSR order).  op: SUM; MEAN (sum divided by the number of incoming edges);
  * MAX / MIN (element-wise; argmax int32 [N,F] receives the CSR position of the winner, the
  * smallest position among equal values; may be NULL).  A node with no incoming edge gets 0 and
- * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes.
+ * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes, asked for the E of
+ * this very call: the edges-per-chunk of the reduction steps with the graph size, so the size is not
+ * monotone in E and a workspace sized for a larger graph can be too small for a smaller one.
  * Bytes moved per call: at least 4E (+4E with weights) + 8N + 2*N*F*s, at most
  * 4E (+4E) + 8N + (E+N)*F*s when no source row is found in L2. */
 size_t gnn_propagate_fused_workspace(int64_t E, int F, gnn_op op);
@@ -153,8 +155,8 @@ gnn_status gnn_propagate_fused(const gnn_csr* g, gnn_msg msg, gnn_op op, const v
  * GPU that loads the library holds those 8 MiB until the process exits.
  *  - Same arguments and results as gnn_propagate_fused, minus ws / ws_bytes.  No cudaMalloc, cudaFree
  *    or other allocating routine is called.
- *  - Size limit: gnn_propagate_fused_workspace(E, F, op) must not exceed the 8 MiB (about 2 M edges
- *    at F = 128 for SUM/MEAN, half that for MAX/MIN); larger problems are rejected with
+ *  - Size limit: gnn_propagate_fused_workspace(E, F, op) must not exceed the 8 MiB (ask that function:
+ *    the size is not monotone in E); larger problems are rejected with
  *    GNN_ERR_WORKSPACE_TOO_SMALL and a message, before anything is launched.
  *  - The first call on each device looks up the device address of the array (with that device
  *    current) and caches it; make that first call outside any stream capture.

@@ -31,9 +31,6 @@
 #ifndef PF_MIN_BLOCKS
 #define PF_MIN_BLOCKS 4
 #endif
-#ifndef PF_WIDE_FLAT
-#define PF_WIDE_FLAT 0
-#endif
 
 namespace gnn {
 
@@ -505,161 +502,6 @@ propagate_chunk_kernel(const PropParams P) {
     scan_empty_rows(P.rowptr, P.N, c, P.nchunks, lane, [&](int r) {
         acc.clear();
         W::write_final(P, r, 0, lane, acc);
-    });
-}
-
-// ------------------------------------------------------------------ full-warp rows: gathers batched across rows
-// Sum / mean over rows that fill a warp (17..32 16-byte chunks: one lane group, nothing to combine) on the
-// large graphs.  Walking such rows one at a time issues the gathers of a short row (most rows of a power-law
-// graph hold a handful of edges) one by one, each paying the full memory latency.  Here the row structure is
-// staged with the indices: while a slab of 256 positions is staged, the rows that start inside it are marked
-// (row id and scale factor stored with their first position), and the inner loop then issues U independent
-// row gathers for U consecutive positions whatever rows they belong to, and closes a row whenever it meets a
-// start mark.  The additions of a row happen in ascending position order as in the row-walking kernel, rows cut
-// by the chunk leave the same head / tail partials, and the same fix-up pass finishes them.
-template <typename T>
-__global__ void __launch_bounds__(PF_WARPS * 32, PF_MIN_BLOCKS)
-propagate_wide_kernel(const PropParams P) {
-    constexpr int EPC = Chunk<T>::N, U = PF_U_WIDE;
-    __shared__ SlabSmem s_slab[PF_WARPS];
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + wib;
-    if (c >= P.nchunks) return;
-    SlabSmem& S = s_slab[wib];
-    const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
-    const int64_t cs = c * P.chunk;
-    const int64_t ce = (cs + P.chunk < P.E) ? cs + P.chunk : P.E;
-    const bool col_lane = lane < P.nvec;  // lanes past a ragged row width gather chunk 0 and never store
-    const char* const Xl = reinterpret_cast<const char*>(P.X) + (size_t)(col_lane ? lane : 0) * 16;
-    char* const outb = reinterpret_cast<char*>(P.out);
-
-    // the row holding position cs: largest r with rowptr[r] <= cs (32-way search)
-    int lo = 0, hi = P.N;
-    while (hi - lo > 1) {
-        const int step = (hi - lo + 31) / 32;
-        const int idx = min(lo + (lane + 1) * step, hi);
-        const bool le = idx < hi && P.rowptr[idx] <= cs;
-        const int k = __popc(__ballot_sync(0xffffffffu, le));
-        const int nlo = lo + k * step;
-        hi = min(nlo + step, hi);
-        lo = nlo;
-    }
-    auto row_factor = [&](int64_t len) { return P.mean ? 1.0f / (float)(len > 1 ? len : 1) : 1.0f; };
-    int row = lo;
-    bool began_before;
-    float rinv;
-    {
-        const int64_t rs = P.rowptr[row], re = P.rowptr[row + 1];
-        began_before = rs < cs;
-        rinv = row_factor(re - rs);
-    }
-    float acc[EPC];
-#pragma unroll
-    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-
-    auto write_partial = [&](int which) {
-        if (!col_lane) return;
-        float* pv = P.part_val + ((size_t)c * 2 + which) * P.F + (size_t)lane * EPC;
-#pragma unroll
-        for (int j = 0; j < EPC; j += 4) *reinterpret_cast<float4*>(pv + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-    };
-    auto write_row = [&](int r, float f) {
-        if (!col_lane) return;
-        float v[EPC];
-#pragma unroll
-        for (int j = 0; j < EPC; ++j) v[j] = acc[j] * f;
-        row_epilogue<T>(P, r, lane, v);
-        st_stream16(outb + (size_t)r * P.out_ld + (size_t)lane * 16, Chunk<T>::pack(v));
-    };
-    // the current row has ended inside the chunk
-    auto close_row = [&]() {
-        if (began_before) write_partial(0);
-        else write_row(row, rinv);
-    };
-
-    int scan = row + 1;  // first row whose start has not been looked at yet
-    for (int64_t sb = cs; sb < ce; sb += PF_SLAB) {
-        const int64_t se = (sb + PF_SLAB < ce) ? sb + PF_SLAB : ce;
-        const int n = (int)(se - sb);
-        __syncwarp();
-        for (int i = lane; i < n; i += 32) {
-            const int cc = P.col ? ld_hint_i32(P.col + sb + i, pol_stream) : (int)(sb + i);
-            float w = P.w ? ld_hint_f32(P.w + sb + i, pol_stream) : 1.0f;
-            if (P.gscale_rowptr) {
-                const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
-                w = w / (float)(d > 1 ? d : 1);
-            }
-            S.e[i] = make_int4(cc, -1, __float_as_int(w), 0);
-        }
-        __syncwarp();
-        // rows that start inside this slab and have edges: mark their first position
-        for (int rb = scan; rb < P.N;) {
-            const int r = rb + lane;
-            int64_t rs = 0, re = 0;
-            bool live = false;
-            if (r < P.N) {
-                rs = P.rowptr[r];
-                live = rs < se;
-                if (live) re = P.rowptr[r + 1];
-            }
-            if (live && re > rs) {
-                const int k = (int)(rs - sb);
-                S.e[k].y = r;
-                S.e[k].w = __float_as_int(row_factor(re - rs));
-            }
-            const unsigned lm = __ballot_sync(0xffffffffu, live);
-            if (lm != 0xffffffffu) { scan = rb + __popc(lm); break; }  // rowptr ascends: the live lanes are a prefix
-            if (__all_sync(0xffffffffu, re == rs)) rb = first_row_ending_after(P.rowptr, rb + 32, P.N, __shfl_sync(0xffffffffu, rs, 0), lane);
-            else rb += 32;
-            scan = rb;
-        }
-        __syncwarp();
-        for (int i = 0; i < n; i += U) {
-            uint4 buf[U];
-            if (i + U <= n) {
-                int cols[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) cols[u] = S.e[i + u].x;
-#pragma unroll
-                for (int u = 0; u < U; ++u) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * P.x_ld, pol_keep);
-            } else {
-#pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (i + u < n) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)S.e[i + u].x * P.x_ld, pol_keep);
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (i + u >= n) break;
-                const int4 e = S.e[i + u];
-                if (e.y >= 0) {  // a row starts here: the one before it is complete
-                    close_row();
-                    row = e.y;
-                    rinv = __int_as_float(e.w);
-                    began_before = false;
-#pragma unroll
-                    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-                }
-                float x[EPC];
-                Chunk<T>::unpack(buf[u], x);
-                const float w = __int_as_float(e.z);
-#pragma unroll
-                for (int j = 0; j < EPC; j += 2) fma2(acc[j], acc[j + 1], x[j], x[j + 1], w, w);
-            }
-        }
-    }
-    // the row that is open at the end of the chunk
-    int32_t tail = -1;
-    if (P.rowptr[row + 1] <= ce) {
-        close_row();
-    } else {
-        write_partial(began_before ? 0 : 1);
-        if (!began_before) tail = row;
-    }
-    if (lane == 0) P.tail_row[c] = tail;
-    scan_empty_rows(P.rowptr, P.N, c, P.nchunks, lane, [&](int r) {
-#pragma unroll
-        for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-        write_row(r, 1.0f);
     });
 }
 
@@ -1410,12 +1252,6 @@ template <typename T, int MODE>
 static void launch_chunks(const PropParams& P, int lpr, int vpl, cudaStream_t st) {
     const int grid = (int)ceil_div(P.nchunks, PF_WARPS);
     const int thr = PF_WARPS * 32;
-    if (MODE == MODE_SUM && lpr == 32 && vpl == 1 && PF_WIDE_FLAT) {  // full-warp rows: gathers batched across rows
-        propagate_wide_kernel<T><<<grid, thr, 0, st>>>(P);
-        const int64_t threads = P.nchunks * P.nvec;
-        propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
-        return;
-    }
 #define GNN_PF_CASE(L, V) \
     if (lpr == L && vpl == V) { propagate_chunk_kernel<T, L, V, MODE><<<grid, thr, 0, st>>>(P); }
     GNN_PF_CASE(4, 1) GNN_PF_CASE(8, 1) GNN_PF_CASE(16, 1) GNN_PF_CASE(32, 1) GNN_PF_CASE(32, 2) GNN_PF_CASE(32, 4)

@@ -26,16 +26,19 @@ bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_r
 bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows);  // fp32, 32-column boxes
 bool tensor_map_encoder_available();
 
-constexpr int PL_GATHER_WARPS = 16;
+#ifndef PL_GATHER_WARPS_N
+#define PL_GATHER_WARPS_N 11
+#endif
+constexpr int PL_GATHER_WARPS = PL_GATHER_WARPS_N;
 constexpr int PL_EPI_WARPS = 4;
 constexpr int PL_THREADS = 32 * (1 + PL_EPI_WARPS + PL_GATHER_WARPS);
 constexpr int PL_U = 8;              // row gathers a lane group keeps in flight
-constexpr int PL_GRAB = 2;           // rows a lane group takes from the tile's counter at a time
 constexpr int PL_LONG = 1024;        // rows longer than this are split over PL_LONG_WARPS warps
 constexpr int PL_LONG_WARPS = 8;
-constexpr int PL_MAX_STAGES = 4;
+constexpr int PL_WINDOW = 2048;      // positions of a tile whose indices (and multipliers) are staged in shared memory
+constexpr int PL_MAX_STAGES = 2;
 constexpr uint32_t PL_SLICE_BYTES = TC_ROWS * 128;  // 64 bf16 columns of the 128-row operand tile
-constexpr size_t PL_SMEM_MAX = 220 * 1024;  // dynamic shared memory per CTA (227 KB less the static part)
+constexpr size_t PL_SMEM_MAX = 222 * 1024;  // dynamic shared memory per CTA (227 KB less the static part)
 constexpr uint32_t PL_SW128 = 2;
 
 __device__ __constant__ unsigned char kPlPairA[6] = {2, 0, 1, 1, 0, 0};  // levels of A and B per product, small terms first
@@ -55,6 +58,7 @@ struct PlParams {
     int mean;
     int b_transposed;
     int stages;
+    int window;         // positions of a tile whose indices and multipliers are staged in shared memory (per stage)
     int acc_stride, tmem_cols;
     int* status;
 };
@@ -105,9 +109,130 @@ struct PlStageCtl {
     int rp[TC_ROWS + 1];         // row pointers of the tile's rows (clamped past the last row); E < 2^31
 };
 
-template <typename T>
+// Phase 1 of a tile for one lane group: row r of the tile, at most PL_LONG positions, PL_U gathers in flight.
+// Out of line so that the registers of this loop are not shared with the rest of the kernel (a spilled
+// register here costs a trip to L2: the kernel's shared memory leaves the L1 almost no room).
+template <typename T, bool WEIGHTED>
+__device__ __noinline__ void pl_take_row(const PlParams& P, int rs, int len, int r, uint32_t stage, uint32_t level_bytes,
+                                         const char* Xl, uint32_t row_bytes, int li, bool col_lane, uint64_t pol_keep,
+                                         const int* scol, const float* sw) {
+    constexpr int EPC = Chunk<T>::N;
+    float acc[EPC];
+#pragma unroll
+    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+    const int32_t* const colp = P.col + rs;
+    if (scol) {  // the row lies inside the staged window: indices and multipliers come from shared memory
+        for (int q0 = 0; q0 < len; q0 += PL_U) {
+            uint4 buf[PL_U];
+#pragma unroll
+            for (int u = 0; u < PL_U; ++u)
+                if (q0 + u < len) buf[u] = ld_hint16(Xl + (size_t)(uint32_t)scol[q0 + u] * row_bytes, pol_keep);
+#pragma unroll
+            for (int u = 0; u < PL_U; ++u) {
+                if (q0 + u >= len) break;
+                float x[EPC];
+                Chunk<T>::unpack(buf[u], x);
+                const float wq = WEIGHTED ? sw[q0 + u] : 1.0f;
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) acc[j] = WEIGHTED ? fmaf(wq, x[j], acc[j]) : acc[j] + x[j];
+            }
+        }
+    } else
+    for (int q0 = 0; q0 < len; q0 += PL_U) {
+        int cols[PL_U];
+        uint4 buf[PL_U];
+        float wv[WEIGHTED ? PL_U : 1];
+#pragma unroll
+        for (int u = 0; u < PL_U; ++u) cols[u] = q0 + u < len ? __ldg(colp + q0 + u) : 0;
+#pragma unroll
+        for (int u = 0; u < PL_U; ++u)
+            if (q0 + u < len) {
+                buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * row_bytes, pol_keep);
+                if (WEIGHTED) {
+                    float wq = P.w ? __ldg(P.w + rs + q0 + u) : 1.0f;
+                    if (P.gscale_rowptr) {
+                        const int64_t d = P.gscale_rowptr[cols[u] + 1] - P.gscale_rowptr[cols[u]];
+                        wq = wq / (float)(d > 1 ? d : 1);
+                    }
+                    wv[WEIGHTED ? u : 0] = wq;
+                }
+            }
+#pragma unroll
+        for (int u = 0; u < PL_U; ++u) {
+            if (q0 + u >= len) break;
+            float x[EPC];
+            Chunk<T>::unpack(buf[u], x);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) acc[j] = WEIGHTED ? fmaf(wv[WEIGHTED ? u : 0], x[j], acc[j]) : acc[j] + x[j];
+        }
+    }
+    if (!col_lane) return;
+    if (P.mean) {
+        const float d = (float)(len > 1 ? len : 1);
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) acc[j] = acc[j] / d;
+    }
+    pl_store_row<T>(stage, level_bytes, r, li, acc);
+}
+
+// Phase 2: this warp's share of one long row (positions rs + gw * per ...), lane groups interleaved, combined by
+// a fixed shuffle tree; lanes of group 0 leave the partial sum in part[gw][...]
+template <typename T, bool WEIGHTED>
+__device__ __noinline__ void pl_long_share(const PlParams& P, int rs, int len, int gw, float* part, const char* Xl, uint32_t row_bytes,
+                                           int lane, int lpr, bool col_lane, uint64_t pol_keep) {
+    constexpr int EPC = Chunk<T>::N;
+    const int K = P.K, g = lane / lpr, li = lane % lpr, ng = 32 / lpr, re = rs + len;
+    const int per = (len + PL_LONG_WARPS - 1) / PL_LONG_WARPS;
+    const int pa = rs + gw * per, pb = (pa + per < re) ? pa + per : re;
+    float acc[EPC];
+#pragma unroll
+    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
+    for (int p0 = pa + g; p0 < pb; p0 += ng * PL_U) {
+        uint4 buf[PL_U];
+        float wv[WEIGHTED ? PL_U : 1];
+#pragma unroll
+        for (int u = 0; u < PL_U; ++u) {
+            const int p = p0 + u * ng;
+            if (p < pb) {
+                const int cc = __ldg(P.col + p);
+                buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * row_bytes, pol_keep);
+                if (WEIGHTED) {
+                    float wq = P.w ? __ldg(P.w + p) : 1.0f;
+                    if (P.gscale_rowptr) {
+                        const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
+                        wq = wq / (float)(d > 1 ? d : 1);
+                    }
+                    wv[WEIGHTED ? u : 0] = wq;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < PL_U; ++u) {
+            if (p0 + u * ng >= pb) break;
+            float x[EPC];
+            Chunk<T>::unpack(buf[u], x);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) acc[j] = WEIGHTED ? fmaf(wv[WEIGHTED ? u : 0], x[j], acc[j]) : acc[j] + x[j];
+        }
+    }
+    __syncwarp();
+    for (int o = lpr; o < 32; o <<= 1) {  // combine the lane groups: both partners add in the same operand order
+        const bool low = (lane & o) == 0;
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) {
+            const float ov = __shfl_xor_sync(0xffffffffu, acc[j], o);
+            acc[j] = low ? (acc[j] + ov) : (ov + acc[j]);
+        }
+    }
+    if (lane < lpr && col_lane) {
+#pragma unroll
+        for (int j = 0; j < EPC; ++j) part[(size_t)gw * K + li * EPC + j] = acc[j];
+    }
+}
+
+template <typename T, bool WEIGHTED>
 __global__ void __launch_bounds__(PL_THREADS, 1)
-propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const PlParams P) {
+propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const __grid_constant__ PlParams P) {
     constexpr int EPC = Chunk<T>::N;
     constexpr int LEVELS = sizeof(T) == 2 ? 1 : 3, PAIRS = sizeof(T) == 2 ? 1 : 6;
     extern __shared__ unsigned char smem_raw[];
@@ -124,6 +249,7 @@ propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const PlParams
     const uint32_t a0 = base + (((uint32_t)LEVELS * b_level + 1023u) & ~1023u);
     const uint32_t stg0 = a0 + (uint32_t)S * stage_bytes;                  // per epilogue warp: 32 rows x 128 bytes
     const uint32_t part0 = stg0 + PL_EPI_WARPS * 4096u;                    // PL_LONG_WARPS partial rows of K floats
+    const uint32_t win0 = part0 + (uint32_t)PL_LONG_WARPS * (uint32_t)K * 4u;           // per stage: window ints + window floats
     const uint32_t bar0 = smem_u32(bars);
     auto a_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto a_empty = [&](int s) { return bar0 + 8u * (uint32_t)(PL_MAX_STAGES + s); };
@@ -271,6 +397,8 @@ propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const PlParams
             const int s = (int)(lt % (uint32_t)S);
             PlStageCtl& C = ctl[s];
             const uint32_t stage = a0 + (uint32_t)s * stage_bytes;
+            int* const ecol = reinterpret_cast<int*>(smem_raw + (win0 - smem_u32(smem_raw)) + (size_t)s * P.window * 8);
+            float* const ew = reinterpret_cast<float*>(ecol + P.window);
             // the tensor core has read the previous contents of this stage (first uses: passes at once)
             int ok = 1;
             if (lane == 0) ok = mbar_wait_bounded(a_empty(s), ((lt / (uint32_t)S) & 1u) ^ 1u) ? 1 : 0;
@@ -288,76 +416,38 @@ propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const PlParams
             }
             if (gt == 0) { C.next_row = 0; C.n_long = 0; }
             pl_named_barrier(1, GT);
+            {   // stage the indices (and multipliers, rescaled once) of the tile's first PL_WINDOW positions
+                const int p0 = C.rp[0], nw = min(C.rp[TC_ROWS] - p0, P.window);
+                for (int i = gt; i < nw; i += GT) {
+                    const int cc = __ldg(P.col + p0 + i);
+                    ecol[i] = cc;
+                    if (WEIGHTED) {
+                        float wq = P.w ? __ldg(P.w + p0 + i) : 1.0f;
+                        if (P.gscale_rowptr) {
+                            const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
+                            wq = wq / (float)(d > 1 ? d : 1);
+                        }
+                        ew[i] = wq;
+                    }
+                }
+            }
+            pl_named_barrier(1, GT);
 
-            // ---- phase 1: a lane group takes PL_GRAB rows at a time and keeps PL_U gathers in flight across them
+            // ---- phase 1: a lane group takes one row at a time from the tile's counter
             for (;;) {
-                int r_first = 0;
-                if (li == 0) r_first = atomicAdd(&C.next_row, PL_GRAB);
-                r_first = __shfl_sync(gmask, r_first, g * lpr);
-                if (r_first >= TC_ROWS) break;
-                const int rp0 = C.rp[r_first], rp1 = C.rp[r_first + 1], rp2 = C.rp[r_first + 2 <= TC_ROWS ? r_first + 2 : r_first + 1];
-                const int lenA = rp1 - rp0, lenB = rp2 - rp1;
-                const bool hasB = r_first + 1 < TC_ROWS;
-                const bool longA = lenA > PL_LONG, longB = lenB > PL_LONG;
-                if (li == 0) {
-                    if (longA) C.long_rows[atomicAdd(&C.n_long, 1)] = r_first;
-                    if (longB) C.long_rows[atomicAdd(&C.n_long, 1)] = r_first + 1;
+                int r = 0;
+                if (li == 0) r = atomicAdd(&C.next_row, 1);
+                r = __shfl_sync(gmask, r, g * lpr);
+                if (r >= TC_ROWS) break;
+                const int rs = C.rp[r], len = C.rp[r + 1] - rs;
+                if (len > PL_LONG) {
+                    if (li == 0) C.long_rows[atomicAdd(&C.n_long, 1)] = r;
+                    continue;
                 }
-                const int nA = longA ? 0 : lenA, nB = longB ? 0 : lenB, total = nA + nB;
-                auto pos_of = [&](int q) { return q < nA ? rp0 + q : rp1 + (q - nA); };
-                float acc[EPC];
-#pragma unroll
-                for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-                auto store = [&](int r, int len) {
-                    if (!col_lane) return;
-                    float v[EPC];
-                    const float d = P.mean ? (float)(len > 1 ? len : 1) : 1.0f;
-#pragma unroll
-                    for (int j = 0; j < EPC; ++j) v[j] = P.mean ? acc[j] / d : acc[j];
-                    pl_store_row<T>(stage, level_bytes, r, li, v);
-                };
-                int cols[PL_U];
-#pragma unroll
-                for (int u = 0; u < PL_U; ++u) cols[u] = u < total ? __ldg(P.col + pos_of(u)) : 0;
-                for (int q0 = 0; q0 < total; q0 += PL_U) {
-                    uint4 buf[PL_U];
-                    float wv[PL_U];
-#pragma unroll
-                    for (int u = 0; u < PL_U; ++u)
-                        if (q0 + u < total) {
-                            buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cols[u] * row_bytes, pol_keep);
-                            wv[u] = P.w ? __ldg(P.w + pos_of(q0 + u)) : 1.0f;
-                            if (P.gscale_rowptr) {
-                                const int64_t d = P.gscale_rowptr[cols[u] + 1] - P.gscale_rowptr[cols[u]];
-                                wv[u] = wv[u] / (float)(d > 1 ? d : 1);
-                            }
-                        }
-#pragma unroll
-                    for (int u = 0; u < PL_U; ++u) cols[u] = q0 + PL_U + u < total ? __ldg(P.col + pos_of(q0 + PL_U + u)) : 0;
-#pragma unroll
-                    for (int u = 0; u < PL_U; ++u) {
-                        if (q0 + u >= total) break;
-                        if (q0 + u == nA) {  // the first row is complete (an empty one is written as zeros)
-                            if (!longA) store(r_first, lenA);
-#pragma unroll
-                            for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-                        }
-                        float x[EPC];
-                        Chunk<T>::unpack(buf[u], x);
-#pragma unroll
-                        for (int j = 0; j < EPC; ++j) acc[j] = fmaf(wv[u], x[j], acc[j]);
-                    }
-                }
-                if (nB == 0) {  // acc holds the first row (zeros if it has no edges); the second one has none to add
-                    if (!longA) store(r_first, lenA);
-                    if (hasB && !longB) {
-#pragma unroll
-                        for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-                        store(r_first + 1, lenB);
-                    }
-                } else {
-                    store(r_first + 1, lenB);
-                }
+                const int off = rs - C.rp[0];
+                const bool staged = off + len <= P.window;
+                pl_take_row<T, WEIGHTED>(P, rs, len, r, stage, level_bytes, Xl, row_bytes, li, col_lane, pol_keep,
+                                         staged ? ecol + off : nullptr, staged ? ew + off : nullptr);
             }
             __syncwarp();
             pl_named_barrier(1, GT);
@@ -367,51 +457,9 @@ propagate_linear_kernel(const __grid_constant__ CUtensorMap mapY, const PlParams
             if (nl > 0 && gw < PL_LONG_WARPS) {
                 for (int k = 0; k < nl; ++k) {
                     const int r = C.long_rows[k];
-                    const int rs = C.rp[r], re = C.rp[r + 1], len = re - rs;
-                    const int per = (len + PL_LONG_WARPS - 1) / PL_LONG_WARPS;
-                    const int pa = rs + gw * per, pb = (pa + per < re) ? pa + per : re;
-                    float acc[EPC];
-#pragma unroll
-                    for (int j = 0; j < EPC; ++j) acc[j] = 0.f;
-                    for (int p0 = pa + g; p0 < pb; p0 += ng * PL_U) {
-                        uint4 buf[PL_U];
-                        float wv[PL_U];
-#pragma unroll
-                        for (int u = 0; u < PL_U; ++u) {
-                            const int p = p0 + u * ng;
-                            if (p < pb) {
-                                const int cc = __ldg(P.col + p);
-                                buf[u] = ld_hint16(Xl + (size_t)(uint32_t)cc * row_bytes, pol_keep);
-                                wv[u] = P.w ? __ldg(P.w + p) : 1.0f;
-                                if (P.gscale_rowptr) {
-                                    const int64_t d = P.gscale_rowptr[cc + 1] - P.gscale_rowptr[cc];
-                                    wv[u] = wv[u] / (float)(d > 1 ? d : 1);
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < PL_U; ++u) {
-                            if (p0 + u * ng >= pb) break;
-                            float x[EPC];
-                            Chunk<T>::unpack(buf[u], x);
-#pragma unroll
-                            for (int j = 0; j < EPC; ++j) acc[j] = fmaf(wv[u], x[j], acc[j]);
-                        }
-                    }
-                    __syncwarp();
-                    for (int o = lpr; o < 32; o <<= 1) {  // combine the lane groups: both partners add in the same operand order
-                        const bool low = (lane & o) == 0;
-#pragma unroll
-                        for (int j = 0; j < EPC; ++j) {
-                            const float ov = __shfl_xor_sync(0xffffffffu, acc[j], o);
-                            acc[j] = low ? (acc[j] + ov) : (ov + acc[j]);
-                        }
-                    }
+                    const int len = C.rp[r + 1] - C.rp[r];
                     float* part = reinterpret_cast<float*>(smem_raw + (part0 - smem_u32(smem_raw)));
-                    if (lane < lpr && col_lane) {
-#pragma unroll
-                        for (int j = 0; j < EPC; ++j) part[(size_t)gw * K + li * EPC + j] = acc[j];
-                    }
+                    pl_long_share<T, WEIGHTED>(P, C.rp[r], len, gw, part, Xl, row_bytes, lane, lpr, col_lane, pol_keep);
                     pl_named_barrier(2, 32 * PL_LONG_WARPS);
                     if (gw == 0 && lane < lpr && col_lane) {
                         float v[EPC];
@@ -467,23 +515,30 @@ static gnn_status pl_launch(const char* who, const int64_t* rowptr, const int32_
     const size_t fixed = pl_fixed_bytes(Kc, Mo, levels), stage = pl_stage_bytes(Kc, levels);
     int stages = (int)((PL_SMEM_MAX - fixed) / stage);
     P.stages = stages > PL_MAX_STAGES ? PL_MAX_STAGES : stages;
+    const size_t left = PL_SMEM_MAX - fixed - (size_t)P.stages * stage;
+    int window = (int)(left / ((size_t)P.stages * 8)) & ~31;
+    P.window = window > PL_WINDOW ? PL_WINDOW : window;
     P.acc_stride = (Mo + 31) & ~31;
     int cols = 32;
     while (cols < 2 * P.acc_stride) cols <<= 1;
     P.tmem_cols = cols;
-    const size_t smem = fixed + (size_t)P.stages * stage;
+    const size_t smem = fixed + (size_t)P.stages * stage + (size_t)P.stages * P.window * 8;
     const int64_t ntiles = ((int64_t)N + TC_ROWS - 1) / TC_ROWS;
     const int grid = (int)(ntiles < 148 ? ntiles : 148);
     gnn_status rc;
-    if (dtype == GNN_F32) {
-        rc = allow_big_smem(who, (const void*)propagate_linear_kernel<float>, 8, PL_SMEM_MAX);
-        if (rc != GNN_OK) return rc;
-        propagate_linear_kernel<float><<<grid, PL_THREADS, smem, st>>>(mapY, P);
-    } else {
-        rc = allow_big_smem(who, (const void*)propagate_linear_kernel<__nv_bfloat16>, 9, PL_SMEM_MAX);
-        if (rc != GNN_OK) return rc;
-        propagate_linear_kernel<__nv_bfloat16><<<grid, PL_THREADS, smem, st>>>(mapY, P);
+    const bool weighted = w != nullptr || gscale_rowptr != nullptr;
+#define GNN_PL_CASE(TYPE, WFLAG, SLOT)                                                                  \
+    {                                                                                                   \
+        rc = allow_big_smem(who, (const void*)propagate_linear_kernel<TYPE, WFLAG>, SLOT, PL_SMEM_MAX); \
+        if (rc != GNN_OK) return rc;                                                                    \
+        propagate_linear_kernel<TYPE, WFLAG><<<grid, PL_THREADS, smem, st>>>(mapY, P);                  \
     }
+    if (dtype == GNN_F32) {
+        if (weighted) GNN_PL_CASE(float, true, 8) else GNN_PL_CASE(float, false, 9)
+    } else {
+        if (weighted) GNN_PL_CASE(__nv_bfloat16, true, 10) else GNN_PL_CASE(__nv_bfloat16, false, 11)
+    }
+#undef GNN_PL_CASE
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
