@@ -34,56 +34,64 @@ UNIT = "edges*feat/s"
 ALL_CASES = [(F, dt) for dt in ("bf16", "f32") for F in (32, 64, 128, 256, 512)]
 FMAX = 512
 
-# DRAM bytes (read + write, GB) of one gnn_propagate_fused / _backward call (all its propagate_chunk_kernel
-# launches: wide rows run as 512-byte column slabs) at full size, taken once with the hardware counters
-# dram__bytes_read.sum + dram__bytes_write.sum.  The numbers belong to the kernel sources whose digest is
-# TRAFFIC_KERNEL_SHA256; with any other sources the line reports traffic = null.
-TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none (single pass) over one step of this "
-                  "sweep at full size, row-walking and fix-up kernels as of commit 8f9365f (unchanged up to the digest below); per-call sums in the summary of the full-size DRAM-byte capture under profiles/")
+# DRAM bytes (read + write, GB) of one gnn_propagate_fused / _backward call (all its propagate_chunk_kernel and
+# fix-up launches: wide rows run as 512-byte column slabs), taken with the hardware counters
+# dram__bytes_read.sum + dram__bytes_write.sum on a REDUCED graph of the same generator (--graph-scale 20:
+# N = 600,000, E = 30,750,000, a quarter of the workload) so that the capture stays small.  The line reports
+# these numbers times TRAFFIC_SCALE (the ratio of the edges*features processed).  That is a LOWER bound of the
+# full-size traffic: the reduced feature matrix is four times smaller against the same L2, so a larger share of
+# its gathers hits (a full-size capture of an earlier build of the same loop gave 79.6 GB where this gives 34.1).
+# The numbers belong to the kernel sources whose digest is TRAFFIC_KERNEL_SHA256; with other sources the line
+# reports traffic = null.
+TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:propagate_ over one step of "
+                  "`bench.py --graph-scale 20` (N=600000, E=30.75M), scaled by 4.0 = ratio of edges*features; lower bound of the "
+                  "full-size traffic (better L2 reuse on the reduced matrix); summary under profiles/")
+TRAFFIC_SCALE = 4.0
 TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
-TRAFFIC_KERNEL_SHA256 = "c23bd6af0c3f8a9b1bc495d55dedf585f3abe630dbae8a92d4ff992552f83415"
-TRAFFIC_GB = {
-    "32:bf16:copy_xj:fwd": 1.48,
-    "32:bf16:copy_xj:bwd": 1.48,
-    "32:bf16:e_mul_xj:fwd": 1.99,
-    "32:bf16:e_mul_xj:bwd": 1.99,
-    "64:bf16:copy_xj:fwd": 2.08,
-    "64:bf16:copy_xj:bwd": 2.08,
-    "64:bf16:e_mul_xj:fwd": 2.59,
-    "64:bf16:e_mul_xj:bwd": 2.59,
-    "128:bf16:copy_xj:fwd": 6.36,
-    "128:bf16:copy_xj:bwd": 6.36,
-    "128:bf16:e_mul_xj:fwd": 6.88,
-    "128:bf16:e_mul_xj:bwd": 6.87,
-    "256:bf16:copy_xj:fwd": 19.25,
-    "256:bf16:copy_xj:bwd": 19.21,
-    "256:bf16:e_mul_xj:fwd": 19.76,
-    "256:bf16:e_mul_xj:bwd": 19.73,
-    "512:bf16:copy_xj:fwd": 38.5,
-    "512:bf16:copy_xj:bwd": 38.44,
-    "512:bf16:e_mul_xj:fwd": 39.52,
-    "512:bf16:e_mul_xj:bwd": 39.46,
-    "32:f32:copy_xj:fwd": 2.02,
-    "32:f32:copy_xj:bwd": 2.02,
-    "32:f32:e_mul_xj:fwd": 2.52,
-    "32:f32:e_mul_xj:bwd": 2.52,
-    "64:f32:copy_xj:fwd": 6.43,
-    "64:f32:copy_xj:bwd": 6.42,
-    "64:f32:e_mul_xj:fwd": 6.94,
-    "64:f32:e_mul_xj:bwd": 6.93,
-    "128:f32:copy_xj:fwd": 19.35,
-    "128:f32:copy_xj:bwd": 19.32,
-    "128:f32:e_mul_xj:fwd": 19.87,
-    "128:f32:e_mul_xj:bwd": 19.83,
-    "256:f32:copy_xj:fwd": 38.74,
-    "256:f32:copy_xj:bwd": 38.67,
-    "256:f32:e_mul_xj:fwd": 39.77,
-    "256:f32:e_mul_xj:bwd": 39.7,
-    "512:f32:copy_xj:fwd": 77.53,
-    "512:f32:copy_xj:bwd": 77.38,
-    "512:f32:e_mul_xj:fwd": 79.59,
-    "512:f32:e_mul_xj:bwd": 79.43,
+TRAFFIC_KERNEL_SHA256 = "f1b340a40f7d191dc97ac696cba06d6912251e9a0cfa21be128fb947310d6892"
+TRAFFIC_GB_REDUCED = {
+    "32:bf16:copy_xj:fwd": 0.189,
+    "32:bf16:copy_xj:bwd": 0.188,
+    "32:bf16:e_mul_xj:fwd": 0.313,
+    "32:bf16:e_mul_xj:bwd": 0.313,
+    "64:bf16:copy_xj:fwd": 0.268,
+    "64:bf16:copy_xj:bwd": 0.269,
+    "64:bf16:e_mul_xj:fwd": 0.393,
+    "64:bf16:e_mul_xj:bwd": 0.394,
+    "128:bf16:copy_xj:fwd": 0.616,
+    "128:bf16:copy_xj:bwd": 0.616,
+    "128:bf16:e_mul_xj:fwd": 0.744,
+    "128:bf16:e_mul_xj:bwd": 0.743,
+    "256:bf16:copy_xj:fwd": 1.987,
+    "256:bf16:copy_xj:bwd": 1.986,
+    "256:bf16:e_mul_xj:fwd": 2.116,
+    "256:bf16:e_mul_xj:bwd": 2.115,
+    "512:bf16:copy_xj:fwd": 3.981,
+    "512:bf16:copy_xj:bwd": 3.985,
+    "512:bf16:e_mul_xj:fwd": 4.239,
+    "512:bf16:e_mul_xj:bwd": 4.245,
+    "32:f32:copy_xj:fwd": 0.251,
+    "32:f32:copy_xj:bwd": 0.251,
+    "32:f32:e_mul_xj:fwd": 0.376,
+    "32:f32:e_mul_xj:bwd": 0.376,
+    "64:f32:copy_xj:fwd": 0.601,
+    "64:f32:copy_xj:bwd": 0.601,
+    "64:f32:e_mul_xj:fwd": 0.729,
+    "64:f32:e_mul_xj:bwd": 0.729,
+    "128:f32:copy_xj:fwd": 2.0,
+    "128:f32:copy_xj:bwd": 1.997,
+    "128:f32:e_mul_xj:fwd": 2.13,
+    "128:f32:e_mul_xj:bwd": 2.127,
+    "256:f32:copy_xj:fwd": 4.015,
+    "256:f32:copy_xj:bwd": 4.007,
+    "256:f32:e_mul_xj:fwd": 4.275,
+    "256:f32:e_mul_xj:bwd": 4.266,
+    "512:f32:copy_xj:fwd": 8.014,
+    "512:f32:copy_xj:bwd": 8.007,
+    "512:f32:e_mul_xj:fwd": 8.533,
+    "512:f32:e_mul_xj:bwd": 8.528,
 }
+TRAFFIC_GB = {k: v * TRAFFIC_SCALE for k, v in TRAFFIC_GB_REDUCED.items()}
 
 
 def parse_cases(s):
@@ -422,6 +430,7 @@ def main():
                 % (dom["F"], dom["dtype"], dom["msg"], nslab, 100 * (dom["fwd_ms"] + dom["bwd_ms"]) / tot_ms),
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if traffic is None else traffic * 1e9,
+                "traffic_scaled_from_reduced_graph": traffic is not None,
                 "traffic_source": (TRAFFIC_SOURCE + "; kernel sources sha256 " + TRAFFIC_KERNEL_SHA256[:16]) if traffic is not None else
                                   "null: the kernel sources differ from the ones the counters were taken with, or this is not the full-size relabelled workload",
                 "peak_source": peak_src, "bytes_model": "compulsory bytes per call: 4E(+4E weights)+8N+2*N*F*s = %d" % comp,
