@@ -197,6 +197,11 @@ struct Walker {
     // issue the last (fewer than U) gathers of a row segment together instead of one by one: measured
     // faster for max/min (-7..-29 % on short-row graphs), slower for the sum and routing modes
     static constexpr bool BATCH_TAIL = (MODE == MODE_MAX || MODE == MODE_MIN);
+    // sum over full-warp fp32 rows: the ragged end of a row segment goes through the same loop as the full batches,
+    // its missing positions predicated off, so that the gathers of a short row are in flight together (measured on
+    // the large graph: -1..-2 % sustained, -7 % in a burst).  Not for bf16: with eight accumulators per lane the
+    // loop spills registers and runs a third slower.
+    static constexpr bool ONE_LOOP = MODE == MODE_SUM && LPR == 32 && Chunk<T>::N == 4;
     static constexpr int EPC = Chunk<T>::N;
     static constexpr int NG = 32 / LPR;
     static constexpr bool EF = (MODE == MODE_EFSUM);  // one multiplier per (position, feature)
@@ -223,10 +228,10 @@ struct Walker {
     }
 
     // copy indices and multipliers of positions [sb, se) into shared memory (one round trip)
-    __device__ __forceinline__ static void stage(const PropParams& P, int64_t sb, int64_t se, int lane,
+    __device__ __forceinline__ static void stage(const PropParams& P, int sb, int se, int lane,
                                                  SlabSmem& S, uint64_t pol_stream) {
         __syncwarp();
-        for (int i = lane; i < (int)(se - sb); i += 32) {
+        for (int i = lane; i < se - sb; i += 32) {
             int c = P.col ? ld_hint_i32(P.col + sb + i, pol_stream) : (int)(sb + i);  // no col: row p of X
             float w = P.w ? ld_hint_f32(P.w + sb + i, pol_stream) : 1.0f;
             if (P.gscale_rowptr) {
@@ -286,7 +291,7 @@ struct Walker {
     // accumulate staged positions [p0, e1) (all inside the slab starting at sb) into acc.
     // Lanes beyond the row width (rows that do not fill LPR*VPL chunks) read chunk 0 instead:
     // always in bounds, never written back, so the loop needs no lane masking.
-    __device__ __forceinline__ static void slab_segment(const PropParams& P, int64_t sb, int64_t p0, int64_t e1,
+    __device__ __forceinline__ static void slab_segment(const PropParams& P, int sb, int p0, int e1,
                                                         int lane, const SlabSmem& S, uint64_t pol_keep, A& acc) {
         const int g = lane / LPR, li = lane % LPR;
         const uint32_t row_bytes = P.x_ld;
@@ -303,8 +308,35 @@ struct Walker {
         for (int v = 0; v < VPL; ++v)
             whl[v] = (MODE == MODE_HEADSUM) ? P.wh + (size_t)sb * P.H + (c0[v] * EPC) / P.fph
                      : EF ? P.ef + (size_t)sb * P.ef_ld + (size_t)c0[v] * EPC : nullptr;
-        const int i1 = (int)(e1 - sb);
-        int i = (int)(p0 - sb) + g;
+        const int i1 = e1 - sb;
+        int i = p0 - sb + g;
+        if (ONE_LOOP) {
+            for (; i < i1; i += NG * U) {
+                int cols[U];
+                uint4 buf[U][VPL];
+#pragma unroll
+                for (int u = 0; u < U; ++u) cols[u] = S.e[i + u * NG < i1 ? i + u * NG : i].x;
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (i + u * NG < i1) {
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) buf[u][v] = ld_hint16(Xl[v] + (size_t)(uint32_t)cols[u] * row_bytes, pol_keep);
+                    }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (i + u * NG < i1) {
+                        const float w = __int_as_float(S.e[i + u * NG].z);  // read again here: not held across the gathers
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v) {
+                            float x[EPC];
+                            Chunk<T>::unpack(buf[u][v], x);
+#pragma unroll
+                            for (int j = 0; j < EPC; j += 2) fma2(acc.v[v][j], acc.v[v][j + 1], x[j], x[j + 1], w, w);
+                        }
+                    }
+            }
+            return;
+        }
         // full groups of U positions per lane group: no predicates
         for (; i + (U - 1) * NG < i1; i += NG * U) {
             int4 e[U];
@@ -391,8 +423,8 @@ struct Walker {
         }
     }
 
-    __device__ __forceinline__ static void write_final(const PropParams& P, int64_t row,
-                                                       int64_t deg, int lane, A& acc) {
+    __device__ __forceinline__ static void write_final(const PropParams& P, int row,
+                                                       int deg, int lane, A& acc) {
         if (lane >= LPR) return;
         char* ob = reinterpret_cast<char*>(P.out) + (size_t)row * P.out_ld;
 #pragma unroll
@@ -418,7 +450,7 @@ struct Walker {
         }
     }
 
-    __device__ __forceinline__ static void write_partial(const PropParams& P, int64_t chunk,
+    __device__ __forceinline__ static void write_partial(const PropParams& P, int chunk,
                                                          int which, int lane, const A& acc) {
         if (lane >= LPR) return;
         size_t off = ((size_t)chunk * 2 + which) * P.F;
@@ -449,37 +481,37 @@ propagate_chunk_kernel(const PropParams P) {
     using W = Walker<T, LPR, VPL, MODE>;
     __shared__ SlabSmem s_slab[PF_WARPS];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int64_t c = (int64_t)blockIdx.x * PF_WARPS + wib;
+    const int c = (int)blockIdx.x * PF_WARPS + wib;  // chunk numbers and positions fit 32 bits (the host checks E < 2^31)
     if (c >= P.nchunks) return;
     SlabSmem& S = s_slab[wib];
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
-    const int64_t cs = c * P.chunk;
-    const int64_t ce = (cs + P.chunk < P.E) ? cs + P.chunk : P.E;
+    const int cs = c * P.chunk;
+    const int ce = ((int64_t)cs + P.chunk < P.E) ? cs + P.chunk : (int)P.E;
 
     typename W::A acc;
 
     // cur = the row containing position cs, or the first (possibly empty) row starting at cs
     int cur = lower_bound_i64(P.rowptr, P.N + 1, cs);
     if (P.rowptr[cur] > cs) --cur;
-    int64_t pos = cs;
-    int64_t sb = cs - PF_SLAB;  // nothing staged yet
+    int pos = cs;
+    int sb = cs - PF_SLAB;  // nothing staged yet
     int32_t tail = -1;
     while (cur < P.N) {
-        const int64_t rs = P.rowptr[cur], re = P.rowptr[cur + 1];
+        const int rs = (int)P.rowptr[cur], re = (int)P.rowptr[cur + 1];
         if (re == rs) {  // no edges (written by the scan above): jump to the next row that has some
             cur = first_row_ending_after(P.rowptr, cur + 1, P.N, rs, lane);
             if (cur >= P.N || P.rowptr[cur] >= ce) break;  // it belongs to a later chunk
             continue;
         }
-        const int64_t b = re < ce ? re : ce;
+        const int b = re < ce ? re : ce;
         acc.clear();
-        const int64_t pos0 = pos;
+        const int pos0 = pos;
         while (pos < b) {
             if (pos >= sb + PF_SLAB) {
                 sb = cs + ((pos - cs) / PF_SLAB) * PF_SLAB;
                 W::stage(P, sb, (sb + PF_SLAB < ce) ? sb + PF_SLAB : ce, lane, S, pol_stream);
             }
-            const int64_t e = (b < sb + PF_SLAB) ? b : sb + PF_SLAB;
+            const int e = (b < sb + PF_SLAB) ? b : sb + PF_SLAB;
             W::slab_segment(P, sb, pos, e, lane, S, pol_keep, acc);
             pos = e;
         }
@@ -1365,6 +1397,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     GNN_REQUIRE(pick_shape(nvec, &lpr, &vpl), GNN_ERR_UNSUPPORTED,
                 "%s: feature rows wider than 2048 bytes are not supported (F=%d)", who, F);
     GNN_REQUIRE(aligned16(X) && aligned16(out), GNN_ERR_INVALID_ARG, "%s: feature matrices must be 16-byte aligned", who);
+    GNN_REQUIRE(E >= 0 && E < ((int64_t)1 << 31) - 4 * PF_SLAB, GNN_ERR_UNSUPPORTED, "%s: positions must fit 32 bits (E < 2^31)", who);
     const bool with_arg = (mode == MODE_MAX || mode == MODE_MIN);
     PfWs wsv = pf_carve(ws, E, F, with_arg);
     GNN_REQUIRE(ws && ws_bytes >= wsv.bytes && aligned16(ws), GNN_ERR_WORKSPACE_TOO_SMALL,
