@@ -40,7 +40,7 @@ FMAX = 512
 # N = 600,000, E = 30,750,000, a quarter of the workload) so that the capture stays small.  The line reports
 # these numbers times TRAFFIC_SCALE (the ratio of the edges*features processed).  That is a LOWER bound of the
 # full-size traffic: the reduced feature matrix is four times smaller against the same L2, so a larger share of
-# its gathers hits (a full-size capture of an earlier build of the same loop gave 79.6 GB where this gives 34.1).
+# its gathers hits (a full-size capture of an earlier build of the same loop gave 79.6 GB where this gives 32.8).
 # The numbers belong to the kernel sources whose digest is TRAFFIC_KERNEL_SHA256; with other sources the line
 # reports traffic = null.
 TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:propagate_ over one step of "
@@ -48,48 +48,48 @@ TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cl
                   "full-size traffic (better L2 reuse on the reduced matrix); summary under profiles/")
 TRAFFIC_SCALE = 4.0
 TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
-TRAFFIC_KERNEL_SHA256 = "f1b340a40f7d191dc97ac696cba06d6912251e9a0cfa21be128fb947310d6892"
+TRAFFIC_KERNEL_SHA256 = "b072d8522ce51f1be9ffd1200a24fc359896326c722ce6fee607bb155dc48b51"
 TRAFFIC_GB_REDUCED = {
-    "32:bf16:copy_xj:fwd": 0.189,
-    "32:bf16:copy_xj:bwd": 0.188,
-    "32:bf16:e_mul_xj:fwd": 0.313,
-    "32:bf16:e_mul_xj:bwd": 0.313,
-    "64:bf16:copy_xj:fwd": 0.268,
-    "64:bf16:copy_xj:bwd": 0.269,
-    "64:bf16:e_mul_xj:fwd": 0.393,
-    "64:bf16:e_mul_xj:bwd": 0.394,
-    "128:bf16:copy_xj:fwd": 0.616,
-    "128:bf16:copy_xj:bwd": 0.616,
-    "128:bf16:e_mul_xj:fwd": 0.744,
-    "128:bf16:e_mul_xj:bwd": 0.743,
-    "256:bf16:copy_xj:fwd": 1.987,
-    "256:bf16:copy_xj:bwd": 1.986,
-    "256:bf16:e_mul_xj:fwd": 2.116,
-    "256:bf16:e_mul_xj:bwd": 2.115,
-    "512:bf16:copy_xj:fwd": 3.981,
-    "512:bf16:copy_xj:bwd": 3.985,
-    "512:bf16:e_mul_xj:fwd": 4.239,
-    "512:bf16:e_mul_xj:bwd": 4.245,
-    "32:f32:copy_xj:fwd": 0.251,
-    "32:f32:copy_xj:bwd": 0.251,
-    "32:f32:e_mul_xj:fwd": 0.376,
-    "32:f32:e_mul_xj:bwd": 0.376,
-    "64:f32:copy_xj:fwd": 0.601,
-    "64:f32:copy_xj:bwd": 0.601,
-    "64:f32:e_mul_xj:fwd": 0.729,
-    "64:f32:e_mul_xj:bwd": 0.729,
-    "128:f32:copy_xj:fwd": 2.0,
-    "128:f32:copy_xj:bwd": 1.997,
-    "128:f32:e_mul_xj:fwd": 2.13,
-    "128:f32:e_mul_xj:bwd": 2.127,
-    "256:f32:copy_xj:fwd": 4.015,
-    "256:f32:copy_xj:bwd": 4.007,
-    "256:f32:e_mul_xj:fwd": 4.275,
-    "256:f32:e_mul_xj:bwd": 4.266,
-    "512:f32:copy_xj:fwd": 8.014,
-    "512:f32:copy_xj:bwd": 8.007,
-    "512:f32:e_mul_xj:fwd": 8.533,
-    "512:f32:e_mul_xj:bwd": 8.528,
+    "32:bf16:copy_xj:fwd": 0.188,
+    "32:bf16:copy_xj:bwd": 0.187,
+    "32:bf16:e_mul_xj:fwd": 0.311,
+    "32:bf16:e_mul_xj:bwd": 0.312,
+    "64:bf16:copy_xj:fwd": 0.265,
+    "64:bf16:copy_xj:bwd": 0.265,
+    "64:bf16:e_mul_xj:fwd": 0.389,
+    "64:bf16:e_mul_xj:bwd": 0.39,
+    "128:bf16:copy_xj:fwd": 0.597,
+    "128:bf16:copy_xj:bwd": 0.597,
+    "128:bf16:e_mul_xj:fwd": 0.724,
+    "128:bf16:e_mul_xj:bwd": 0.724,
+    "256:bf16:copy_xj:fwd": 2.002,
+    "256:bf16:copy_xj:bwd": 2.003,
+    "256:bf16:e_mul_xj:fwd": 2.131,
+    "256:bf16:e_mul_xj:bwd": 2.131,
+    "512:bf16:copy_xj:fwd": 4.014,
+    "512:bf16:copy_xj:bwd": 4.017,
+    "512:bf16:e_mul_xj:fwd": 4.272,
+    "512:bf16:e_mul_xj:bwd": 4.275,
+    "32:f32:copy_xj:fwd": 0.249,
+    "32:f32:copy_xj:bwd": 0.249,
+    "32:f32:e_mul_xj:fwd": 0.374,
+    "32:f32:e_mul_xj:bwd": 0.374,
+    "64:f32:copy_xj:fwd": 0.587,
+    "64:f32:copy_xj:bwd": 0.586,
+    "64:f32:e_mul_xj:fwd": 0.713,
+    "64:f32:e_mul_xj:bwd": 0.714,
+    "128:f32:copy_xj:fwd": 1.915,
+    "128:f32:copy_xj:bwd": 1.914,
+    "128:f32:e_mul_xj:fwd": 2.046,
+    "128:f32:e_mul_xj:bwd": 2.043,
+    "256:f32:copy_xj:fwd": 3.842,
+    "256:f32:copy_xj:bwd": 3.838,
+    "256:f32:e_mul_xj:fwd": 4.101,
+    "256:f32:e_mul_xj:bwd": 4.097,
+    "512:f32:copy_xj:fwd": 7.672,
+    "512:f32:copy_xj:bwd": 7.668,
+    "512:f32:e_mul_xj:fwd": 8.191,
+    "512:f32:e_mul_xj:bwd": 8.186,
 }
 TRAFFIC_GB = {k: v * TRAFFIC_SCALE for k, v in TRAFFIC_GB_REDUCED.items()}
 

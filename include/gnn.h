@@ -381,6 +381,9 @@ gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, con
  * head must span a power-of-two number (1..32) of 16-byte chunks (C = 4, 8, 16, ... for float,
  * 8, 16, 32, ... for bf16); other shapes return GNN_ERR_UNSUPPORTED from the forward and the
  * backward call alike.  The E x F message tensor is never formed.
+ * The first gnn_gat_fused / _backward call on a device creates two helper streams and three events (no device
+ * memory) on which row classes of the attention kernels run side by side; they are forked from and joined back
+ * into `stream`, so the call keeps its place in the stream's order.  Make that first call outside a stream capture.
  * ws: gnn_gat_fused_workspace(N, E, H, C, backward) bytes. */
 size_t gnn_gat_fused_workspace(int32_t N, int64_t E, int H, int C, int backward);
 gnn_status gnn_gat_fused(const gnn_csr* g, const void* Wx, const float* a_src, const float* a_dst,

@@ -197,11 +197,11 @@ struct Walker {
     // issue the last (fewer than U) gathers of a row segment together instead of one by one: measured
     // faster for max/min (-7..-29 % on short-row graphs), slower for the sum and routing modes
     static constexpr bool BATCH_TAIL = (MODE == MODE_MAX || MODE == MODE_MIN);
-    // sum over full-warp fp32 rows: the ragged end of a row segment goes through the same loop as the full batches,
-    // its missing positions predicated off, so that the gathers of a short row are in flight together (measured on
-    // the large graph: -1..-2 % sustained, -7 % in a burst).  Not for bf16: with eight accumulators per lane the
-    // loop spills registers and runs a third slower.
-    static constexpr bool ONE_LOOP = MODE == MODE_SUM && LPR == 32 && Chunk<T>::N == 4;
+    // fp32 sums: the ragged end of a row segment goes through the same loop as the full batches, its missing
+    // positions predicated off, so that the gathers of a short row are in flight together (measured on the large
+    // graph: F = 64 -6 %, F = 128..512 -1..-2 % sustained, -7 % in a burst).  Not for bf16: with eight accumulators
+    // per lane the loop spills registers on full-warp rows (a third slower) and gains nothing on narrow ones.
+    static constexpr bool ONE_LOOP = MODE == MODE_SUM && VPL == 1 && Chunk<T>::N == 4;
     static constexpr int EPC = Chunk<T>::N;
     static constexpr int NG = 32 / LPR;
     static constexpr bool EF = (MODE == MODE_EFSUM);  // one multiplier per (position, feature)

@@ -5,6 +5,8 @@
 // One warp per row for ordinary rows; rows longer than SM_LONG_ROW positions are left to a
 // second kernel that gives each of them a whole block.  Reductions use fixed shuffle / shared
 // memory trees, so results are bit-reproducible.  All arithmetic is fp32.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace gnn {
@@ -459,13 +461,61 @@ static int row_grid_sub(int N) {
     return (int)(want < cap ? (want > 0 ? want : 1) : cap);
 }
 
+// The three row tiers (8 threads, a warp, a block per row) touch disjoint rows and none of them fills the
+// machine alone (the block tier runs two blocks per SM and is as long as its longest row).  They run side by
+// side: the block tier on the caller's stream, the other two on two helper streams that are forked from the
+// caller's stream and joined back into it with events, so the call keeps its place in the caller's stream order.
+// The helper streams and events are created on the first call on a device (make that call outside any stream
+// capture); if they cannot be had, the tiers run one after the other.
+struct TierStreams {
+    cudaStream_t s[2];
+    cudaEvent_t fork, join[2];
+    int state;  // 0: not tried, 1: ready, -1: unavailable
+};
+static std::mutex g_tier_mutex;
+static TierStreams g_tier[64];
+
+template <class Long, class Warp, class Sub>
+static void run_row_tiers(cudaStream_t st, Long run_long, Warp run_warp, Sub run_sub) {
+    std::lock_guard<std::mutex> lock(g_tier_mutex);  // one host thread at a time forks and joins through the shared events
+    int dev = -1;
+    TierStreams* t = nullptr;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        t = &g_tier[dev];
+        if (t->state == 0) {
+            bool ok = cudaStreamCreateWithFlags(&t->s[0], cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaStreamCreateWithFlags(&t->s[1], cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&t->fork, cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&t->join[0], cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&t->join[1], cudaEventDisableTiming) == cudaSuccess;
+            t->state = ok ? 1 : -1;
+            if (!ok) (void)cudaGetLastError();
+        }
+        if (t->state != 1) t = nullptr;
+    }
+    if (!t || cudaEventRecord(t->fork, st) != cudaSuccess || cudaStreamWaitEvent(t->s[0], t->fork, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(t->s[1], t->fork, 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        run_long(st); run_warp(st); run_sub(st);
+        return;
+    }
+    run_long(st);
+    run_warp(t->s[0]);
+    run_sub(t->s[1]);
+    cudaEventRecord(t->join[0], t->s[0]);
+    cudaEventRecord(t->join[1], t->s[1]);
+    cudaStreamWaitEvent(st, t->join[0], 0);
+    cudaStreamWaitEvent(st, t->join[1], 0);
+}
+
 gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float slope, int H, float* alpha, cudaStream_t st) {
     if (g->N == 0 || g->E == 0) return GNN_OK;
     const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true), sg = row_grid_sub(g->N);
-#define GNN_GA(HV)                                                                                                    \
-    gat_alpha_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);       \
-    gat_alpha_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);          \
-    gat_alpha_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha);
+#define GNN_GA(HV)                                                                                                                       \
+    run_row_tiers(                                                                                                                       \
+        st, [&](cudaStream_t q) { gat_alpha_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha); }, \
+        [&](cudaStream_t q) { gat_alpha_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha); },    \
+        [&](cudaStream_t q) { gat_alpha_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha); });
     if (H == 4) { GNN_GA(1) } else if (H == 8) { GNN_GA(2) } else if (H == 16) { GNN_GA(4) } else if (H == 32) { GNN_GA(8) } else {
         gat_alpha_kernel<false><<<row_grid(g->N, false), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
         gat_alpha_kernel<true><<<row_grid(g->N, true), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
@@ -479,10 +529,11 @@ gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float s
 bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz, const float* al, const float* ar,
                           float slope, int H, float* dar, cudaStream_t st) {
     const int wg = row_grid_pl(g->N, false), lg = row_grid_pl(g->N, true), sg = row_grid_sub(g->N);
-#define GNN_GB(HV)                                                                                                               \
-    gat_rows_bwd_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar); \
-    gat_rows_bwd_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);  \
-    gat_rows_bwd_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar);
+#define GNN_GB(HV)                                                                                                                                       \
+    run_row_tiers(                                                                                                                                       \
+        st, [&](cudaStream_t q) { gat_rows_bwd_pl_kernel<HV, true><<<lg, PL_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar); }, \
+        [&](cudaStream_t q) { gat_rows_bwd_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar); },    \
+        [&](cudaStream_t q) { gat_rows_bwd_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, alpha, dalpha_dz, al, ar, slope, dar); });
     if (H == 4) { GNN_GB(1) } else if (H == 8) { GNN_GB(2) } else if (H == 16) { GNN_GB(4) } else if (H == 32) { GNN_GB(8) } else return false;
 #undef GNN_GB
     return true;

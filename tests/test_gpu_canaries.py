@@ -167,3 +167,65 @@ def test_unfused_softmax_pooling_attention_and_dense_stay_inside_their_buffers(g
         gt.check(f"linear_backward {N}x{K}x{M}")
     gnn.axpby(0.5, X, 2.0, X)
     gt.check("axpby")
+
+
+def test_new_messages_merged_graphs_and_fused_transform_stay_inside_their_buffers(guarded):
+    import torch
+    gnn, gt = guarded
+    n, e = 1500, 30_000
+    src, dst = graph(n, e, 21, hub=5000)
+    g = gnn.coo_to_csr(n, to_dev(src), to_dev(dst))
+    gt.check("coo_to_csr")
+    for dtype, F, H in [("f32", 64, 4), ("bf16", 128, 8), ("bf16", 1024, 4), ("f32", 260, 1)]:
+        X = to_dev(synth.normal((n, F), dtype, 22))
+        R = to_dev(synth.normal((n, F), dtype, 23))
+        bias = to_dev(synth.uniform_f32((F,), -1.0, 1.0, 24))
+        for op in ("sum", "mean", "max", "min"):
+            r = gnn.propagate_msg(g, gnn.XI_SUB_XJ, X, Xi=R, op=op, epi=dict(bias=bias, relu=True))
+            gt.check(f"x_i - x_j {op} F={F} {dtype}")
+            arg = r[1] if op in ("max", "min") else None
+            gnn.propagate_msg_backward(g, gnn.XI_SUB_XJ, R, op=op, argmax=arg, want_dXi=True,
+                                       self_grad=dict(Xself=R, self_coef=1.0, self_mode=gnn.SELF_IF_NONEMPTY))
+            gt.check(f"x_i - x_j backward {op} F={F} {dtype}")
+        widths = [F] if H == 1 else [H, F]
+        for ew in widths:
+            ef = to_dev(synth.uniform_f32((e, ew), -1.0, 1.0, 25))
+            gnn.propagate_msg(g, gnn.E_MUL_XJ, X, e_csr=ef, op="mean")
+            gt.check(f"edge factors width {ew}")
+            gnn.propagate_msg_backward(g, gnn.E_MUL_XJ, R, op="mean", Xj=X, e_csrT=ef, want_de=True)
+            gt.check(f"edge factors backward width {ew}")
+        Y = gnn.gin(g, X, 0.5)
+        gt.check("gin")
+        gnn.gin_backward(g, R, 0.5, X=X, want_deps=True)
+        gt.check("gin_backward")
+        gnn.row_epilogue_backward(Y, R, relu=True)
+        gt.check("row_epilogue_backward")
+        if F <= 512:
+            s = gnn.edge_dot(g, X, R, H)
+            gt.check("edge_dot")
+            gnn.edge_dot_backward(g, X, R, s, H)
+            gt.check("edge_dot_backward")
+    # merged multi-relation graph
+    a = (to_dev(src[:9000] % 500), to_dev(dst[:9000] % 600), 0, 0)
+    b = (to_dev(src[9000:] % 800), to_dev(dst[9000:] % 600), 500, 0)
+    ms, md, seg = gnn.merge_edge_lists([a, b])
+    gt.check("merge_edge_lists")
+    gm = gnn.coo_to_csr(1300, ms, md)
+    seg_csr = gnn.permute_edge_data(gm.eid[:gm.E], seg)
+    coef, coefT = gnn.segment_coef(gm, seg_csr, torch.tensor([1, 0], dtype=torch.int32, device="cuda"))
+    gt.check("segment_coef")
+    # aggregate -> transform fusion and the dense transform with its tail
+    for dt, K, M in [(torch.bfloat16, 128, 128), (torch.bfloat16, 256, 256), (torch.float32, 64, 64), (torch.float32, 128, 128),
+                     (torch.float32, 256, 64), (torch.bfloat16, 48, 80)]:
+        X = torch.randn(n, K, device="cuda").to(dt)
+        W = torch.randn(K, M, device="cuda").to(dt)
+        dY = torch.randn(n, M, device="cuda").to(dt)
+        bias = torch.randn(M, device="cuda")
+        gnn.propagate_linear(g, X, W, op="mean", bias=bias, relu=True)
+        gt.check(f"propagate_linear {K}x{M}")
+        gnn.propagate_linear_backward(g, dY, X, W, op="mean", want_dW=False)
+        gt.check(f"propagate_linear_backward dX {K}x{M}")
+        gnn.propagate_linear_backward(g, dY, X, W, op="mean")
+        gt.check(f"propagate_linear_backward dX+dW {K}x{M}")
+        gnn.linear_bias_act(X, W, bias, relu=True)
+        gt.check(f"linear_bias_act {K}x{M}")
