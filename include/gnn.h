@@ -274,6 +274,25 @@ gnn_status gnn_edge_dot_backward(const gnn_csr* g, const void* Xj, const void* X
                                  const float* ds_csr, int H, int C, gnn_dtype dtype, void* dXj,
                                  void* dXi, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* GATv2-style attention logits (Sec. 3 "Message Passing": apply_edges with target and source features; the
+ * attention layers of Sec. 3 "Graph Convolutional Layers"): the nonlinearity sits between the sum of the two
+ * transformed endpoints and the attention vector, so both rows meet at every edge:
+ *   s[p,h] = sum_c a[h,c] * LeakyReLU_slope(Xl[col[p],h,c] + Xr[i,h,c])     for p in row i
+ * Xl, Xr: [N,H,C] of dtype (source-side and target-side transforms), a: float [H,C], s_csr: float [E,H] in CSR
+ * order (feed it to gnn_edge_softmax, then aggregate Xl with the coefficients through gnn_propagate_msg with
+ * e_width = H).  Rows of H*C elements up to 512 bytes; with H > 1 a head must span a power-of-two number of
+ * 16-byte chunks.  The E x F tensor is never formed.
+ * Backward for ds_csr float [E,H]: dXl, dXr [N,H,C] of dtype and da float [H,C] (da needs dXr and the
+ * workspace; each may be NULL); the derivative of LeakyReLU at 0 is slope.  Rows are walked by a warp, rows over
+ * 256 positions by a block, in a fixed order.  ws: gnn_gatv2_logits_backward_workspace(N, H, C) bytes. */
+gnn_status gnn_gatv2_logits(const gnn_csr* g, const void* Xl, const void* Xr, const float* a, int H, int C,
+                            gnn_dtype dtype, float slope, float* s_csr, gnn_stream stream);
+size_t gnn_gatv2_logits_backward_workspace(int32_t N, int H, int C);
+gnn_status gnn_gatv2_logits_backward(const gnn_csr* g, const void* Xl, const void* Xr, const float* a,
+                                     const float* ds_csr, int H, int C, gnn_dtype dtype, float slope,
+                                     void* dXl, void* dXr, float* da, void* ws, size_t ws_bytes,
+                                     gnn_stream stream);
+
 /* ------------------------------------------------------------------ heterogeneous and temporal graphs */
 
 /* A heterogeneous graph (Sec. 3 "Graph Data Structures": several node and edge types) or a sequence

@@ -366,6 +366,32 @@ def gin_backward(N, src, dst, X, eps, R):
                 deps=float((R64 * _to64(X)).sum()), Sdeps=float(np.abs(R64 * _to64(X)).sum()))
 
 
+def gatv2_logits(src, dst, Xl, Xr, a, H, slope=0.2):
+    """GATv2-style attention logits (the nonlinearity sits between the sum of the two transformed endpoints and
+    the attention vector): s[k,h] = sum_c a[h,c] * LeakyReLU(Xl[src_k,h,c] + Xr[dst_k,h,c]).
+    Composition: the element-wise GAT_LOGIT message over all H*C features, then one dot product per head with a.
+    -> (s [E,H], S [E,H] sums of |terms|, m [E,F] the element-wise messages)."""
+    m = apply_edges(GAT_LOGIT, src, dst, Xl, Y=Xr, slope=slope)
+    E, F = m.shape
+    a64 = _to64(a).reshape(H, F // H)
+    m3 = m.reshape(E, H, F // H)
+    return (m3 * a64[None]).sum(-1), (np.abs(m3) * np.abs(a64)[None]).sum(-1), m
+
+
+def gatv2_logits_backward(N, src, dst, Xl, Xr, a, H, ds, slope=0.2):
+    """For dL/ds = ds [E,H]: dm[k,h,c] = ds[k,h] * a[h,c] * LeakyReLU'(z) (slope at z <= 0), dXl = scatter-add of dm
+    by source, dXr by target, da[h,c] = sum_k ds[k,h] * LeakyReLU(z)[k,h,c] -> dict(dXl, SXl, dXr, SXr, da, Sda)."""
+    _, _, m = gatv2_logits(src, dst, Xl, Xr, a, H, slope)
+    E, F = m.shape
+    a64 = _to64(a).reshape(H, F // H)
+    ds64 = np.asarray(ds, np.float64)
+    dm = (ds64[:, :, None] * a64[None] * np.where(m.reshape(E, H, F // H) > 0, 1.0, float(slope))).reshape(E, F)
+    dXl, SXl = gather_backward(N, src, dm)
+    dXr, SXr = gather_backward(N, dst, dm)
+    t = ds64[:, :, None] * m.reshape(E, H, F // H)
+    return dict(dXl=dXl, SXl=SXl, dXr=dXr, SXr=SXr, da=t.sum(0), Sda=np.abs(t).sum(0))
+
+
 def hetero_propagate(N_dst, relations):
     """Heterogeneous graph: relations = list of dict(src, dst, X, w (or None), op ('sum' | 'mean')); every
     relation sends from its own source node set (rows of its X) to the same target node set; the results are

@@ -236,6 +236,8 @@ bool gat_rows_backward_pl(const gnn_csr* g, const float* alpha, float* dalpha_dz
                           float slope, int H, float* dar, cudaStream_t st);
 gnn_status sddmm_heads(const char* who, const gnn_csr* g, const void* X, const void* dOut, int H, int C,
                        gnn_dtype dtype, float* dW_EH, cudaStream_t st, int mean);
+cudaStream_t side_fork(cudaStream_t st);
+void side_join(cudaStream_t st, cudaStream_t side);
 
 }  // namespace gnn
 
@@ -323,23 +325,33 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
         gat_dal_simple_kernel<<<(int)ceil_div((int64_t)g->N * H, 256), 256, 0, st>>>(g->rowptrT, g->t2f, g->N, H, w.dz, w.dal);
         GNN_CHECK_LAUNCH(who);
     }
-    // attention-vector gradients
+    // attention-vector gradients: two small reductions that need dal and dar only, on a side branch of the stream
+    // beside the transposed gather below (joined before the call returns its place in the stream)
+    cudaStream_t side = side_fork(st);
     if (dtype == GNN_F32)
-        gat_da_partial_kernel<float><<<GA_BLOCKS, 256, 0, st>>>((const float*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
+        gat_da_partial_kernel<float><<<GA_BLOCKS, 256, 0, side>>>((const float*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
     else
-        gat_da_partial_kernel<__nv_bfloat16><<<GA_BLOCKS, 256, 0, st>>>((const __nv_bfloat16*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
-    gat_da_final_kernel<<<(int)ceil_div(F, 16), 256, 0, st>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
-    GNN_CHECK_LAUNCH(who);
+        gat_da_partial_kernel<__nv_bfloat16><<<GA_BLOCKS, 256, 0, side>>>((const __nv_bfloat16*)Wx, w.dal, w.dar, g->N, H, C, w.partial);
+    gat_da_final_kernel<<<(int)ceil_div(F, 16), 256, 0, side>>>(w.partial, GA_BLOCKS, F, da_src, da_dst);
+    if (cudaGetLastError() != cudaSuccess) {
+        side_join(st, side);
+        GNN_FAIL(GNN_ERR_CUDA, "%s: launch failed", who);
+    }
     // dWx[j,h,:] = sum_q alpha[t2f[q],h]*dOut[colT[q],h,:] + dal[j,h]*a_src[h,:] + dar[j,h]*a_dst[h,:]
     // the flat kernel reads alpha through t2f; the row-walking one wants it permuted to transposed order first
     const bool indexed = chunked_is_flat(g->E, F, dtype);
     if (g->E > 0 && !indexed) {
         rc = gnn_permute_edge_data(g->t2f, g->E, H, 4, alpha_csr, w.alphaT, stream);
-        if (rc != GNN_OK) return rc;
+        if (rc != GNN_OK) {
+            side_join(st, side);
+            return rc;
+        }
     }
     HeadExtra hx = {indexed ? alpha_csr : w.alphaT, indexed ? g->t2f : nullptr, H, w.dal, w.dar, a_src, a_dst};
-    return run_chunked(who, MODE_HEADSUM, g->N, g->E, g->rowptrT, g->colT, nullptr, dOut, dWx, nullptr, nullptr,
-                       nullptr, nullptr, 0, F, dtype, w.chunk_ws, w.chunk_bytes, st, &hx);
+    rc = run_chunked(who, MODE_HEADSUM, g->N, g->E, g->rowptrT, g->colT, nullptr, dOut, dWx, nullptr, nullptr,
+                     nullptr, nullptr, 0, F, dtype, w.chunk_ws, w.chunk_bytes, st, &hx);
+    side_join(st, side);  // the call's work is complete in the caller's stream only once the side branch is
+    return rc;
 }
 
 }  // extern "C"

@@ -475,9 +475,8 @@ struct TierStreams {
 static std::mutex g_tier_mutex;
 static TierStreams g_tier[64];
 
-template <class Long, class Warp, class Sub>
-static void run_row_tiers(cudaStream_t st, Long run_long, Warp run_warp, Sub run_sub) {
-    std::lock_guard<std::mutex> lock(g_tier_mutex);  // one host thread at a time forks and joins through the shared events
+// the current device's helper streams, created on first use; nullptr if they cannot be had (call with the mutex held)
+static TierStreams* tier_streams() {
     int dev = -1;
     TierStreams* t = nullptr;
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
@@ -493,6 +492,33 @@ static void run_row_tiers(cudaStream_t st, Long run_long, Warp run_warp, Sub run
         }
         if (t->state != 1) t = nullptr;
     }
+    return t;
+}
+
+// A side branch of the caller's stream: work enqueued on the returned stream starts after everything enqueued on
+// st so far; side_join makes st wait for it.  Returns st itself if no helper stream is available.
+cudaStream_t side_fork(cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_tier_mutex);
+    TierStreams* t = tier_streams();
+    if (!t || cudaEventRecord(t->fork, st) != cudaSuccess || cudaStreamWaitEvent(t->s[0], t->fork, 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return st;
+    }
+    return t->s[0];
+}
+void side_join(cudaStream_t st, cudaStream_t side) {
+    if (side == st) return;
+    std::lock_guard<std::mutex> lock(g_tier_mutex);
+    TierStreams* t = tier_streams();
+    if (!t) return;
+    cudaEventRecord(t->join[0], side);
+    cudaStreamWaitEvent(st, t->join[0], 0);
+}
+
+template <class Long, class Warp, class Sub>
+static void run_row_tiers(cudaStream_t st, Long run_long, Warp run_warp, Sub run_sub) {
+    std::lock_guard<std::mutex> lock(g_tier_mutex);  // one host thread at a time forks and joins through the shared events
+    TierStreams* t = tier_streams();
     if (!t || cudaEventRecord(t->fork, st) != cudaSuccess || cudaStreamWaitEvent(t->s[0], t->fork, 0) != cudaSuccess ||
         cudaStreamWaitEvent(t->s[1], t->fork, 0) != cudaSuccess) {
         (void)cudaGetLastError();

@@ -74,6 +74,9 @@ SIGNATURES = {
     "gnn_edge_dot": (_INT, [_CSR, _VP, _VP, _INT, _INT, _INT, _VP, _VP]),
     "gnn_edge_dot_backward_workspace": (_SZ, [_I64, _INT, _INT]),
     "gnn_edge_dot_backward": (_INT, [_CSR, _VP, _VP, _VP, _INT, _INT, _INT, _VP, _VP, _VP, _SZ, _VP]),
+    "gnn_gatv2_logits": (_INT, [_CSR, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP]),
+    "gnn_gatv2_logits_backward_workspace": (_SZ, [_I32, _INT, _INT]),
+    "gnn_gatv2_logits_backward": (_INT, [_CSR, _VP, _VP, _VP, _VP, _INT, _INT, _INT, _F, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "gnn_merge_edge_lists": (_INT, [_SEG, _INT, _VP, _VP, _VP, _VP]),
     "gnn_segment_coef": (_INT, [_CSR, _VP, _VP, _VP, _INT, _VP, _VP, _VP]),
     "gnn_gather": (_INT, [_VP, _I64, _VP, _I32, _INT, _INT, _VP, _VP]),
@@ -388,6 +391,28 @@ def edge_dot_backward(g: Graph, Xj, Xi, ds_csr, H=1, want_dXj=True, want_dXi=Tru
         ws = torch.empty(load().gnn_edge_dot_backward_workspace(g.E, H, F // H), dtype=torch.uint8, device=Xj.device)
     _check(load().gnn_edge_dot_backward(g.ref, _p(Xj), _p(Xi), _pf32(ds_csr, "ds_csr"), H, F // H, _dtype(Xj), _p(dXj), _p(dXi), _p(ws), ws.numel(), _stream()))
     return dXj, dXi
+
+
+def gatv2_logits(g: Graph, Xl, Xr, a, H, slope=0.2):
+    """s[p,h] = sum_c a[h,c] * LeakyReLU(Xl[col[p],h,c] + Xr[row(p),h,c]) -> float32 [E,H], CSR order."""
+    Xl, Xr = _dev(Xl), _dev(Xr)
+    F = Xl.shape[1]
+    s = torch.empty((max(g.E, 1), H), dtype=torch.float32, device=Xl.device)
+    _check(load().gnn_gatv2_logits(g.ref, _p(Xl), _p(Xr), _pf32(a, "a"), H, F // H, _dtype(Xl), float(slope), _p(s), _stream()))
+    return s[:g.E]
+
+
+def gatv2_logits_backward(g: Graph, Xl, Xr, a, ds_csr, H, slope=0.2, ws=None):
+    """-> (dXl, dXr, da)"""
+    Xl, Xr = _dev(Xl), _dev(Xr)
+    N, F = Xl.shape
+    dXl, dXr = torch.empty_like(Xl), torch.empty_like(Xr)
+    da = torch.empty((H, F // H), dtype=torch.float32, device=Xl.device)
+    if ws is None:
+        ws = torch.empty(load().gnn_gatv2_logits_backward_workspace(N, H, F // H), dtype=torch.uint8, device=Xl.device)
+    _check(load().gnn_gatv2_logits_backward(g.ref, _p(Xl), _p(Xr), _pf32(a, "a"), _pf32(ds_csr, "ds_csr"), H, F // H, _dtype(Xl), float(slope),
+                                            _p(dXl), _p(dXr), _p(da), _p(ws), ws.numel(), _stream()))
+    return dXl, dXr, da
 
 
 # ------------------------------------------------------------------ heterogeneous / temporal graphs

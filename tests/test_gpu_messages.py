@@ -209,3 +209,25 @@ def test_message_argument_errors(gnn):
     with pytest.raises(gnn.GnnError) as err:  # GAT logits are not a propagate message
         gnn.propagate_msg(g, gnn.GAT_LOGIT, X)
     assert err.value.status == 5
+
+
+@pytest.mark.parametrize("dtype,H,C", [("f32", 1, 64), ("f32", 4, 16), ("f32", 8, 16), ("bf16", 8, 32), ("bf16", 2, 64), ("bf16", 1, 40)])
+def test_gatv2_logits_forward_backward(gnn, dtype, H, C):
+    n, src, dst = ragged_graph(140 + H * C)  # a 6000-edge hub (block tier of the backward), short rows, empty rows
+    g = build_graph(gnn, n, src, dst)
+    ref = host_csr(n, src, dst)
+    F = H * C
+    Xl = feats((n, F), dtype, 1500 + F)
+    Xr = feats((n, F), dtype, 1501 + F, stream=1)
+    a = synth.uniform_f32((H, C), -1.0, 1.0, 26)
+    s = gnn.gatv2_logits(g, to_dev(Xl), to_dev(Xr), to_dev(a), H)
+    o, S, _ = oracle.gatv2_logits(src, dst, Xl, Xr, a, H)
+    assert_close(to_host64(s), o[ref["eid"]], S[ref["eid"]], "f32", "GATv2 logits")
+    ds = synth.normal_f32((len(src), H), 27)
+    dXl, dXr, da = gnn.gatv2_logits_backward(g, to_dev(Xl), to_dev(Xr), to_dev(a), to_dev(ds[ref["eid"]]), H)
+    rb = oracle.gatv2_logits_backward(n, src, dst, Xl, Xr, a, H, ds)
+    assert_close(to_host64(dXl), rb["dXl"], rb["SXl"], dtype, "GATv2 dXl")
+    assert_close(to_host64(dXr), rb["dXr"], rb["SXr"], dtype, "GATv2 dXr")
+    assert_close(to_host64(da), rb["da"], rb["Sda"], "f32", "GATv2 da")
+    again = gnn.gatv2_logits_backward(g, to_dev(Xl), to_dev(Xr), to_dev(a), to_dev(ds[ref["eid"]]), H)
+    assert all(np.array_equal(bits(x), bits(y)) for x, y in zip((dXl, dXr, da), again)), "not bit-reproducible"

@@ -690,3 +690,30 @@ def test_epilogue_bias_relu_and_its_backward():
     ids = RNG.choice(Z.size, 30, replace=False)
     assert np.allclose(fd(lambda: (oracle.epilogue(Z, b, "relu") * R).sum(), Z, ids, h=1e-7), dZ.reshape(-1)[ids], atol=1e-6)
     assert np.allclose(fd(lambda: (oracle.epilogue(Z, b, "relu") * R).sum(), b, np.arange(5), h=1e-7), db, atol=1e-6)
+
+
+def test_gatv2_logits_brute_force_linear_case_and_gradient():
+    """GATv2-style logits: brute force by Python loops on a tiny graph; with slope 1 the nonlinearity vanishes and
+    the logit is <a_h, xl_j + xr_i>; gradients against fp64 finite differences."""
+    n, e, H, Cw = 9, 40, 2, 3
+    F = H * Cw
+    src, dst = rand_graph(n, e)
+    Xl, Xr, a = RNG.standard_normal((n, F)), RNG.standard_normal((n, F)), RNG.standard_normal((H, Cw))
+    s, S, _ = oracle.gatv2_logits(src, dst, Xl, Xr, a, H, slope=0.2)
+    ref = np.zeros((e, H))
+    for k in range(e):
+        for h in range(H):
+            for c in range(Cw):
+                z = Xl[src[k], h * Cw + c] + Xr[dst[k], h * Cw + c]
+                ref[k, h] += a[h, c] * (z if z > 0 else 0.2 * z)
+    assert np.allclose(s, ref, atol=1e-13) and (np.abs(s) <= S + 1e-15).all()
+    lin = oracle.gatv2_logits(src, dst, Xl, Xr, a, H, slope=1.0)[0]
+    dense = np.einsum("khc,hc->kh", (Xl[src] + Xr[dst]).reshape(e, H, Cw), a)
+    assert np.allclose(lin, dense, atol=1e-13)
+    ds = RNG.standard_normal((e, H))
+    loss = lambda: (oracle.gatv2_logits(src, dst, Xl, Xr, a, H, slope=0.2)[0] * ds).sum()
+    bw = oracle.gatv2_logits_backward(n, src, dst, Xl, Xr, a, H, ds, slope=0.2)
+    ids = RNG.choice(Xl.size, 30, replace=False)
+    assert np.allclose(fd(loss, Xl, ids), bw["dXl"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    assert np.allclose(fd(loss, Xr, ids), bw["dXr"].reshape(-1)[ids], rtol=1e-6, atol=1e-8)
+    assert np.allclose(fd(loss, a, np.arange(a.size)), bw["da"].reshape(-1), rtol=1e-6, atol=1e-8)
