@@ -138,6 +138,9 @@ gnn_status gnn_permute_edge_data(const int32_t* perm, int64_t E, int width, int 
  * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes, asked for the E of
  * this very call: the edges-per-chunk of the reduction steps with the graph size, so the size is not
  * monotone in E and a workspace sized for a larger graph can be too small for a smaller one.
+ * Which of the two reduction kernels runs (rows walked one by one, or positions first) is a fixed function of
+ * N, E, F, dtype and op (small graphs and, for sums, large graphs of low mean degree take positions first);
+ * results are bit-reproducible for a given graph and shape.
  * Bytes moved per call: at least 4E (+4E with weights) + 8N + 2*N*F*s, at most
  * 4E (+4E) + 8N + (E+N)*F*s when no source row is found in L2. */
 size_t gnn_propagate_fused_workspace(int64_t E, int F, gnn_op op);

@@ -1351,13 +1351,30 @@ static void launch_sddmm(const SddmmParams& P, int lpr, int vpl, cudaStream_t st
 // edges per warp: four slabs once there are enough edges to fill the machine many times over (fewer
 // partial rows to write and re-read), one slab below that, and a half or a quarter slab on graphs so
 // small that whole slabs would leave most SMs without a warp
+#ifndef PF_BIG_E
+#define PF_BIG_E ((int64_t)8 * 1024 * 1024)
+#endif
 static int chunk_edges(int64_t E) {
-    if (E >= (int64_t)8 * 1024 * 1024) return 4 * PF_SLAB;
+    if (E >= PF_BIG_E) return 4 * PF_SLAB;
     if (E >= 512 * 1024) return PF_SLAB;
     return E >= 128 * 1024 ? PF_SLAB / 2 : PF_SLAB / 4;
 }
 static int64_t num_chunks(int64_t E) { return E > 0 ? ceil_div(E, chunk_edges(E)) : 1; }
 static int64_t num_slabs(int64_t E) { return E > 0 ? ceil_div(E, PF_SLAB) : 1; }
+
+// Large graphs of low mean degree: almost every row is a handful of positions, and the position-first kernel
+// (one-slab chunks) beats the row walk at any size.  Measured on uniform random graphs of 1-8 M rows (times in
+// ms, row walk / positions first, 4 M rows): mean degree 4: 64-byte rows 1.34 / 0.70, 256-byte bf16 rows
+// 2.03 / 1.08, 512-byte rows 2.21 / 1.91; mean degree 8: 1.55 / 1.26, 2.92 / 1.93, 3.10 / 3.44; mean degree 16:
+// 2.37 / 2.39, 4.06 / 3.61, 5.46 / 6.48.  fp32 rows walk faster (one predicated loop per row), so their
+// crossover is lower: 256-byte rows 1.70 / 1.08 at mean degree 4, 1.84 / 1.92 at 8.  Graphs with hub rows
+// and a higher mean degree keep the row walk (hubs are where it is strongest).
+static bool flat_by_degree(int mode, int32_t N, int64_t E, int nvec, int elem_bytes) {
+    if (mode != MODE_SUM || nvec > 32 || N <= 0 || E <= 0) return false;
+    const double d = (double)E / (double)N;
+    if (nvec > 16) return d <= 4.0;
+    return elem_bytes == 2 ? d <= 12.0 : d <= 6.0;
+}
 
 struct PfWs {
     int32_t* tail_row;
@@ -1367,7 +1384,10 @@ struct PfWs {
 };
 static PfWs pf_carve(void* ws, int64_t E, int F, bool with_arg) {
     PfWs w;
+    // sums over rows that the position-first kernel can take (at most 512 bytes: F <= 256 whatever the type) may
+    // run on one-slab chunks at any size (flat_by_degree): room for the larger of the two chunk counts
     int64_t nc = num_chunks(E);
+    if (F <= 256 && num_slabs(E) > nc) nc = num_slabs(E);
     char* p = (char*)ws;
     size_t off = 0;
     w.tail_row = (int32_t*)(p + off); off += up256((size_t)nc * 4);
@@ -1407,6 +1427,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     P.rowptr = rowptr; P.col = col; P.w = w; P.X = X; P.out = out; P.argmax = argmax;
     P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
     P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
+    if (flat_by_degree(mode, N, E, nvec, s)) { P.chunk = P.chunk < PF_SLAB ? P.chunk : PF_SLAB; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
     P.wh = nullptr; P.wh_index = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
     if (hx) {

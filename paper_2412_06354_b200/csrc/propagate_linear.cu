@@ -8,8 +8,9 @@
 //                  operand tile in the tensor core's K-major 128-byte-swizzled layout.  A lane group owns
 //                  whole rows, taken from a per-tile counter, and keeps eight row gathers in flight across the
 //                  rows it owns (most rows have a handful of edges); rows longer than PL_LONG positions are
-//                  left to a second phase in which eight warps split each such row and add their partial sums
-//                  in warp order.  Which group reduces a row does not change the order of its additions, so
+//                  left to a second phase in which all gather warps split each such row and add their partial
+//                  sums in warp order (a 1000-position row walked by one lane group, eight gathers at a time,
+//                  would hold its tile for a hundred load latencies).  Which group reduces a row does not change the order of its additions, so
 //                  results are bit-reproducible.
 //   warp 0         issues tcgen05.mma (128 x M x 16, fp32 accumulator in tensor memory; fp32 input: the six
 //                  products of the three-term split with i + j <= 4) on the tile and the resident weights.
@@ -33,8 +34,15 @@ constexpr int PL_GATHER_WARPS = PL_GATHER_WARPS_N;
 constexpr int PL_EPI_WARPS = 4;
 constexpr int PL_THREADS = 32 * (1 + PL_EPI_WARPS + PL_GATHER_WARPS);
 constexpr int PL_U = 8;              // row gathers a lane group keeps in flight
-constexpr int PL_LONG = 1024;        // rows longer than this are split over PL_LONG_WARPS warps
-constexpr int PL_LONG_WARPS = 8;
+#ifndef PL_LONG_N
+#define PL_LONG_N 128
+#endif
+#ifndef PL_LONG_WARPS_N
+#define PL_LONG_WARPS_N 11
+#endif
+constexpr int PL_LONG = PL_LONG_N;   // rows longer than this are split over PL_LONG_WARPS warps
+constexpr int PL_LONG_WARPS = PL_LONG_WARPS_N;
+static_assert(PL_LONG_WARPS <= PL_GATHER_WARPS, "the second phase runs on gather warps");
 constexpr int PL_WINDOW = 2048;      // positions of a tile whose indices (and multipliers) are staged in shared memory
 constexpr int PL_MAX_STAGES = 2;
 constexpr uint32_t PL_SLICE_BYTES = TC_ROWS * 128;  // 64 bf16 columns of the 128-row operand tile

@@ -397,3 +397,40 @@ def test_long_runs_of_rows_without_edges(gnn, dtype, F):
     _, dW = gnn.propagate_fused_backward(g, to_dev(R), "sum", X=Xd, want_dX=False, want_dW=True)
     bw = oracle.propagate_backward("sum", n, src, dst, X, np.ones(e, np.float32), R, want_dX=False, want_dw=True)
     assert_close(to_host64(dW), bw["dw"][ref["eid"]], bw["Sdw"][ref["eid"]], "f32", "dW with long empty runs")
+
+
+@pytest.mark.parametrize("dtype,F", [("bf16", 32), ("f32", 64), ("f32", 128), ("bf16", 128)])
+def test_low_mean_degree_above_8mi_edges_takes_positions_first(gnn, dtype, F):
+    """Graphs of 8 Mi edges and more whose mean degree is a handful run sums on one-slab chunks (positions first)
+    instead of the row walk: forward sum, mean and the backward of the mean, on sampled rows, with a hub cut by
+    hundreds of chunks, rows without edges and a ragged last chunk."""
+    import torch
+    n, e = 2_300_000, 8_600_037
+    rng = np.random.default_rng(91)
+    src = rng.integers(0, n, e).astype(np.int32)
+    dst = rng.integers(0, n - 50_000, e).astype(np.int32)  # the last rows receive nothing
+    dst[:70_000] = 13
+    g = build_graph(gnn, n, src, dst)
+    X = feats((n, F), dtype, 92 + F)
+    R = feats((n, F), dtype, 93 + F, stream=1)
+    w = synth.uniform_f32((e,), 0.0, 1.0, 94)
+    eid = g.eid[:g.E].cpu().numpy()
+    rows = np.unique(np.concatenate([[0, 13, n - 50_001, n - 1], rng.integers(0, n, 3000)]))
+    dev_rows = torch.from_numpy(rows).cuda()
+    oracle.set_threads(8)
+    try:
+        out = gnn.propagate_fused(g, to_dev(X), to_dev(w[eid]), "sum")
+        o, S, _ = oracle.propagate("sum", n, src, dst, X, w, rows=rows)
+        assert_close(to_host64(out[dev_rows]), o, S, dtype, "weighted sum")
+        assert np.array_equal(bits(out), bits(gnn.propagate_fused(g, to_dev(X), to_dev(w[eid]), "sum"))), "not bit-reproducible"
+        assert torch.count_nonzero(out[n - 50_000:]) == 0
+        out = gnn.propagate_fused(g, to_dev(X), None, "mean")
+        o, S, _ = oracle.propagate("mean", n, src, dst, X, None, rows=rows)
+        assert_close(to_host64(out[dev_rows]), o, S, dtype, "mean")
+        # backward of the mean: rows of the transposed form, each gathered row divided by its target's degree
+        dX, _ = gnn.propagate_fused_backward(g, to_dev(R), "mean")
+        srows = np.unique(np.concatenate([[0, n - 1], rng.integers(0, n, 3000)]))
+        bw = oracle.propagate_backward("mean", n, src, dst, None, None, R, rows=srows)
+        assert_close(to_host64(dX[torch.from_numpy(srows).cuda()]), bw["dX"], bw["SdX"], dtype, "backward of the mean")
+    finally:
+        oracle.set_threads(1)
