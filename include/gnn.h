@@ -135,9 +135,10 @@ gnn_status gnn_permute_edge_data(const int32_t* perm, int64_t E, int width, int 
  * scalar per edge, CSR order).  op: SUM; MEAN (sum divided by the number of incoming edges);
  * MAX / MIN (element-wise; argmax int32 [N,F] receives the CSR position of the winner, the
  * smallest position among equal values; may be NULL).  A node with no incoming edge gets 0 and
- * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes, asked for the E of
- * this very call: the edges-per-chunk of the reduction steps with the graph size, so the size is not
- * monotone in E and a workspace sized for a larger graph can be too small for a smaller one.
+ * argmax -1.  X, out: [N,F] of dtype.  ws: at least gnn_propagate_fused_workspace bytes, asked for the E and
+ * the F of this very call: the edges-per-chunk of the reduction steps with the graph size and the row width,
+ * so the size is monotone neither in E nor in F (a workspace sized for a larger graph, or for wider rows, can
+ * be too small; take the maximum over the calls that share it).
  * Which of the two reduction kernels runs (rows walked one by one, or positions first) is a fixed function of
  * N, E, F, dtype and op (small graphs and, for sums, large graphs of low mean degree take positions first);
  * results are bit-reproducible for a given graph and shape.

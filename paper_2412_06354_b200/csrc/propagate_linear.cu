@@ -33,7 +33,10 @@ bool tensor_map_encoder_available();
 constexpr int PL_GATHER_WARPS = PL_GATHER_WARPS_N;
 constexpr int PL_EPI_WARPS = 4;
 constexpr int PL_THREADS = 32 * (1 + PL_EPI_WARPS + PL_GATHER_WARPS);
-constexpr int PL_U = 8;              // row gathers a lane group keeps in flight
+#ifndef PL_U_N
+#define PL_U_N 8
+#endif
+constexpr int PL_U = PL_U_N;         // row gathers a lane group keeps in flight
 #ifndef PL_LONG_N
 #define PL_LONG_N 128
 #endif
