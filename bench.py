@@ -277,6 +277,7 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--cases", default="sweep")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-lanes", type=int, default=3, help="streams per direction of the end-to-end leg (forward calls alternate over this many, backward calls likewise)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-dw", action="store_true", help="skip the separate timing of the edge-weight gradient")
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5],
@@ -482,56 +483,64 @@ def run_e2e(args, torch, gnn, g, plan, hX, hR, w_csr, w_csrT, ws, N, E, fmax, de
     pin = dict(pin_memory=True)
     hXp, hRp = hX, hR  # already pinned
     hXb, hRb = hX.to(torch.bfloat16).pin_memory(), hR.to(torch.bfloat16).pin_memory()
-    # forward calls run on the current stream, backward calls on a second one, each with its own pinned
-    # result buffer, device staging buffers and workspace: the host->device copy of one call overlaps
-    # the device->host copy of the other (the link is full duplex)
-    hout = torch.empty(N * fmax, dtype=torch.float32, **pin)
-    hdX = torch.empty(N * fmax, dtype=torch.float32, **pin)
-    stage = [torch.empty(N * fmax, dtype=torch.float32, device=dev) for _ in range(4)]
-    ws2 = torch.empty_like(ws)
-    s_fwd, s_bwd = torch.cuda.current_stream(), torch.cuda.Stream()
+    # forward calls and backward calls each alternate between `lanes` streams; every stream has its own pinned
+    # result buffer, device staging buffers and workspace, so that independent calls overlap: the host->device
+    # copy of one call runs beside the device->host copy of another (the link is full duplex) and beside the
+    # kernels of a third
+    lanes = max(1, args.e2e_lanes)
+    nl = 2 * lanes
+    hres = [torch.empty(N * fmax, dtype=torch.float32, **pin) for _ in range(nl)]
+    stage = [torch.empty(N * fmax, dtype=torch.float32, device=dev) for _ in range(2 * nl)]
+    wss = [ws] + [torch.empty_like(ws) for _ in range(nl - 1)]
+    s_main = torch.cuda.current_stream()
+    streams = [s_main] + [torch.cuda.Stream() for _ in range(nl - 1)]
     h2d = d2h = 0
     calls = []
-    for F, dt, weighted, _ in plan:
+    for i, (F, dt, weighted, _) in enumerate(plan):
         n = N * F
-        if dt == "f32":
-            hx, hr, ho, hd = hXp[:n].view(N, F), hRp[:n].view(N, F), hout[:n].view(N, F), hdX[:n].view(N, F)
-            st = [b[:n].view(N, F) for b in stage]
-        else:
-            hx, hr = hXb[:n].view(N, F), hRb[:n].view(N, F)
-            ho, hd = hout.view(torch.bfloat16)[:n].view(N, F), hdX.view(torch.bfloat16)[:n].view(N, F)
-            st = [b.view(torch.bfloat16)[:n].view(N, F) for b in stage]
-        calls.append((hx, hr, ho, hd, st, weighted))
+        lf, lb = 2 * (i % lanes), 2 * (i % lanes) + 1  # lanes of this case's forward and backward call
+
+        def view(t):
+            return (t if dt == "f32" else t.view(torch.bfloat16))[:n].view(N, F)
+        hx, hr = (hXp, hRp) if dt == "f32" else (hXb, hRb)
+        hx, hr = hx[:n].view(N, F), hr[:n].view(N, F)
+        calls.append((hx, hr, view(hres[lf]), view(hres[lb]), [view(stage[2 * lf]), view(stage[2 * lf + 1]), view(stage[2 * lb]), view(stage[2 * lb + 1])],
+                      weighted, lf, lb))
         h2d += 2 * hx.numel() * hx.element_size()
-        d2h += 2 * ho.numel() * ho.element_size()
+        d2h += 2 * hx.numel() * hx.element_size()
 
     def step():
-        for hx, hr, ho, hd, st, weighted in calls:
-            gnn.propagate_fused_host(g, hx, w_csr if weighted else None, "sum", ho, st[0], st[1], ws)
-            with torch.cuda.stream(s_bwd):
-                gnn.propagate_fused_backward_host(g, hr, "sum", w_csrT if weighted else None, hd, st[2], st[3], ws2)
+        for hx, hr, ho, hd, st, weighted, lf, lb in calls:
+            with torch.cuda.stream(streams[lf]):
+                gnn.propagate_fused_host(g, hx, w_csr if weighted else None, "sum", ho, st[0], st[1], wss[lf])
+            with torch.cuda.stream(streams[lb]):
+                gnn.propagate_fused_backward_host(g, hr, "sum", w_csrT if weighted else None, hd, st[2], st[3], wss[lb])
 
-    def join():  # the forward stream waits for everything queued on the backward stream
-        s_fwd.wait_stream(s_bwd)
+    def join():  # the main stream waits for everything queued on the others
+        for s_ in streams[1:]:
+            s_main.wait_stream(s_)
 
-    s_bwd.wait_stream(s_fwd)
+    for s_ in streams[1:]:
+        s_.wait_stream(s_main)
     step()
     join()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    t0.record(s_fwd)
-    s_bwd.wait_event(t0)
+    t0.record(s_main)
+    for s_ in streams[1:]:
+        s_.wait_event(t0)
     for _ in range(args.e2e_steps):
         step()
     join()
-    t1.record(s_fwd)
+    t1.record(s_main)
     barrier()
     ms = t0.elapsed_time(t1) / args.e2e_steps
     ms = all_max(ms, dev, world)
     work = sum(E * F for F, _, _, _ in plan)
     return {"value": whole_job_value(work, ms, world), "unit": UNIT, "ms_per_step": ms, "steps": args.e2e_steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "note": "features and gradients copied from pinned host memory, results copied back, per case; forward and backward calls on two streams (copies in both directions overlap); graph and edge weights resident"}
+            "streams": nl,
+            "note": "features and gradients copied from pinned host memory, results copied back, per case; forward and backward calls alternate over %d streams (copies in both directions and kernels of independent calls overlap); graph and edge weights resident" % nl}
 
 
 if __name__ == "__main__":
