@@ -61,6 +61,7 @@ struct PropParams {
     int mean;  // divide the finished row by max(1, row length)
     int chunk;  // edges per warp: 64, 128, 256 or 1024
     int64_t nchunks;
+    int fix_long;           // rows cut into more than FIX_LONG chunks are left to propagate_fixup_long_kernel
     int32_t* tail_row;  // [nchunks] row whose tail partial lives in slot 1, or -1
     float* part_val;    // [nchunks][2][F]
     int32_t* part_arg;  // [nchunks][2][F] (MODE_MAX/MIN)
@@ -545,6 +546,17 @@ propagate_chunk_kernel(const PropParams P) {
     });
 }
 
+// Rows cut into more than FIX_LONG chunks (hub rows of large graphs) are finished by a block each instead of a
+// thread per 16-byte column: one thread walking a hub's hundreds of partial rows pays a load latency per eight of
+// them (45-150 us per call on a graph whose largest row spans 300 chunks, far more on a star-like graph).
+constexpr int FIX_LONG = 64;
+constexpr int FIXL_THREADS = 256;
+constexpr int FIXL_BLOCKS = 592;
+#ifndef FIXL_MIN_CHUNKS_N
+#define FIXL_MIN_CHUNKS_N 16384
+#endif
+constexpr int64_t FIXL_MIN_CHUNKS = FIXL_MIN_CHUNKS_N;  // below this many chunks the extra launch costs more than the walk
+
 // second pass: finish the rows that were cut by chunk boundaries, in ascending chunk order
 template <typename T, int MODE>
 __global__ void propagate_fixup_kernel(const PropParams P) {
@@ -558,6 +570,7 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
     if (r < 0) return;
     const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
     const int64_t c_end = (re - 1) / P.chunk;
+    if (!ARG && P.fix_long && c_end - c > FIX_LONG) return;  // a hub row: propagate_fixup_long_kernel finishes it
     float v[EPC];
     int32_t a[EPC];
     const size_t F = P.F;
@@ -621,6 +634,90 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
         int32_t* ap = P.argmax + (size_t)r * F + (size_t)ci * EPC;
 #pragma unroll
         for (int j = 0; j < EPC; ++j) ap[j] = a[j];
+    }
+}
+
+// Sum modes only.  Block b looks at its share of the chunks; for every row that starts in one of them and is cut
+// into more than FIX_LONG chunks, thread (k, q) adds column float4 q of the partial rows k, k + K, k + 2K, ... of
+// that row (K = 256 / (F/4) walkers per column, four loads in flight each), the K sums are added in walker order,
+// and the row is scaled, given its epilogue and stored as in the kernel above.  The order of the additions is a
+// fixed function of the row's length and F.
+template <typename T, int MODE>
+__global__ void __launch_bounds__(FIXL_THREADS)
+propagate_fixup_long_kernel(const PropParams P) {
+    constexpr int EPC = Chunk<T>::N;
+    __shared__ float4 sums[FIXL_THREADS];
+    __shared__ int todo[64];
+    __shared__ int ntodo;
+    const int tid = threadIdx.x;
+    const int F = P.F, F4 = F / 4;
+    const int K = FIXL_THREADS / F4 > 0 ? FIXL_THREADS / F4 : 1;
+    const int k = tid / F4, q = tid - k * F4;
+    const int64_t per = (P.nchunks + gridDim.x - 1) / gridDim.x;
+    const int64_t c0 = (int64_t)blockIdx.x * per, c1 = c0 + per < P.nchunks ? c0 + per : P.nchunks;
+    for (int64_t cb = c0; cb < c1; cb += 64) {  // 64 chunks at a time: find the long rows, then do them one by one
+        if (tid == 0) ntodo = 0;
+        __syncthreads();
+        if (tid < 64 && cb + tid < c1) {
+            const int32_t r = P.tail_row[cb + tid];
+            if (r >= 0 && (P.rowptr[r + 1] - 1) / P.chunk - (cb + tid) > FIX_LONG) todo[atomicAdd(&ntodo, 1)] = tid;
+        }
+        __syncthreads();
+        const int n = ntodo;
+        for (int i = 0; i < n; ++i) {
+            // rows of one block are independent: the order in which the list was filled does not matter
+            const int64_t c = cb + todo[i];
+            const int32_t r = P.tail_row[c];
+            const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
+            const int64_t span = (re - 1) / P.chunk - c;  // partial rows: (c, tail), then the heads of c + 1 .. c + span
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (k < K && q < F4) {
+                for (int64_t j = k; j <= span; j += 4 * (int64_t)K) {
+                    float4 t[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int64_t jj = j + (int64_t)u * K;
+                        if (jj <= span) {
+                            const size_t slot = jj == 0 ? (size_t)c * 2 + 1 : (size_t)(c + jj) * 2;
+                            t[u] = *(reinterpret_cast<const float4*>(P.part_val + slot * (size_t)F) + q);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (j + (int64_t)u * K <= span) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+                }
+                sums[k * F4 + q] = acc;
+            }
+            __syncthreads();
+            if (tid < P.nvec) {
+                const int ci = tid;
+                float v[EPC];
+#pragma unroll
+                for (int j4 = 0; j4 < EPC / 4; ++j4) {
+                    float4 a = sums[ci * (EPC / 4) + j4];
+                    for (int kk = 1; kk < K; ++kk) {
+                        const float4 b = sums[kk * F4 + ci * (EPC / 4) + j4];
+                        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                    }
+                    v[4 * j4] = a.x; v[4 * j4 + 1] = a.y; v[4 * j4 + 2] = a.z; v[4 * j4 + 3] = a.w;
+                }
+                if (P.mean) {
+                    const float d = (float)(re - rs);
+#pragma unroll
+                    for (int j = 0; j < EPC; ++j) v[j] = v[j] / d;
+                }
+                if (MODE == MODE_HEADSUM && P.epi_l) {
+                    const int h = (ci * EPC) / P.fph;  // a 16-byte chunk lies inside one head
+                    const float el = P.epi_l[(size_t)r * P.H + h], er = P.epi_r[(size_t)r * P.H + h];
+#pragma unroll
+                    for (int j = 0; j < EPC; ++j) v[j] += el * P.epi_a[ci * EPC + j] + er * P.epi_b[ci * EPC + j];
+                }
+                row_epilogue<T>(P, r, ci, v);
+                char* ob = reinterpret_cast<char*>(P.out) + (size_t)r * P.out_ld + (size_t)ci * 16;
+                *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
+            }
+            __syncthreads();
+        }
     }
 }
 
@@ -1298,6 +1395,7 @@ static void launch_chunks(const PropParams& P, int lpr, int vpl, cudaStream_t st
 #undef GNN_PF_CASE
     const int64_t threads = P.nchunks * P.nvec;
     propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
+    if (P.fix_long) propagate_fixup_long_kernel<T, MODE><<<FIXL_BLOCKS, FIXL_THREADS, 0, st>>>(P);
 }
 
 // sum / mean / max / min over rows of at most 512 bytes on graphs small enough for one-slab chunks
@@ -1313,6 +1411,7 @@ static void launch_flat(const PropParams& P, int lpr, cudaStream_t st) {
     }
     const int64_t threads = P.nchunks * P.nvec;
     propagate_fixup_kernel<T, MODE><<<(int)ceil_div(threads, 256), 256, 0, st>>>(P);
+    if (P.fix_long) propagate_fixup_long_kernel<T, MODE><<<FIXL_BLOCKS, FIXL_THREADS, 0, st>>>(P);
 }
 
 template <typename T>
@@ -1437,6 +1536,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
     if (flat_by_degree(mode, N, E, nvec, s)) { P.chunk = P.chunk < PF_SLAB ? P.chunk : PF_SLAB; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
+    P.fix_long = (!with_arg && P.nchunks >= FIXL_MIN_CHUNKS) ? 1 : 0;
     P.wh = nullptr; P.wh_index = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
     if (hx) {
         const int epc = 16 / s;
