@@ -100,6 +100,17 @@ size_t gnn_coo_to_csr_workspace(int32_t N, int64_t E);
 gnn_status gnn_coo_to_csr(int32_t N, int64_t E, const int32_t* src, const int32_t* dst,
                           gnn_csr* out, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* Check of a gnn_csr that did not come from gnn_coo_to_csr (a caller who converts the sparse adjacency form of
+ * Sec. 3 "Graph Data Structures" elsewhere): row pointers from 0 to E and non-decreasing, node and edge indices
+ * in range, eid / eidT / t2f permutations, edge ids ascending inside every row (the order gnn_coo_to_csr
+ * produces, which the deterministic reductions and the argmax convention rely on), and position t2f[q] of the
+ * form by target the same edge as position q of the form by source.  Reads the graph only; every read stays in
+ * bounds whatever the arrays hold.  Returns GNN_OK, or GNN_ERR_INVALID_ARG with the failed checks named in
+ * gnn_last_error_string().  Synchronises the stream (once or twice) to read the result.
+ * ws: gnn_csr_validate_workspace(E) bytes of device scratch. */
+size_t gnn_csr_validate_workspace(int64_t E);
+gnn_status gnn_csr_validate(const gnn_csr* g, void* ws, size_t ws_bytes, gnn_stream stream);
+
 /* Degrees (graph utility of Sec. 3 "Graph Data Structures").  transposed == 0: incoming edges
  * per node; != 0: outgoing.  w == NULL: deg_out is int32 [N] (edge counts, duplicates and
  * loops included).  w != NULL: float [N], the sum of w over the row, w in the order of the

@@ -27,6 +27,68 @@ __global__ void validate_coo_kernel(int32_t N, int64_t E, const int32_t* __restr
     if (bad) *flag = 1;  // benign race: every writer stores the same value
 }
 
+// ------------------------------------------------------------------ validation of a caller-built sparse form
+// Bits of the result word; every read stays in bounds whatever the arrays hold (an index is used only after its
+// range check, row look-ups search rowptr[0..N] by position).
+enum : int {
+    CSR_BAD_ROWPTR = 1,     // rowptr / rowptrT: first entry 0, last entry E, non-decreasing
+    CSR_BAD_NODE = 2,       // col / colT outside [0, N)
+    CSR_BAD_EDGE = 4,       // eid / eidT / t2f outside [0, E)
+    CSR_BAD_PERM = 8,       // eid, eidT or t2f holds a value twice
+    CSR_BAD_ORDER = 16,     // edge ids not ascending inside a row (the order that makes the forms unique)
+    CSR_BAD_CROSS = 32,     // the two forms disagree: position t2f[q] is not the same edge as transposed position q
+};
+
+__device__ __forceinline__ int csr_row_of(const int64_t* __restrict__ rowptr, int32_t N, int64_t p) {
+    int lo = 0, hi = N;  // largest i in [0, N) with rowptr[i] <= p (rowptr[0] = 0 <= p when the pointers are sound)
+    while (hi - lo > 1) {
+        const int mid = lo + (hi - lo) / 2;
+        if (rowptr[mid] <= p) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void csr_validate_pointers_kernel(int32_t N, int64_t E, const int64_t* __restrict__ rowptr,
+                                             const int64_t* __restrict__ rowptrT, int* __restrict__ flag) {
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i > N) return;
+    bool bad = false;
+    const int64_t a = rowptr[i], b = rowptrT[i];
+    bad |= a < 0 || a > E || b < 0 || b > E;
+    if (i == 0) bad |= a != 0 || b != 0;
+    if (i == N) bad |= a != E || b != E;
+    if (i < N) bad |= rowptr[i + 1] < a || rowptrT[i + 1] < b;
+    if (bad) atomicOr(flag, CSR_BAD_ROWPTR);
+}
+
+// runs only when the pointers passed: one thread per position of either form
+__global__ void csr_validate_positions_kernel(int32_t N, int64_t E, const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                                              const int32_t* __restrict__ eid, const int64_t* __restrict__ rowptrT,
+                                              const int32_t* __restrict__ colT, const int32_t* __restrict__ eidT,
+                                              const int32_t* __restrict__ t2f, unsigned* __restrict__ seen, int64_t words,
+                                              int* __restrict__ flag) {
+    const int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (p >= E) return;
+    int bad = 0;
+    const int32_t c = col[p], cT = colT[p], e = eid[p], eT = eidT[p], f = t2f[p];
+    if (c < 0 || c >= N || cT < 0 || cT >= N) bad |= CSR_BAD_NODE;
+    const bool e_ok = e >= 0 && e < E, eT_ok = eT >= 0 && eT < E, f_ok = f >= 0 && f < E;
+    if (!e_ok || !eT_ok || !f_ok) bad |= CSR_BAD_EDGE;
+    // each of the three arrays must hold every value once: a bit per value and array
+    if (e_ok && (atomicOr(seen + (e >> 5), 1u << (e & 31)) >> (e & 31)) & 1u) bad |= CSR_BAD_PERM;
+    if (eT_ok && (atomicOr(seen + words + (eT >> 5), 1u << (eT & 31)) >> (eT & 31)) & 1u) bad |= CSR_BAD_PERM;
+    if (f_ok && (atomicOr(seen + 2 * words + (f >> 5), 1u << (f & 31)) >> (f & 31)) & 1u) bad |= CSR_BAD_PERM;
+    // ascending edge ids inside a row, in both forms
+    const int i = csr_row_of(rowptr, N, p), j = csr_row_of(rowptrT, N, p);
+    if (p + 1 < rowptr[i + 1] && e_ok && eid[p + 1] <= e) bad |= CSR_BAD_ORDER;
+    if (p + 1 < rowptrT[j + 1] && eT_ok && eidT[p + 1] <= eT) bad |= CSR_BAD_ORDER;
+    // transposed position p (row j = the edge's source, colT = its target) and position t2f[p] are one edge
+    if (f_ok && eT_ok) {
+        if (eid[f] != eT || col[f] != j || csr_row_of(rowptr, N, f) != cT) bad |= CSR_BAD_CROSS;
+    }
+    if (bad) atomicOr(flag, bad);
+}
+
 // ------------------------------------------------------------------ exclusive scan (uint32)
 // three launches: per-tile sums, scan of the tile sums by one block, per-tile scan + offset
 constexpr int SCAN_THREADS = 256;
@@ -426,6 +488,43 @@ gnn_status gnn_coo_to_csr(int32_t N, int64_t E, const int32_t* src, const int32_
         compose_perm_kernel<<<grid_for(E, 256), 256, 0, st>>>(E, w.kA, out->eidT, out->t2f);
         GNN_CHECK_LAUNCH("t2f");
     }
+    return GNN_OK;
+}
+
+size_t gnn_csr_validate_workspace(int64_t E) {
+    if (E < 0) return 0;
+    return 256 + up256((size_t)3 * (size_t)((E + 31) / 32) * 4);
+}
+
+gnn_status gnn_csr_validate(const gnn_csr* g, void* ws, size_t ws_bytes, gnn_stream stream) {
+    GNN_REQUIRE(g, GNN_ERR_INVALID_ARG, "gnn_csr_validate: null graph");
+    GNN_REQUIRE(g->N >= 0 && g->E >= 0 && g->E <= 0x7FFFFFFFLL - 1, GNN_ERR_INVALID_ARG, "gnn_csr_validate: bad sizes (N=%d, E=%lld)", g->N, (long long)g->E);
+    GNN_REQUIRE(g->rowptr && g->rowptrT, GNN_ERR_INVALID_ARG, "gnn_csr_validate: null row pointers");
+    GNN_REQUIRE(g->E == 0 || (g->col && g->eid && g->colT && g->eidT && g->t2f), GNN_ERR_INVALID_ARG, "gnn_csr_validate: null edge array");
+    const size_t need = gnn_csr_validate_workspace(g->E);
+    GNN_REQUIRE(ws && ws_bytes >= need, GNN_ERR_WORKSPACE_TOO_SMALL, "gnn_csr_validate: workspace of %zu bytes needed", need);
+    cudaStream_t st = as_stream(stream);
+    int* flag = (int*)ws;
+    unsigned* seen = (unsigned*)((char*)ws + 256);
+    const int64_t words = (g->E + 31) / 32;
+    if (cudaMemsetAsync(ws, 0, need, st) != cudaSuccess) GNN_FAIL(GNN_ERR_CUDA, "gnn_csr_validate: memset failed (is ws a device pointer?)");
+    auto read_flag = [&](int* h) {
+        return cudaMemcpyAsync(h, flag, sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
+    };
+    csr_validate_pointers_kernel<<<grid_for((int64_t)g->N + 1, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->rowptrT, flag);
+    GNN_CHECK_LAUNCH("csr_validate_pointers");
+    int h = 0;
+    if (!read_flag(&h)) GNN_FAIL(GNN_ERR_CUDA, "gnn_csr_validate: reading the result failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (h == 0 && g->E > 0 && g->N > 0) {  // the position checks look rows up through the pointers: only once those are sound
+        csr_validate_positions_kernel<<<grid_for(g->E, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->col, g->eid, g->rowptrT, g->colT,
+                                                                           g->eidT, g->t2f, seen, words, flag);
+        GNN_CHECK_LAUNCH("csr_validate_positions");
+        if (!read_flag(&h)) GNN_FAIL(GNN_ERR_CUDA, "gnn_csr_validate: reading the result failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    GNN_REQUIRE(h == 0, GNN_ERR_INVALID_ARG, "gnn_csr_validate: not a sparse form of one edge list:%s%s%s%s%s%s",
+                (h & CSR_BAD_ROWPTR) ? " row pointers (0 .. E, non-decreasing);" : "", (h & CSR_BAD_NODE) ? " node index outside [0, N);" : "",
+                (h & CSR_BAD_EDGE) ? " edge index outside [0, E);" : "", (h & CSR_BAD_PERM) ? " eid / eidT / t2f not a permutation;" : "",
+                (h & CSR_BAD_ORDER) ? " edge ids not ascending inside a row;" : "", (h & CSR_BAD_CROSS) ? " the two forms describe different edges;" : "");
     return GNN_OK;
 }
 

@@ -55,6 +55,8 @@ SIGNATURES = {
     "gnn_version": (_INT, []),
     "gnn_coo_to_csr_workspace": (_SZ, [_I32, _I64]),
     "gnn_coo_to_csr": (_INT, [_I32, _I64, _VP, _VP, _CSR, _VP, _SZ, _VP]),
+    "gnn_csr_validate_workspace": (_SZ, [_I64]),
+    "gnn_csr_validate": (_INT, [_CSR, _VP, _SZ, _VP]),
     "gnn_degree": (_INT, [_CSR, _INT, _VP, _VP, _VP]),
     "gnn_add_self_loops": (_INT, [_I32, _I64, _VP, _VP, _VP, _VP, _VP]),
     "gnn_gcn_norm": (_INT, [_CSR, _VP, _VP, _VP, _VP, _VP]),
@@ -197,6 +199,13 @@ def coo_to_csr(N, src, dst, ws=None) -> Graph:
         ws = torch.empty(need, dtype=torch.uint8, device=src.device)
     _check(load().gnn_coo_to_csr(N, E, _pi(src, torch.int32, "src"), _pi(dst, torch.int32, "dst"), g.ref, _p(ws), ws.numel(), _stream()))
     return g
+
+
+def csr_validate(g: Graph, ws=None):
+    """Raises GnnError (INVALID_ARG, the failed checks in its text) unless g is a sound sparse form."""
+    if ws is None:
+        ws = torch.empty(load().gnn_csr_validate_workspace(g.E), dtype=torch.uint8, device=g.rowptr.device)
+    _check(load().gnn_csr_validate(g.ref, _p(ws), ws.numel(), _stream()))
 
 
 def degree(g: Graph, transposed=False, w=None):
