@@ -48,48 +48,48 @@ TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cl
                   "full-size traffic (better L2 reuse on the reduced matrix); summary under profiles/")
 TRAFFIC_SCALE = 4.0
 TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
-TRAFFIC_KERNEL_SHA256 = "15f4f347b34a6d887acd9fae575dd375d90ec900214abdcfad9e484c7b718fc7"
+TRAFFIC_KERNEL_SHA256 = "50681bf6e8be4806cd28b11f3c1dea1c2865a72ca003e44f128cc8eb82fb8acc"
 TRAFFIC_GB_REDUCED = {
-    "32:bf16:copy_xj:fwd": 0.193,
-    "32:bf16:copy_xj:bwd": 0.194,
-    "32:bf16:e_mul_xj:fwd": 0.315,
-    "32:bf16:e_mul_xj:bwd": 0.317,
-    "64:bf16:copy_xj:fwd": 0.27,
+    "32:bf16:copy_xj:fwd": 0.192,
+    "32:bf16:copy_xj:bwd": 0.191,
+    "32:bf16:e_mul_xj:fwd": 0.316,
+    "32:bf16:e_mul_xj:bwd": 0.315,
+    "64:bf16:copy_xj:fwd": 0.269,
     "64:bf16:copy_xj:bwd": 0.27,
     "64:bf16:e_mul_xj:fwd": 0.395,
     "64:bf16:e_mul_xj:bwd": 0.395,
-    "128:bf16:copy_xj:fwd": 0.599,
-    "128:bf16:copy_xj:bwd": 0.6,
-    "128:bf16:e_mul_xj:fwd": 0.726,
+    "128:bf16:copy_xj:fwd": 0.6,
+    "128:bf16:copy_xj:bwd": 0.599,
+    "128:bf16:e_mul_xj:fwd": 0.727,
     "128:bf16:e_mul_xj:bwd": 0.727,
-    "256:bf16:copy_xj:fwd": 2.002,
-    "256:bf16:copy_xj:bwd": 2.003,
+    "256:bf16:copy_xj:fwd": 2.004,
+    "256:bf16:copy_xj:bwd": 2.004,
     "256:bf16:e_mul_xj:fwd": 2.133,
-    "256:bf16:e_mul_xj:bwd": 2.132,
+    "256:bf16:e_mul_xj:bwd": 2.133,
     "512:bf16:copy_xj:fwd": 4.018,
-    "512:bf16:copy_xj:bwd": 4.014,
+    "512:bf16:copy_xj:bwd": 4.021,
     "512:bf16:e_mul_xj:fwd": 4.277,
-    "512:bf16:e_mul_xj:bwd": 4.274,
-    "32:f32:copy_xj:fwd": 0.257,
+    "512:bf16:e_mul_xj:bwd": 4.281,
+    "32:f32:copy_xj:fwd": 0.256,
     "32:f32:copy_xj:bwd": 0.257,
     "32:f32:e_mul_xj:fwd": 0.382,
-    "32:f32:e_mul_xj:bwd": 0.381,
-    "64:f32:copy_xj:fwd": 0.588,
-    "64:f32:copy_xj:bwd": 0.589,
+    "32:f32:e_mul_xj:bwd": 0.382,
+    "64:f32:copy_xj:fwd": 0.589,
+    "64:f32:copy_xj:bwd": 0.59,
     "64:f32:e_mul_xj:fwd": 0.716,
-    "64:f32:e_mul_xj:bwd": 0.716,
-    "128:f32:copy_xj:fwd": 1.92,
-    "128:f32:copy_xj:bwd": 1.919,
-    "128:f32:e_mul_xj:fwd": 2.049,
-    "128:f32:e_mul_xj:bwd": 2.047,
+    "64:f32:e_mul_xj:bwd": 0.717,
+    "128:f32:copy_xj:fwd": 1.918,
+    "128:f32:copy_xj:bwd": 1.916,
+    "128:f32:e_mul_xj:fwd": 2.048,
+    "128:f32:e_mul_xj:bwd": 2.045,
     "256:f32:copy_xj:fwd": 3.848,
-    "256:f32:copy_xj:bwd": 3.841,
-    "256:f32:e_mul_xj:fwd": 4.108,
+    "256:f32:copy_xj:bwd": 3.843,
+    "256:f32:e_mul_xj:fwd": 4.107,
     "256:f32:e_mul_xj:bwd": 4.102,
-    "512:f32:copy_xj:fwd": 7.676,
-    "512:f32:copy_xj:bwd": 7.684,
-    "512:f32:e_mul_xj:fwd": 8.197,
-    "512:f32:e_mul_xj:bwd": 8.203,
+    "512:f32:copy_xj:fwd": 7.684,
+    "512:f32:copy_xj:bwd": 7.681,
+    "512:f32:e_mul_xj:fwd": 8.202,
+    "512:f32:e_mul_xj:bwd": 8.199,
 }
 TRAFFIC_GB = {k: v * TRAFFIC_SCALE for k, v in TRAFFIC_GB_REDUCED.items()}
 

@@ -1476,6 +1476,17 @@ static int64_t num_slabs(int64_t E) { return E > 0 ? ceil_div(E, PF_SLAB) : 1; }
 // 2.37 / 2.39, 4.06 / 3.61, 5.46 / 6.48.  fp32 rows walk faster (one predicated loop per row), so their
 // crossover is lower: 256-byte rows 1.70 / 1.08 at mean degree 4, 1.84 / 1.92 at 8.  Graphs with hub rows
 // and a higher mean degree keep the row walk (hubs are where it is strongest).
+// Sums over rows of 256 bytes and more on graphs of 0.5-4 M edges: a one-slab chunk of such rows is 64-128 KB of
+// gathers behind one warp, and the graph fills the machine only one to five times, so half slabs balance better
+// (1.36 M edges, 128 features: fp32 sums 129 -> 113 us, backward of the mean 145 -> 125 us, bf16 75 -> 74 us).
+// Not for narrower rows (the 32-byte rows of the attention backward lose 2 %), nor for max / min and the
+// per-head mode (+5..8 %), nor where the mean degree says that hub rows carry the edges: every extra cut of a hub
+// row is one more partial row (R-MAT graph of 1.6 M edges, mean degree 16, 512-byte rows: 148 -> 167 us).
+constexpr int64_t SUM_HALF_SLAB_BELOW = (int64_t)4 * 1024 * 1024;
+static bool sum_half_slab(int mode, int32_t N, int64_t E, int nvec) {
+    return mode == MODE_SUM && nvec >= 16 && nvec <= 32 && E >= 512 * 1024 && E < SUM_HALF_SLAB_BELOW && E <= (int64_t)12 * N;
+}
+
 static bool flat_by_degree(int mode, int32_t N, int64_t E, int nvec, int elem_bytes) {
     if (mode != MODE_SUM || nvec > 32 || N <= 0 || E <= 0) return false;
     const double d = (double)E / (double)N;
@@ -1495,6 +1506,7 @@ static PfWs pf_carve(void* ws, int64_t E, int F, bool with_arg) {
     // run on one-slab chunks at any size (flat_by_degree): room for the larger of the two chunk counts
     int64_t nc = num_chunks(E);
     if (F <= 256 && num_slabs(E) > nc) nc = num_slabs(E);
+    if (E < SUM_HALF_SLAB_BELOW && ceil_div(E, PF_SLAB / 2) > nc) nc = ceil_div(E, PF_SLAB / 2);
     char* p = (char*)ws;
     size_t off = 0;
     w.tail_row = (int32_t*)(p + off); off += up256((size_t)nc * 4);
@@ -1535,6 +1547,7 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     P.gscale_rowptr = gscale_rowptr; P.route_arg = route_arg; P.route_pos = route_pos;
     P.N = N; P.E = E; P.nvec = nvec; P.F = F; P.mean = mean; P.chunk = chunk_edges(E); P.nchunks = num_chunks(E);
     if (flat_by_degree(mode, N, E, nvec, s)) { P.chunk = P.chunk < PF_SLAB ? P.chunk : PF_SLAB; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
+    if (sum_half_slab(mode, N, E, nvec)) { P.chunk = PF_SLAB / 2; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
     P.fix_long = (!with_arg && P.nchunks >= FIXL_MIN_CHUNKS) ? 1 : 0;
     P.wh = nullptr; P.wh_index = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
