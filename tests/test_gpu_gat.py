@@ -118,10 +118,13 @@ def test_gat_attention_workload_full_size(gnn):
         oracle.set_threads(1)
 
 
-def test_gat_more_than_8mi_edges_uses_the_row_walking_kernels(gnn):
+@pytest.mark.parametrize("E", [8_400_000, 17_000_000])
+def test_gat_more_than_8mi_edges_uses_the_row_walking_kernels(gnn, E):
     """8.4 M edges: above the size where the per-head gather, its transposed form (with the permuted
-    coefficients) and the per-head dot products switch from the position-first kernels to the row-walking ones."""
-    n, E, H, C = 200_000, 8_400_000, 4, 8
+    coefficients) and the per-head dot products switch from the position-first kernels to the row-walking ones.
+    17 M edges: more than 16384 chunks, so the hub rows (cut into more than 64 chunks) are finished by the
+    block-per-row fix-up, here with the per-head multipliers and the rank-1 row epilogue of the backward pass."""
+    n, H, C = 200_000, 4, 8
     src, dst = synth.rmat(18, n, E, 4321, symmetric=False)
     Wx = synth.normal_f32((n, H * C), 4322)
     a = (6.0 / (C + 1)) ** 0.5
@@ -129,6 +132,8 @@ def test_gat_more_than_8mi_edges_uses_the_row_walking_kernels(gnn):
     a_d = synth.uniform_f32((H, C), -a, a, 4324)
     oracle.set_threads(8)
     try:
-        run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, "f32", "gat 8.4M edges")
+        g, _ = run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, "f32", "gat %.1fM edges" % (E / 1e6))
+        if E > 16_000_000:
+            assert int(np.diff(g.rowptr.cpu().numpy()).max()) > 65 * 1024 and int(np.diff(g.rowptrT.cpu().numpy()).max()) > 65 * 1024
     finally:
         oracle.set_threads(1)
