@@ -511,12 +511,12 @@ gnn_status gnn_csr_validate(const gnn_csr* g, void* ws, size_t ws_bytes, gnn_str
     auto read_flag = [&](int* h) {
         return cudaMemcpyAsync(h, flag, sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
     };
-    csr_validate_pointers_kernel<<<grid_for((int64_t)g->N + 1, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->rowptrT, flag);
+    csr_validate_pointers_kernel<<<(int)ceil_div((int64_t)g->N + 1, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->rowptrT, flag);
     GNN_CHECK_LAUNCH("csr_validate_pointers");
     int h = 0;
     if (!read_flag(&h)) GNN_FAIL(GNN_ERR_CUDA, "gnn_csr_validate: reading the result failed: %s", cudaGetErrorString(cudaGetLastError()));
     if (h == 0 && g->E > 0 && g->N > 0) {  // the position checks look rows up through the pointers: only once those are sound
-        csr_validate_positions_kernel<<<grid_for(g->E, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->col, g->eid, g->rowptrT, g->colT,
+        csr_validate_positions_kernel<<<(int)ceil_div(g->E, 256), 256, 0, st>>>(g->N, g->E, g->rowptr, g->col, g->eid, g->rowptrT, g->colT,
                                                                            g->eidT, g->t2f, seen, words, flag);
         GNN_CHECK_LAUNCH("csr_validate_positions");
         if (!read_flag(&h)) GNN_FAIL(GNN_ERR_CUDA, "gnn_csr_validate: reading the result failed: %s", cudaGetErrorString(cudaGetLastError()));

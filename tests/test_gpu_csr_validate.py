@@ -95,3 +95,19 @@ def test_each_kind_of_damage_is_named(gnn):
     with pytest.raises(gnn.GnnError) as err:
         gnn.csr_validate(g, ws=torch.empty(64, dtype=torch.uint8, device="cuda"))
     assert err.value.status == 4
+
+
+def test_damage_far_into_a_large_graph_is_found(gnn):
+    """More rows and positions than one wave of threads covers: the check reaches every one of them."""
+    import torch
+    n, e = 1_500_000, 2_600_000
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    src = torch.randint(0, n, (e,), device="cuda", generator=gen, dtype=torch.int32)
+    dst = torch.randint(0, n, (e,), device="cuda", generator=gen, dtype=torch.int32)
+    g = gnn.coo_to_csr(n, src, dst)
+    gnn.csr_validate(g)
+    g.col[e - 3] = n + 5
+    expect(gnn, g, ["node index"])
+    g = gnn.coo_to_csr(n, src, dst)
+    g.rowptrT[n - 1] = g.rowptrT[n] + 1
+    expect(gnn, g, ["row pointers"])
