@@ -280,6 +280,7 @@ def main():
     ap.add_argument("--e2e-lanes", type=int, default=3, help="streams per direction of the end-to-end leg (forward calls alternate over this many, backward calls likewise)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-dw", action="store_true", help="skip the separate timing of the edge-weight gradient")
+    ap.add_argument("--no-probe", action="store_true", help="skip the bare gather loop (the measured L2 -> SM ceiling)")
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5],
                     help="5 (default): the large sweep.  1-4: device times of the layer-level calls of the smaller workloads, warm and after an L2 flush")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -402,6 +403,24 @@ def main():
             dw_ms[(F, dt)] = a.elapsed_time(b) / 3
         del dWbuf
 
+    # ---- the bare gathers of one pass (no rows, no multipliers, no output) per row width: the ceiling that the
+    # L2 -> SM return path sets for the reduction kernels on this index stream, measured here on this machine
+    gather_loop = {}
+    if not args.no_probe:
+        sink = torch.empty(gnn.load().gnn_probe_gather_sink_floats(E), dtype=torch.float32, device=dev)
+        for rb in (64, 128, 256, 512):
+            Xv = X32[:N * (rb // 4)].view(N, rb // 4)
+            for _ in range(3):
+                gnn.probe_gather(g.col[:E], Xv, rb, sink=sink)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(8):
+                gnn.probe_gather(g.col[:E], Xv, rb, sink=sink)
+            b.record(stream)
+            torch.cuda.synchronize()
+            gather_loop[rb] = E * rb / (a.elapsed_time(b) / 8) / 1e6  # GB/s
+        del sink
+
     # ---- per-case breakdown and the roofline of the chunked propagate kernel
     peak, peak_src = measured_peak()
     per_case, tot_ms, tot_comp, tot_gath = [], 0.0, 0.0, 0.0
@@ -418,6 +437,8 @@ def main():
                          "l2_side_model_GBs_fwd": gath / f_ms / 1e6, "compulsory_frac_fwd": comp / f_ms / 1e6 / peak})
         if weighted and (F, dt) in dw_ms:
             per_case[-1]["bwd_dW_ms"] = round(dw_ms[(F, dt)], 4)
+        if gather_loop:  # rows wider than 512 bytes run as 512-byte column slabs
+            per_case[-1]["frac_of_gather_loop_fwd"] = E * F * s / f_ms / 1e6 / gather_loop[min(F * s, 512)]
     # dominant kernel instance = the case with the largest share of the step
     dom = max(per_case, key=lambda c: c["fwd_ms"] + c["bwd_ms"])
     sdom = 2 if dom["dtype"] == "bf16" else 4
@@ -440,6 +461,8 @@ def main():
                 "dram_traffic_GBs": None if traffic is None else traffic * 1e3 / dom["fwd_ms"],
                 "dram_traffic_frac_of_peak": None if traffic is None else traffic * 1e3 / dom["fwd_ms"] / peak,
                 "l2_side_model_GBs": gather_bytes(N, E, dom["F"], sdom, wdom) / dom["fwd_ms"] / 1e6,
+                "gather_loop_GBs": {str(k): v for k, v in gather_loop.items()} or None,
+                "gather_loop_note": "E * row bytes / time of gnn_probe_gather (the gathers of one pass and nothing else) per row width, measured in this run after the timed steps: the L2 -> SM ceiling of this index stream; per_case.frac_of_gather_loop_fwd = gathered bytes of the forward call / time / that ceiling",
                 "l2_side_model_note": "bytes if every edge fetched its row with no reuse, over time: a rate on the L2 -> SM side (it can exceed any HBM peak), not DRAM bandwidth",
                 "all_launches": {"compulsory_GBs": tot_comp / tot_ms / 1e6, "frac": tot_comp / tot_ms / 1e6 / peak,
                                  "l2_side_model_GBs": tot_gath / tot_ms / 1e6,

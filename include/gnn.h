@@ -515,6 +515,15 @@ gnn_status gnn_propagate_linear_backward(const gnn_csr* g, gnn_msg msg, gnn_op o
                                          const float* w_csrT, const void* W, int K, int M, gnn_dtype dtype,
                                          void* dX, void* dW, void* ws, size_t ws_bytes, gnn_stream stream);
 
+/* Measurement aid (no counterpart in the paper): the bare gathers of a fused propagate.  For every position p of
+ * col int32 [E] the 16-byte chunks of row col[p] of X (rows of row_bytes = 64, 128, 256 or 512 bytes, at least
+ * max(col) + 1 of them) are loaded and added up; nothing else is computed and no row is written.  The rate
+ * E * row_bytes / time is the ceiling that the L2 -> SM return path sets for the reduction kernels on that index
+ * stream and row width.  sink: float [gnn_probe_gather_sink_floats(E)], receives one meaningless value per lane. */
+size_t gnn_probe_gather_sink_floats(int64_t E);
+gnn_status gnn_probe_gather(const int32_t* col, int64_t E, const void* X, int32_t N, int row_bytes, float* sink,
+                            gnn_stream stream);
+
 /* Host-buffer variants for callers whose features live in host memory (one call = copy in,
  * compute, copy out; no counterpart in the paper beyond its "transfer the batch to the gpu"
  * step in the training example).  h_X / h_dOut and h_out / h_dX are HOST arrays [N,F] (pinned

@@ -179,6 +179,25 @@ def large_calls():
     return calls
 
 
+def gatherloop_calls():
+    """The bare gathers of one pass over the large graph (no rows, no output) per row width, beside the sum over
+    fp32 rows of the same width."""
+    wl = synth.workload_large_graph()
+    g = gnn.coo_to_csr(wl["N"], to_dev(wl["src"]), to_dev(wl["dst"]))
+    n, E = wl["N"], g.E
+    del wl
+    calls = []
+    sink = torch.empty(gnn.load().gnn_probe_gather_sink_floats(E), dtype=torch.float32, device="cuda")
+    for rb in (64, 128, 256, 512):
+        gen = torch.Generator(device="cuda").manual_seed(rb)
+        X = torch.randn(n, rb // 4, device="cuda", generator=gen)
+        out = torch.empty_like(X)
+        ws = torch.empty(gnn.propagate_fused_workspace(E, rb // 4, "sum"), dtype=torch.uint8, device="cuda")
+        calls.append((f"large graph (N={n}, E={E}) {rb}-byte rows: bare gather loop", lambda X=X, rb=rb: gnn.probe_gather(g.col[:E], X, rb, sink=sink), E * rb))
+        calls.append((f"large graph {rb}-byte fp32 rows: propagate copy_xj+sum", lambda X=X, out=out, ws=ws: gnn.propagate_fused(g, X, None, "sum", out=out, ws=ws), E * rb))
+    return calls
+
+
 def fused_calls():
     """Aggregate -> transform: the fused call beside the two calls it replaces (configs 1, 3 and 4 shapes)."""
     lib = gnn.load()
@@ -213,7 +232,7 @@ def fused_calls():
 
 
 TABLE = {"linear": linear_calls, "fused": fused_calls, "config1": config1_calls, "config2": config2_calls, "config3": config3_calls,
-         "config4": config4_calls, "large": large_calls,
+         "config4": config4_calls, "large": large_calls, "gatherloop": gatherloop_calls,
          # older names: the propagate calls of configs 1-3 together, the attention calls of config 4
          "propagate": lambda: config1_calls() + config2_calls() + config3_calls(), "gat": config4_calls}
 

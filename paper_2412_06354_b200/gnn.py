@@ -55,6 +55,8 @@ SIGNATURES = {
     "gnn_version": (_INT, []),
     "gnn_coo_to_csr_workspace": (_SZ, [_I32, _I64]),
     "gnn_coo_to_csr": (_INT, [_I32, _I64, _VP, _VP, _CSR, _VP, _SZ, _VP]),
+    "gnn_probe_gather_sink_floats": (_SZ, [_I64]),
+    "gnn_probe_gather": (_INT, [_VP, _I64, _VP, _I32, _INT, _VP, _VP]),
     "gnn_csr_validate_workspace": (_SZ, [_I64]),
     "gnn_csr_validate": (_INT, [_CSR, _VP, _SZ, _VP]),
     "gnn_degree": (_INT, [_CSR, _INT, _VP, _VP, _VP]),
@@ -199,6 +201,15 @@ def coo_to_csr(N, src, dst, ws=None) -> Graph:
         ws = torch.empty(need, dtype=torch.uint8, device=src.device)
     _check(load().gnn_coo_to_csr(N, E, _pi(src, torch.int32, "src"), _pi(dst, torch.int32, "dst"), g.ref, _p(ws), ws.numel(), _stream()))
     return g
+
+
+def probe_gather(col, X, row_bytes, sink=None):
+    """The bare gathers of one pass over col (see gnn_probe_gather): returns the sink buffer."""
+    E = col.numel()
+    if sink is None:
+        sink = torch.empty(load().gnn_probe_gather_sink_floats(E), dtype=torch.float32, device=col.device)
+    _check(load().gnn_probe_gather(_pi(col, torch.int32, "col"), E, _p(X), X.shape[0], int(row_bytes), _p(sink), _stream()))
+    return sink
 
 
 def csr_validate(g: Graph, ws=None):
