@@ -135,6 +135,9 @@ bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype);
 gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
                                   cudaStream_t st, const float* bias = nullptr, int relu = 0);
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
+bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
+int linear_tma_f32_dw_partials(int64_t N);
+gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
 int linear_tma_dw_partials(int64_t N);
 gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
 bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
@@ -222,7 +225,11 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         float* part = (float*)((char*)ws + 256);
         int slabs = dw_slabs(N);
         const int64_t km = (int64_t)K * M;
-        if (linear_tma_dw_supported(N, K, M, dtype)) {
+        if (linear_tma_f32_dw_supported(N, K, M, dtype)) {
+            slabs = linear_tma_f32_dw_partials(N);
+            gnn_status rc = linear_tma_f32_dw(X, dY, N, K, M, part, (int*)ws, st);
+            if (rc != GNN_OK) return rc;
+        } else if (linear_tma_dw_supported(N, K, M, dtype)) {
             slabs = linear_tma_dw_partials(N);
             gnn_status rc = linear_tma_dw(X, dY, N, K, M, part, (int*)ws, st);
             if (rc != GNN_OK) return rc;

@@ -714,6 +714,205 @@ bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int b
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// ------------------------------------------------------------------ fp32: dW = X^T * dY on the bf16 tensor cores, pipelined
+// Contraction over the N rows, 32 rows per pipeline slot.  Roles of the persistent CTA:
+//   warp 0      loader: a slot is K/32 + M/32 boxes of 32 rows x 32 fp32 columns (128-byte rows, 128-byte swizzle)
+//               of X and dY, in a ring of shared-memory slots;
+//   warps 2..9  converters: split every value exactly into three bf16 terms and write the levels of both operands
+//               into one of two operand buffers in the canonical no-swizzle layout, MN-major (16-byte chunk c = 8
+//               features or columns of row n at c*512 + (n/8)*128 + (n%8)*16);
+//   warp 1      MMA issuer: 2 k-steps of 16 rows x 6 level pairs per slot, all into one accumulator [128 features x M]
+//               that stays in tensor memory for the whole kernel;
+//   at the end the converter warps write the accumulator as this CTA's fp32 partial [K,M]; the caller sums the
+//   partials in CTA order (fixed order: deterministic).
+// K = 128 features (the MMA's 128 rows), M a multiple of 32 up to 128.  Every wait is bounded.
+constexpr int FD_ROWS = 32;
+constexpr int FD_CONV_WARPS = 8;
+constexpr int FD_THREADS = 32 * (2 + FD_CONV_WARPS);
+constexpr uint32_t FD_BOX_BYTES = FD_ROWS * 128;           // one box: 32 rows x 32 fp32 columns
+constexpr uint32_t FD_SBO = (FD_ROWS / 8) * 128;           // next chunk of 8 features / columns in an operand level
+constexpr int FD_MAX_STAGES = 4;
+
+struct TmaF32DwParams {
+    float* part;  // [gridDim.x][K][M]
+    int64_t N;
+    int K, M;
+    int stages;
+    int tmem_cols;
+    int* status;
+};
+
+__global__ void __launch_bounds__(FD_THREADS, 1)
+linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapD, const TmaF32DwParams P) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * FD_MAX_STAGES + 5];  // f_full[S], f_empty[S], o_full[2], o_empty[2], acc_full
+    __shared__ uint32_t tmem_base_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = P.K, M = P.M, S = P.stages;
+    const int xboxes = K / 32, dboxes = M / 32;
+    const uint32_t slot_bytes = (uint32_t)(xboxes + dboxes) * FD_BOX_BYTES;
+    const uint32_t a_level = (uint32_t)K * FD_ROWS * 2, b_level = (uint32_t)M * FD_ROWS * 2;
+    const uint32_t op_bytes = 3u * (a_level + b_level);
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t ring0 = base, op0 = ring0 + (uint32_t)S * slot_bytes;
+    const uint32_t bar0 = smem_u32(bars);
+    auto f_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto f_empty = [&](int s) { return bar0 + 8u * (uint32_t)(FD_MAX_STAGES + s); };
+    auto o_full = [&](int o) { return bar0 + 8u * (uint32_t)(2 * FD_MAX_STAGES + o); };
+    auto o_empty = [&](int o) { return bar0 + 8u * (uint32_t)(2 * FD_MAX_STAGES + 2 + o); };
+    const uint32_t acc_full = bar0 + 8u * (uint32_t)(2 * FD_MAX_STAGES + 4);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(f_full(s), 1); mbar_init(f_empty(s), FD_CONV_WARPS); }
+        for (int o = 0; o < 2; ++o) { mbar_init(o_full(o), FD_CONV_WARPS); mbar_init(o_empty(o), 1); }
+        mbar_init(acc_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapX)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapD)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const int64_t nslots = (P.N + FD_ROWS - 1) / FD_ROWS;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            const uint64_t stream = policy_evict_first();
+            uint32_t it = 0;
+            for (int64_t t = blockIdx.x; t < nslots; t += gridDim.x, ++it) {
+                const int s = (int)(it % (uint32_t)S);
+                if (!mbar_wait_bounded(f_empty(s), ((it / (uint32_t)S) & 1u) ^ 1u)) { failed = true; break; }
+                mbar_arrive_expect_tx(f_full(s), slot_bytes);  // rows past N arrive as zeros and count all the same
+                const uint32_t dst = ring0 + (uint32_t)s * slot_bytes;
+                for (int b = 0; b < xboxes; ++b) tma_load_2d(dst + (uint32_t)b * FD_BOX_BYTES, &mapX, b * 32, (int)(t * FD_ROWS), f_full(s), stream);
+                for (int b = 0; b < dboxes; ++b) tma_load_2d(dst + (uint32_t)(xboxes + b) * FD_BOX_BYTES, &mapD, b * 32, (int)(t * FD_ROWS), f_full(s), stream);
+            }
+            if (failed) {  // let the copies in flight land before the CTA goes away
+                const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+                for (uint32_t i = first; i < it; ++i) mbar_wait_bounded(f_full((int)(i % (uint32_t)S)), (i / (uint32_t)S) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(M, 1) | (1u << 15);  // A and B both MN-major
+            uint32_t it = 0;
+            for (int64_t t = blockIdx.x; t < nslots; t += gridDim.x, ++it) {
+                const uint32_t o = it & 1u;
+                if (!mbar_wait_bounded(o_full((int)o), (it >> 1) & 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t abuf = op0 + o * op_bytes, bbuf = abuf + 3u * a_level;
+                for (int kk = 0; kk < FD_ROWS / 16; ++kk)
+                    for (int q = 0; q < 6; ++q) {
+                        const uint64_t adesc = make_smem_desc(abuf + (uint32_t)kPairA3[q] * a_level + (uint32_t)kk * 256u, 128, FD_SBO);
+                        const uint64_t bdesc = make_smem_desc(bbuf + (uint32_t)kPairB3[q] * b_level + (uint32_t)kk * 256u, 128, FD_SBO);
+                        mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (it > 0 || kk > 0 || q > 0) ? 1u : 0u);
+                    }
+                mma_commit(o_empty((int)o));
+            }
+            if (!failed) mma_commit(acc_full);
+        }
+    } else {
+        // ------------------------------------------------------------ converters (every warp works on every slot, in order)
+        constexpr int GT = 32 * FD_CONV_WARPS;
+        const int ct = tid - 64;
+        const int xchunks = K / 8, dchunks = M / 8;
+        const int xops = FD_ROWS * xchunks, ops = xops + FD_ROWS * dchunks;
+        uint32_t it = 0;
+        for (int64_t t = blockIdx.x; t < nslots && !failed; t += gridDim.x, ++it) {
+            const int s = (int)(it % (uint32_t)S);
+            const uint32_t o = it & 1u;
+            if (!mbar_wait_bounded(f_full(s), (it / (uint32_t)S) & 1u)) { failed = true; break; }
+            if (!mbar_wait_bounded(o_empty((int)o), ((it >> 1) & 1u) ^ 1u)) { failed = true; break; }
+            tc_fence_after();
+            const uint32_t src0 = ring0 + (uint32_t)s * slot_bytes;
+            const uint32_t abuf = op0 + o * op_bytes, bbuf = abuf + 3u * a_level;
+#pragma unroll 4
+            for (int e = ct; e < ops; e += GT) {
+                // eight consecutive threads take the eight rows of one core matrix: contiguous 16-byte stores
+                const bool isx = e < xops;
+                const int ee = isx ? e : e - xops, chunks = isx ? xchunks : dchunks;
+                const int q = ee >> 3, rg = q / chunks, c8 = q - rg * chunks, r = rg * 8 + (ee & 7);
+                const int bx = (isx ? 0 : xboxes) + (c8 >> 2), kc = c8 & 3;
+                // fp32 row r of the box: 128 bytes, 16-byte chunk c at position c ^ (r % 8)
+                const uint32_t rowa = src0 + (uint32_t)bx * FD_BOX_BYTES + (uint32_t)r * 128u;
+                const uint4 c0 = ld_shared16(rowa + (uint32_t)(((2 * kc) ^ (r & 7)) << 4));
+                const uint4 c1 = ld_shared16(rowa + (uint32_t)(((2 * kc + 1) ^ (r & 7)) << 4));
+                const float x[8] = {__uint_as_float(c0.x), __uint_as_float(c0.y), __uint_as_float(c0.z), __uint_as_float(c0.w),
+                                    __uint_as_float(c1.x), __uint_as_float(c1.y), __uint_as_float(c1.z), __uint_as_float(c1.w)};
+                uint4 lv[3];
+                split8(x, lv);
+                const uint32_t level = isx ? a_level : b_level;
+                const uint32_t dst = (isx ? abuf : bbuf) + (uint32_t)c8 * FD_SBO + (uint32_t)(r >> 3) * 128u + (uint32_t)(r & 7) * 16u;
+#pragma unroll
+                for (int l = 0; l < 3; ++l) st_shared16(dst + (uint32_t)l * level, lv[l]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(f_empty(s)); mbar_arrive(o_full((int)o)); }
+        }
+        // accumulator -> this CTA's partial.  Lane = feature row; warps 2..5 take the lower half of the columns, 6..9 the upper
+        if (!failed && !mbar_wait_bounded(acc_full, 0u)) failed = true;
+        tc_fence_after();
+        if (!failed) {
+            const int quarter = warp & 3, half = (warp - 2) >> 2;
+            const int krow = quarter * 32 + lane;
+            float* prow = P.part + ((size_t)blockIdx.x * K + krow) * M;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            for (int c0 = half * (M / 2); c0 < (half + 1) * (M / 2); c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<float4*>(prow + c0 + 4 * q) = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                                                               __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+            }
+        }
+    }
+    if (failed) atomicExch(P.status, 7);  // GNN_ERR_TIMEOUT
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+}
+
+bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
+    if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - FD_ROWS) return false;
+    if (K != 128 || M % 32 != 0 || M < 32 || M > 128) return false;
+    return encoder() != nullptr;
+}
+
+// every CTA has at least one slot, so every partial is written
+int linear_tma_f32_dw_partials(int64_t N) {
+    const int64_t nslots = (N + FD_ROWS - 1) / FD_ROWS;
+    return (int)(nslots < 148 ? (nslots > 0 ? nslots : 1) : 148);
+}
+
+// writes linear_tma_f32_dw_partials(N) fp32 partials [K,M] to part
+gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
+    const char* who = "gnn_linear_backward (pipelined fp32 tensor-core dW)";
+    GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
+    CUtensorMap mapX, mapD;
+    if (!make_map_f32(&mapX, X, N, K, FD_ROWS) || !make_map_f32(&mapD, dY, N, M, FD_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    TmaF32DwParams P;
+    P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
+    const size_t slot = (size_t)(K / 32 + M / 32) * FD_BOX_BYTES, ops = 2 * 3 * ((size_t)K * FD_ROWS * 2 + (size_t)M * FD_ROWS * 2);
+    int stages = (int)((TM_SMEM_MAX - 1024 - ops) / slot);
+    P.stages = stages > FD_MAX_STAGES ? FD_MAX_STAGES : stages;
+    int cols = 32;
+    while (cols < M) cols <<= 1;
+    P.tmem_cols = cols;
+    gnn_status rc = allow_big_smem(who, (const void*)linear_tma_f32_dw_kernel, 12, TM_SMEM_MAX);
+    if (rc != GNN_OK) return rc;
+    linear_tma_f32_dw_kernel<<<linear_tma_f32_dw_partials(N), FD_THREADS, 1024 + ops + (size_t)P.stages * slot, st>>>(mapX, mapD, P);
+    GNN_CHECK_LAUNCH(who);
+    return GNN_OK;
+}
+
 static size_t tf_fixed_bytes(int Kc, int Mo) {
     return 1024 + (((size_t)3 * Mo * Kc * 2 + 1023) & ~(size_t)1023) + 2 * 3 * (size_t)TF_LEVEL_BYTES + (size_t)TF_EPI_WARPS * 4096;
 }
