@@ -247,7 +247,7 @@ __device__ __forceinline__ void reduce_heads(float (&v)[4 * HV], float* red) {
 }
 
 constexpr int PL_BLOCK = 512;     // threads per long row
-constexpr int PL_LONG_ROW = 256;  // rows above this many positions get a block instead of a warp
+constexpr int PL_LONG_ROW = 1024;  // rows above this many positions get a block instead of a warp (256: +2 % on the attention workload, 2048: +13 %)
 // positions per thread and batch (their loads are all in flight together): 32 head values per thread
 __host__ __device__ constexpr int pl_unroll(int HV) { return HV <= 2 ? 4 : (HV == 4 ? 2 : 1); }
 
