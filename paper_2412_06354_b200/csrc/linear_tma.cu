@@ -725,7 +725,8 @@ bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int b
 //               that stays in tensor memory for the whole kernel;
 //   at the end the converter warps write the accumulator as this CTA's fp32 partial [K,M]; the caller sums the
 //   partials in CTA order (fixed order: deterministic).
-// K = 128 features (the MMA's 128 rows), M a multiple of 32 up to 128.  Every wait is bounded.
+// K a multiple of 32 up to 128 features (the MMA has 128 rows; those past K are zeros), M a multiple of 32 up to 128.
+// Every wait is bounded.
 constexpr int FD_ROWS = 32;
 constexpr int FD_CONV_WARPS = 8;
 constexpr int FD_THREADS = 32 * (2 + FD_CONV_WARPS);
@@ -751,7 +752,8 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
     const int K = P.K, M = P.M, S = P.stages;
     const int xboxes = K / 32, dboxes = M / 32;
     const uint32_t slot_bytes = (uint32_t)(xboxes + dboxes) * FD_BOX_BYTES;
-    const uint32_t a_level = (uint32_t)K * FD_ROWS * 2, b_level = (uint32_t)M * FD_ROWS * 2;
+    // the A operand always has the MMA's 128 feature rows; with K < 128 the rows past K stay zero
+    const uint32_t a_level = 128u * FD_ROWS * 2, b_level = (uint32_t)M * FD_ROWS * 2;
     const uint32_t op_bytes = 3u * (a_level + b_level);
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t ring0 = base, op0 = ring0 + (uint32_t)S * slot_bytes;
@@ -771,6 +773,12 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapD)) : "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
+    if (K < 128) {  // the converters never write the feature rows past K: zero both buffers' A levels once
+        for (int o = 0; o < 2; ++o)
+            for (uint32_t off = (uint32_t)tid * 16u; off < 3u * a_level; off += FD_THREADS * 16u)
+                st_shared16(op0 + (uint32_t)o * op_bytes + off, make_uint4(0u, 0u, 0u, 0u));
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -858,9 +866,9 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
         // accumulator -> this CTA's partial.  Lane = feature row; warps 2..5 take the lower half of the columns, 6..9 the upper
         if (!failed && !mbar_wait_bounded(acc_full, 0u)) failed = true;
         tc_fence_after();
-        if (!failed) {
-            const int quarter = warp & 3, half = (warp - 2) >> 2;
-            const int krow = quarter * 32 + lane;
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int krow = quarter * 32 + lane;
+        if (!failed && quarter * 32 < K) {  // tcgen05.ld is warp-wide: a warp whose 32 feature rows all lie past K skips it as one
             float* prow = P.part + ((size_t)blockIdx.x * K + krow) * M;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
             for (int c0 = half * (M / 2); c0 < (half + 1) * (M / 2); c0 += 16) {
@@ -869,8 +877,9 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
                 tmem_ld_wait();
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<float4*>(prow + c0 + 4 * q) = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                                                               __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                    if (krow < K)
+                        *reinterpret_cast<float4*>(prow + c0 + 4 * q) = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                                                                   __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
             }
         }
     }
@@ -882,7 +891,7 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
 
 bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
     if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - FD_ROWS) return false;
-    if (K != 128 || M % 32 != 0 || M < 32 || M > 128) return false;
+    if (K % 32 != 0 || K < 32 || K > 128 || M % 32 != 0 || M < 32 || M > 128) return false;
     return encoder() != nullptr;
 }
 
@@ -900,7 +909,7 @@ gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, in
     if (!make_map_f32(&mapX, X, N, K, FD_ROWS) || !make_map_f32(&mapD, dY, N, M, FD_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaF32DwParams P;
     P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
-    const size_t slot = (size_t)(K / 32 + M / 32) * FD_BOX_BYTES, ops = 2 * 3 * ((size_t)K * FD_ROWS * 2 + (size_t)M * FD_ROWS * 2);
+    const size_t slot = (size_t)(K / 32 + M / 32) * FD_BOX_BYTES, ops = 2 * 3 * ((size_t)128 * FD_ROWS * 2 + (size_t)M * FD_ROWS * 2);
     int stages = (int)((TM_SMEM_MAX - 1024 - ops) / slot);
     P.stages = stages > FD_MAX_STAGES ? FD_MAX_STAGES : stages;
     int cols = 32;

@@ -28,8 +28,10 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          ("bf16", 300, 48, 112), ("bf16", 257, 40, 24),
          # one row; exactly one tile with K and M off the 64-element boxes; several tiles and slots per CTA
          ("bf16", 1, 64, 64), ("bf16", 128, 208, 240), ("bf16", 40000, 128, 64), ("bf16", 20001, 256, 144),
-         # fp32 dW on the pipelined kernel (K = 128, M a multiple of 32): one row, a ragged last slot of 32 rows, many slots per CTA
-         ("f32", 1, 128, 32), ("f32", 31, 128, 96), ("f32", 33, 128, 64), ("f32", 30017, 128, 128)]
+         # fp32 dW on the pipelined kernel (K and M multiples of 32 up to 128): one row, a ragged last slot of 32 rows, many slots per CTA
+         ("f32", 1, 128, 32), ("f32", 31, 128, 96), ("f32", 33, 128, 64), ("f32", 30017, 128, 128),
+         # ... and with fewer than the 128 feature rows of the MMA
+         ("f32", 500, 32, 128), ("f32", 77, 96, 32), ("f32", 6001, 64, 96)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
