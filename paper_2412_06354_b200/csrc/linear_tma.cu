@@ -715,7 +715,8 @@ bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int b
 }
 
 // ------------------------------------------------------------------ fp32: dW = X^T * dY on the bf16 tensor cores, pipelined
-// Contraction over the N rows, 32 rows per pipeline slot.  Roles of the persistent CTA:
+// Contraction over the N rows, 32 rows per pipeline slot (16 where K or M is 256, so that two operand buffers and a
+// ring still fit shared memory).  Roles of the persistent CTA:
 //   warp 0      loader: a slot is K/32 + M/32 boxes of 32 rows x 32 fp32 columns (128-byte rows, 128-byte swizzle)
 //               of X and dY, in a ring of shared-memory slots;
 //   warps 2..9  converters: split every value exactly into three bf16 terms and write the levels of both operands
@@ -727,17 +728,16 @@ bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int b
 //   partials in CTA order (fixed order: deterministic).
 // K a multiple of 32 up to 128 features (the MMA has 128 rows; those past K are zeros), M a multiple of 32 up to 128.
 // Every wait is bounded.
-constexpr int FD_ROWS = 32;
+constexpr int FD_ROWS_MAX = 32;
 constexpr int FD_CONV_WARPS = 8;
 constexpr int FD_THREADS = 32 * (2 + FD_CONV_WARPS);
-constexpr uint32_t FD_BOX_BYTES = FD_ROWS * 128;           // one box: 32 rows x 32 fp32 columns
-constexpr uint32_t FD_SBO = (FD_ROWS / 8) * 128;           // next chunk of 8 features / columns in an operand level
 constexpr int FD_MAX_STAGES = 4;
 
 struct TmaF32DwParams {
     float* part;  // [gridDim.x][K][M]
     int64_t N;
     int K, M;
+    int rows;  // rows of X / dY per slot: 32 or 16
     int stages;
     int tmem_cols;
     int* status;
@@ -749,11 +749,13 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
     __shared__ __align__(8) uint64_t bars[2 * FD_MAX_STAGES + 5];  // f_full[S], f_empty[S], o_full[2], o_empty[2], acc_full
     __shared__ uint32_t tmem_base_slot;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int K = P.K, M = P.M, S = P.stages;
+    const int K = P.K, M = P.M, S = P.stages, FD_ROWS = P.rows, halves = (K + 127) / 128;
+    const uint32_t FD_BOX_BYTES = (uint32_t)FD_ROWS * 128u;   // one box: FD_ROWS rows x 32 fp32 columns
+    const uint32_t FD_SBO = (uint32_t)(FD_ROWS / 8) * 128u;   // next chunk of 8 features / columns in an operand level
     const int xboxes = K / 32, dboxes = M / 32;
     const uint32_t slot_bytes = (uint32_t)(xboxes + dboxes) * FD_BOX_BYTES;
-    // the A operand always has the MMA's 128 feature rows; with K < 128 the rows past K stay zero
-    const uint32_t a_level = 128u * FD_ROWS * 2, b_level = (uint32_t)M * FD_ROWS * 2;
+    // the A operand always has whole blocks of the MMA's 128 feature rows; with K < 128 the rows past K stay zero
+    const uint32_t a_level = (uint32_t)halves * 128u * FD_ROWS * 2, b_level = (uint32_t)M * FD_ROWS * 2;
     const uint32_t op_bytes = 3u * (a_level + b_level);
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t ring0 = base, op0 = ring0 + (uint32_t)S * slot_bytes;
@@ -773,7 +775,7 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&mapD)) : "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), (uint32_t)P.tmem_cols);
-    if (K < 128) {  // the converters never write the feature rows past K: zero both buffers' A levels once
+    if (K % 128 != 0) {  // the converters never write the feature rows past K: zero both buffers' A levels once
         for (int o = 0; o < 2; ++o)
             for (uint32_t off = (uint32_t)tid * 16u; off < 3u * a_level; off += FD_THREADS * 16u)
                 st_shared16(op0 + (uint32_t)o * op_bytes + off, make_uint4(0u, 0u, 0u, 0u));
@@ -814,12 +816,13 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
                 if (!mbar_wait_bounded(o_full((int)o), (it >> 1) & 1u)) { failed = true; break; }
                 tc_fence_after();
                 const uint32_t abuf = op0 + o * op_bytes, bbuf = abuf + 3u * a_level;
-                for (int kk = 0; kk < FD_ROWS / 16; ++kk)
-                    for (int q = 0; q < 6; ++q) {
-                        const uint64_t adesc = make_smem_desc(abuf + (uint32_t)kPairA3[q] * a_level + (uint32_t)kk * 256u, 128, FD_SBO);
-                        const uint64_t bdesc = make_smem_desc(bbuf + (uint32_t)kPairB3[q] * b_level + (uint32_t)kk * 256u, 128, FD_SBO);
-                        mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (it > 0 || kk > 0 || q > 0) ? 1u : 0u);
-                    }
+                for (int h = 0; h < halves; ++h)  // features [128h, 128h + 128): chunks 16h.., accumulator columns h*M..
+                    for (int kk = 0; kk < FD_ROWS / 16; ++kk)
+                        for (int q = 0; q < 6; ++q) {
+                            const uint64_t adesc = make_smem_desc(abuf + (uint32_t)kPairA3[q] * a_level + (uint32_t)h * 16u * FD_SBO + (uint32_t)kk * 256u, 128, FD_SBO);
+                            const uint64_t bdesc = make_smem_desc(bbuf + (uint32_t)kPairB3[q] * b_level + (uint32_t)kk * 256u, 128, FD_SBO);
+                            mma_bf16_ss(tmem_base + (uint32_t)h * (uint32_t)M, adesc, bdesc, idesc, (it > 0 || kk > 0 || q > 0) ? 1u : 0u);
+                        }
                 mma_commit(o_empty((int)o));
             }
             if (!failed) mma_commit(acc_full);
@@ -867,10 +870,11 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
         if (!failed && !mbar_wait_bounded(acc_full, 0u)) failed = true;
         tc_fence_after();
         const int quarter = warp & 3, half = (warp - 2) >> 2;
-        const int krow = quarter * 32 + lane;
-        if (!failed && quarter * 32 < K) {  // tcgen05.ld is warp-wide: a warp whose 32 feature rows all lie past K skips it as one
+        for (int h = 0; h < halves && !failed; ++h) {
+            const int krow = h * 128 + quarter * 32 + lane;
+            if (h * 128 + quarter * 32 >= K) break;  // tcgen05.ld is warp-wide: a warp whose 32 feature rows all lie past K skips it as one
             float* prow = P.part + ((size_t)blockIdx.x * K + krow) * M;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)h * (uint32_t)M;
             for (int c0 = half * (M / 2); c0 < (half + 1) * (M / 2); c0 += 16) {
                 uint32_t r[16];
                 tmem_ld16(taddr + (uint32_t)c0, r);
@@ -890,14 +894,15 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
 }
 
 bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
-    if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - FD_ROWS) return false;
-    if (K % 32 != 0 || K < 32 || K > 128 || M % 32 != 0 || M < 32 || M > 128) return false;
+    if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - FD_ROWS_MAX) return false;
+    if (K % 32 != 0 || K < 32 || K > 256 || M % 32 != 0 || M < 32 || M > 256) return false;
     return encoder() != nullptr;
 }
 
 // every CTA has at least one slot, so every partial is written
+static int fd_rows(int K, int M) { return (K > 128 || M > 128) ? 16 : 32; }
 int linear_tma_f32_dw_partials(int64_t N) {
-    const int64_t nslots = (N + FD_ROWS - 1) / FD_ROWS;
+    const int64_t nslots = (N + FD_ROWS_MAX - 1) / FD_ROWS_MAX;  // never more CTAs than slots, whichever the slot height
     return (int)(nslots < 148 ? (nslots > 0 ? nslots : 1) : 148);
 }
 
@@ -906,14 +911,15 @@ gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, in
     const char* who = "gnn_linear_backward (pipelined fp32 tensor-core dW)";
     GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
     CUtensorMap mapX, mapD;
-    if (!make_map_f32(&mapX, X, N, K, FD_ROWS) || !make_map_f32(&mapD, dY, N, M, FD_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    const int R = fd_rows(K, M), ka = (K + 127) / 128 * 128;
+    if (!make_map_f32(&mapX, X, N, K, R) || !make_map_f32(&mapD, dY, N, M, R)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaF32DwParams P;
-    P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
-    const size_t slot = (size_t)(K / 32 + M / 32) * FD_BOX_BYTES, ops = 2 * 3 * ((size_t)128 * FD_ROWS * 2 + (size_t)M * FD_ROWS * 2);
+    P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag; P.rows = R;
+    const size_t slot = (size_t)(K / 32 + M / 32) * R * 128, ops = 2 * 3 * ((size_t)ka * R * 2 + (size_t)M * R * 2);
     int stages = (int)((TM_SMEM_MAX - 1024 - ops) / slot);
     P.stages = stages > FD_MAX_STAGES ? FD_MAX_STAGES : stages;
     int cols = 32;
-    while (cols < M) cols <<= 1;
+    while (cols < M * (ka / 128)) cols <<= 1;
     P.tmem_cols = cols;
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_f32_dw_kernel, 12, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;

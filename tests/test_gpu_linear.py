@@ -31,7 +31,9 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          # fp32 dW on the pipelined kernel (K and M multiples of 32 up to 128): one row, a ragged last slot of 32 rows, many slots per CTA
          ("f32", 1, 128, 32), ("f32", 31, 128, 96), ("f32", 33, 128, 64), ("f32", 30017, 128, 128),
          # ... and with fewer than the 128 feature rows of the MMA
-         ("f32", 500, 32, 128), ("f32", 77, 96, 32), ("f32", 6001, 64, 96)]
+         ("f32", 500, 32, 128), ("f32", 77, 96, 32), ("f32", 6001, 64, 96),
+         # ... and up to 256 wide: 16-row slots, two accumulator halves, feature rows past K zero in the second half
+         ("f32", 2049, 256, 256), ("f32", 900, 160, 224), ("f32", 300, 128, 256)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
