@@ -327,7 +327,8 @@ __device__ __forceinline__ uint4 ld_shared16(uint32_t addr) {
 }
 
 struct TmaF32Params {
-    const float* W;  // [Kc,Mo] (b_transposed = 0) or [Mo,Kc] (b_transposed = 1)
+    const float* W;  // [Kc,Mo] (b_transposed = 0) or [Mo,Kc] (b_transposed = 1), rows ldw elements apart
+    int ldw;
     int64_t N;
     int Kc, Mo;
     int b_transposed;
@@ -380,7 +381,7 @@ linear_tma_f32_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
         const int rows = P.b_transposed ? Mo : Kc, chunks = (P.b_transposed ? Kc : Mo) / 8;
         for (int e = tid; e < rows * chunks; e += TF_THREADS) {
             const int q = e >> 3, rg = q / chunks, c = q - rg * chunks, r = rg * 8 + (e & 7);
-            const float4* src = reinterpret_cast<const float4*>(P.W + ((size_t)r * chunks + c) * 8);
+            const float4* src = reinterpret_cast<const float4*>(P.W + (size_t)r * P.ldw + (size_t)c * 8);
             const float4 lo = __ldg(src), hi = __ldg(src + 1);
             const float x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
             uint4 lv[3];
@@ -703,11 +704,16 @@ gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M,
 }
 
 // row-major fp32 matrix [rows, cols]; box = 32 columns (128 bytes, swizzled) x box_rows rows
+// the same for a block of columns of a wider matrix: rows ld elements apart
+static bool make_map_f32_ld(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int ld, int box_rows);
 bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+    return make_map_f32_ld(m, ptr, rows, cols, cols, box_rows);
+}
+static bool make_map_f32_ld(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int ld, int box_rows) {
     EncodeTiledFn enc = encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
     const cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -932,33 +938,53 @@ static size_t tf_fixed_bytes(int Kc, int Mo) {
     return 1024 + (((size_t)3 * Mo * Kc * 2 + 1023) & ~(size_t)1023) + 2 * 3 * (size_t)TF_LEVEL_BYTES + (size_t)TF_EPI_WARPS * 4096;
 }
 
+// widest block of output columns (a multiple of 16) whose three weight levels fit shared memory beside two slices
+static int tf_column_block(int Kc, int Mo) {
+    int mc = Mo;
+    while (mc >= 16 && tf_fixed_bytes(Kc, mc) + 2 * TF_SLICE_BYTES > TM_SMEM_MAX) mc -= 16;
+    return mc >= 16 ? mc : 0;
+}
+
 bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype) {
     if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
     if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
-    if (tf_fixed_bytes(Kc, Mo) + 2 * TF_SLICE_BYTES > TM_SMEM_MAX) return false;
+    if (tf_column_block(Kc, Mo) == 0) return false;
     return encoder() != nullptr;
 }
 
+// Weights too large for shared memory in one piece (3 x Kc x Mo x 2 bytes: 256 x 256, 256 x 128, 192 x 192 ...) run as
+// one launch per block of output columns: X is read once per block, which is still an order of magnitude faster than
+// the FFMA kernel these shapes fell to before.
 gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
                                   cudaStream_t st, const float* bias, int relu) {
     const char* who = "gnn_linear (pipelined fp32 tensor-core path)";
     GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
-    CUtensorMap mapX, mapY;
-    if (!make_map_f32(&mapX, X, N, Kc, TC_ROWS) || !make_map_f32(&mapY, Y, N, Mo, 32)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
-    TmaF32Params P;
-    P.W = (const float*)W; P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag; P.bias = bias; P.relu = relu;
-    const size_t fixed = tf_fixed_bytes(Kc, Mo);
-    int stages = (int)((TM_SMEM_MAX - fixed) / TF_SLICE_BYTES);
-    P.stages = stages > TF_MAX_STAGES ? TF_MAX_STAGES : stages;
-    P.acc_stride = (Mo + 31) & ~31;
-    int cols = 32;
-    while (cols < 2 * P.acc_stride) cols <<= 1;
-    P.tmem_cols = cols;
+    const int block = tf_column_block(Kc, Mo);
+    GNN_REQUIRE(block > 0, GNN_ERR_UNSUPPORTED, "%s: weights do not fit shared memory", who);
+    CUtensorMap mapX;
+    if (!make_map_f32(&mapX, X, N, Kc, TC_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_f32_kernel, 6, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;
     const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
-    linear_tma_f32_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TF_THREADS, fixed + (size_t)P.stages * TF_SLICE_BYTES, st>>>(mapX, mapY, P);
-    GNN_CHECK_LAUNCH(who);
+    for (int c0 = 0; c0 < Mo; c0 += block) {
+        const int mc = Mo - c0 < block ? Mo - c0 : block;
+        CUtensorMap mapY;
+        if (!make_map_f32_ld(&mapY, (const float*)Y + c0, N, mc, Mo, 32)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+        TmaF32Params P;
+        // stored [Kc,Mo]: a block of columns starts c0 elements into every row; stored [Mo,Kc]: a block of rows
+        P.W = b_transposed ? (const float*)W + (size_t)c0 * Kc : (const float*)W + c0;
+        P.ldw = b_transposed ? Kc : Mo;
+        P.N = N; P.Kc = Kc; P.Mo = mc; P.b_transposed = b_transposed; P.status = d_flag; P.bias = bias ? bias + c0 : nullptr; P.relu = relu;
+        const size_t fixed = tf_fixed_bytes(Kc, mc);
+        int stages = (int)((TM_SMEM_MAX - fixed) / TF_SLICE_BYTES);
+        P.stages = stages > TF_MAX_STAGES ? TF_MAX_STAGES : stages;
+        P.acc_stride = (mc + 31) & ~31;
+        int cols = 32;
+        while (cols < 2 * P.acc_stride) cols <<= 1;
+        P.tmem_cols = cols;
+        linear_tma_f32_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TF_THREADS, fixed + (size_t)P.stages * TF_SLICE_BYTES, st>>>(mapX, mapY, P);
+        GNN_CHECK_LAUNCH(who);
+    }
     return GNN_OK;
 }
 
