@@ -561,7 +561,8 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int K = P.K, M = P.M, S = P.stages;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const int xboxes = K / 64, dboxes = (M + 63) / 64, halves = K / 128;
+    // whole blocks of the MMA's 128 feature rows: boxes that start past column K arrive as zeros
+    const int halves = (K + 127) / 128, xboxes = 2 * halves, dboxes = (M + 63) / 64;
     const uint32_t slot_bytes = (uint32_t)(xboxes + dboxes) * DW_BOX_BYTES;
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
@@ -632,6 +633,7 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
             // stages 32 feature rows x 32 columns of fp32 there and sends them with a bulk tensor store
             const uint32_t stg = base + (uint32_t)ew * 4096u;
             for (int h = 0; h < halves; ++h) {
+                if (h * 128 + quarter * 32 >= K) break;  // feature rows past K (K is a multiple of 32): the next CTA's rows of the partial matrix
                 const int prow0 = (int)blockIdx.x * K + h * 128 + quarter * 32;  // row of the [parts*K, M] partial matrix
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * M);
                 for (int cb = half; cb * 32 < M; cb += 2) {
@@ -669,7 +671,7 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
 
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
     if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
-    if ((K != 128 && K != 256) || M % 16 != 0 || M < 16 || M > 256) return false;
+    if (K % 32 != 0 || K < 32 || K > 256 || M % 16 != 0 || M < 16 || M > 256) return false;
     return encoder() != nullptr;
 }
 
@@ -690,11 +692,11 @@ gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M,
         GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaDwParams P;
     P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag;
-    const size_t slot = (size_t)(K / 64 + (M + 63) / 64) * DW_BOX_BYTES;
+    const size_t slot = (size_t)(2 * ((K + 127) / 128) + (M + 63) / 64) * DW_BOX_BYTES;
     int stages = (int)((TM_SMEM_MAX - 1024) / slot);
     P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
     int cols = 32;
-    while (cols < M * (K / 128)) cols <<= 1;
+    while (cols < M * ((K + 127) / 128)) cols <<= 1;
     P.tmem_cols = cols;
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_dw_kernel, 5, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;

@@ -33,7 +33,9 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          # ... and with fewer than the 128 feature rows of the MMA
          ("f32", 500, 32, 128), ("f32", 77, 96, 32), ("f32", 6001, 64, 96),
          # ... and up to 256 wide: 16-row slots, two accumulator halves, feature rows past K zero in the second half
-         ("f32", 2049, 256, 256), ("f32", 900, 160, 224), ("f32", 300, 128, 256)]
+         ("f32", 2049, 256, 256), ("f32", 900, 160, 224), ("f32", 300, 128, 256),
+         # bf16 dW with K off the 128-row blocks of the MMA (boxes past column K arrive as zeros)
+         ("bf16", 5000, 192, 192), ("bf16", 1234, 96, 80), ("bf16", 777, 224, 256), ("bf16", 40, 32, 16)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
