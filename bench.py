@@ -48,48 +48,48 @@ TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cl
                   "full-size traffic (better L2 reuse on the reduced matrix); summary under profiles/")
 TRAFFIC_SCALE = 4.0
 TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
-TRAFFIC_KERNEL_SHA256 = "50681bf6e8be4806cd28b11f3c1dea1c2865a72ca003e44f128cc8eb82fb8acc"
+TRAFFIC_KERNEL_SHA256 = "effb35ed55c1c35edf6d33bb613429287dfddc12a789daf14c7e88164d4be5a5"
 TRAFFIC_GB_REDUCED = {
     "32:bf16:copy_xj:fwd": 0.192,
-    "32:bf16:copy_xj:bwd": 0.191,
-    "32:bf16:e_mul_xj:fwd": 0.316,
+    "32:bf16:copy_xj:bwd": 0.19,
+    "32:bf16:e_mul_xj:fwd": 0.315,
     "32:bf16:e_mul_xj:bwd": 0.315,
-    "64:bf16:copy_xj:fwd": 0.269,
+    "64:bf16:copy_xj:fwd": 0.27,
     "64:bf16:copy_xj:bwd": 0.27,
     "64:bf16:e_mul_xj:fwd": 0.395,
     "64:bf16:e_mul_xj:bwd": 0.395,
     "128:bf16:copy_xj:fwd": 0.6,
-    "128:bf16:copy_xj:bwd": 0.599,
-    "128:bf16:e_mul_xj:fwd": 0.727,
-    "128:bf16:e_mul_xj:bwd": 0.727,
+    "128:bf16:copy_xj:bwd": 0.6,
+    "128:bf16:e_mul_xj:fwd": 0.726,
+    "128:bf16:e_mul_xj:bwd": 0.726,
     "256:bf16:copy_xj:fwd": 2.004,
     "256:bf16:copy_xj:bwd": 2.004,
     "256:bf16:e_mul_xj:fwd": 2.133,
     "256:bf16:e_mul_xj:bwd": 2.133,
-    "512:bf16:copy_xj:fwd": 4.018,
-    "512:bf16:copy_xj:bwd": 4.021,
+    "512:bf16:copy_xj:fwd": 4.017,
+    "512:bf16:copy_xj:bwd": 4.022,
     "512:bf16:e_mul_xj:fwd": 4.277,
-    "512:bf16:e_mul_xj:bwd": 4.281,
+    "512:bf16:e_mul_xj:bwd": 4.28,
     "32:f32:copy_xj:fwd": 0.256,
     "32:f32:copy_xj:bwd": 0.257,
-    "32:f32:e_mul_xj:fwd": 0.382,
+    "32:f32:e_mul_xj:fwd": 0.381,
     "32:f32:e_mul_xj:bwd": 0.382,
     "64:f32:copy_xj:fwd": 0.589,
-    "64:f32:copy_xj:bwd": 0.59,
-    "64:f32:e_mul_xj:fwd": 0.716,
+    "64:f32:copy_xj:bwd": 0.589,
+    "64:f32:e_mul_xj:fwd": 0.717,
     "64:f32:e_mul_xj:bwd": 0.717,
     "128:f32:copy_xj:fwd": 1.918,
-    "128:f32:copy_xj:bwd": 1.916,
-    "128:f32:e_mul_xj:fwd": 2.048,
-    "128:f32:e_mul_xj:bwd": 2.045,
-    "256:f32:copy_xj:fwd": 3.848,
-    "256:f32:copy_xj:bwd": 3.843,
+    "128:f32:copy_xj:bwd": 1.915,
+    "128:f32:e_mul_xj:fwd": 2.047,
+    "128:f32:e_mul_xj:bwd": 2.044,
+    "256:f32:copy_xj:fwd": 3.849,
+    "256:f32:copy_xj:bwd": 3.844,
     "256:f32:e_mul_xj:fwd": 4.107,
-    "256:f32:e_mul_xj:bwd": 4.102,
-    "512:f32:copy_xj:fwd": 7.684,
-    "512:f32:copy_xj:bwd": 7.681,
-    "512:f32:e_mul_xj:fwd": 8.202,
-    "512:f32:e_mul_xj:bwd": 8.199,
+    "256:f32:e_mul_xj:bwd": 4.1,
+    "512:f32:copy_xj:fwd": 7.683,
+    "512:f32:copy_xj:bwd": 7.679,
+    "512:f32:e_mul_xj:fwd": 8.201,
+    "512:f32:e_mul_xj:bwd": 8.198,
 }
 TRAFFIC_GB = {k: v * TRAFFIC_SCALE for k, v in TRAFFIC_GB_REDUCED.items()}
 

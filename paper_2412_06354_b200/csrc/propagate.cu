@@ -484,8 +484,14 @@ struct Walker {
     }
 };
 
+// max / min (value and winner per element): blocks per SM measured on a 12 M-edge R-MAT graph, forward time in us at
+// 2 / 3 / 4 blocks: fp32 64-byte rows 479 / 458 / 440, 256-byte 754 / 684 / 692, 512-byte 954 / 873 / 891; bf16 32-byte
+// rows 823 / 655 / 623, 128-byte 861 / 710 / 677, 256-byte 1024 / 1060 / 1138, 512-byte 1346 / 1341 / 1383
+__host__ __device__ constexpr int pf_arg_blocks(int lpr, int elem_bytes) { return lpr <= 8 ? 4 : (elem_bytes == 4 ? 3 : 2); }
+
 template <typename T, int LPR, int VPL, int MODE>
-__global__ void __launch_bounds__(PF_WARPS * 32, (VPL == 1 && (MODE == MODE_SUM || MODE == MODE_HEADSUM)) ? (LPR <= PF_NARROW_LPR ? PF_MIN_BLOCKS_NARROW : PF_MIN_BLOCKS) : 2)
+__global__ void __launch_bounds__(PF_WARPS * 32, (VPL == 1 && (MODE == MODE_SUM || MODE == MODE_HEADSUM)) ? (LPR <= PF_NARROW_LPR ? PF_MIN_BLOCKS_NARROW : PF_MIN_BLOCKS)
+                  : ((VPL == 1 && (MODE == MODE_MAX || MODE == MODE_MIN)) ? pf_arg_blocks(LPR, (int)sizeof(T)) : 2))
 propagate_chunk_kernel(const PropParams P) {
     using W = Walker<T, LPR, VPL, MODE>;
     __shared__ SlabSmem s_slab[PF_WARPS];
