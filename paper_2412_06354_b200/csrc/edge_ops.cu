@@ -11,6 +11,26 @@ __device__ __forceinline__ int row_of_position(const int64_t* rowptr, int N, int
     return lower_bound_i64(rowptr, N + 1, p + 1) - 1;
 }
 
+// Row of position p for a thread whose positions only grow: a block owns a contiguous span of (position, chunk) pairs,
+// so from one step to the next a thread's position moves on by blockDim / chunks-per-position and its row by a step or
+// two.  A full search per 16-byte chunk made the calls below run at a sixth of the memory rate; now there is one full
+// search per thread, and another only where more than eight rows (a run of empty ones) are skipped at once.
+__device__ __forceinline__ int advance_row(const int64_t* __restrict__ rowptr, int N, int row, int64_t p) {
+    if (row < 0) return row_of_position(rowptr, N, p);
+#pragma unroll 1
+    for (int k = 0; k < 8; ++k) {
+        if (rowptr[row + 1] > p) return row;  // rowptr[row] <= p holds throughout
+        ++row;
+    }
+    return rowptr[row + 1] > p ? row : row_of_position(rowptr, N, p);
+}
+// first pair of this block's span and one past its last; spans are multiples of the block size
+__device__ __forceinline__ void block_span(int64_t total, int64_t* t0, int64_t* t1) {
+    const int64_t per = ((total + gridDim.x - 1) / gridDim.x + blockDim.x - 1) / blockDim.x * blockDim.x;
+    *t0 = (int64_t)blockIdx.x * per;
+    *t1 = *t0 + per < total ? *t0 + per : total;
+}
+
 // Grid-stride walk over (position, 16-byte chunk) pairs t = p*nvec + ci without a division per step:
 // one 64-bit division when the thread starts, then p and ci advance by the quotient and remainder of
 // the stride.
@@ -65,12 +85,13 @@ __global__ void apply_edges_mul_kernel(const int32_t* __restrict__ col, int64_t 
 __global__ void gat_logit_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, int N,
                                  int64_t E, int H, const float* __restrict__ al, const float* __restrict__ ar,
                                  float slope, float* __restrict__ s) {
-    int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * H;
-    for (PosChunk q(t, stride, H); t < total; t += stride, q.next()) {
-        const int64_t p = q.p;
-        const int h = q.ci;
-        const int i = row_of_position(rowptr, N, p);
+    int64_t t0, t1;
+    block_span(E * H, &t0, &t1);
+    int i = -1;
+    for (int64_t t = t0 + threadIdx.x; t < t1; t += blockDim.x) {
+        const int64_t p = t / H;
+        const int h = (int)(t - p * H);
+        i = advance_row(rowptr, N, i, p);
         const float z = al[(size_t)col[p] * H + h] + ar[(size_t)i * H + h];
         s[t] = z > 0.f ? z : slope * z;
     }
@@ -82,12 +103,13 @@ __global__ void aggregate_backward_kernel(const int64_t* __restrict__ rowptr, in
                                           const uint4* __restrict__ dOut, const int32_t* __restrict__ argmax,
                                           int nvec, uint4* __restrict__ dm) {
     constexpr int EPC = Chunk<T>::N;
-    int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x, total = E * nvec;
-    for (PosChunk q(t, stride, nvec); t < total; t += stride, q.next()) {
-        const int64_t p = q.p;
-        const int ci = q.ci;
-        const int i = row_of_position(rowptr, N, p);
+    int64_t t0, t1;
+    block_span(E * nvec, &t0, &t1);
+    int i = -1;
+    for (int64_t t = t0 + threadIdx.x; t < t1; t += blockDim.x) {
+        const int64_t p = t / nvec;
+        const int ci = (int)(t - p * nvec);
+        i = advance_row(rowptr, N, i, p);
         uint4 raw = dOut[(size_t)i * nvec + ci];
         if (op == GNN_SUM) { dm[t] = raw; continue; }
         float x[EPC];
