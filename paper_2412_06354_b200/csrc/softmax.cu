@@ -580,13 +580,17 @@ gnn_status gnn_edge_softmax(const gnn_csr* g, const void* logits_EH, int H, gnn_
     GNN_REQUIRE(g->E == 0 || (logits_EH && alpha_EH), GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
     const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
-    if (dtype == GNN_F32) {
-        edge_softmax_kernel<float, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum);
-        edge_softmax_kernel<float, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum);
-    } else {
-        edge_softmax_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum);
-        edge_softmax_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum);
-    }
+    // the two row tiers write disjoint rows: side by side (the long rows' blocks beside the warps of the short ones)
+    if (dtype == GNN_F32)
+        run_row_tiers(
+            st, [&](cudaStream_t q) { edge_softmax_kernel<float, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum); },
+            [&](cudaStream_t q) { edge_softmax_kernel<float, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum); },
+            [&](cudaStream_t) {});
+    else
+        run_row_tiers(
+            st, [&](cudaStream_t q) { edge_softmax_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum); },
+            [&](cudaStream_t q) { edge_softmax_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum); },
+            [&](cudaStream_t) {});
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
@@ -600,13 +604,16 @@ gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, con
     GNN_REQUIRE(alpha_EH && dAlpha_EH && dLogits_EH, GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
     const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
-    if (dtype == GNN_F32) {
-        edge_softmax_backward_kernel<float, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH);
-        edge_softmax_backward_kernel<float, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH);
-    } else {
-        edge_softmax_backward_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH);
-        edge_softmax_backward_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, st>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH);
-    }
+    if (dtype == GNN_F32)
+        run_row_tiers(
+            st, [&](cudaStream_t q) { edge_softmax_backward_kernel<float, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH); },
+            [&](cudaStream_t q) { edge_softmax_backward_kernel<float, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH); },
+            [&](cudaStream_t) {});
+    else
+        run_row_tiers(
+            st, [&](cudaStream_t q) { edge_softmax_backward_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH); },
+            [&](cudaStream_t q) { edge_softmax_backward_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH); },
+            [&](cudaStream_t) {});
     GNN_CHECK_LAUNCH(who);
     return GNN_OK;
 }
