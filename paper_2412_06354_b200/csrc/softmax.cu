@@ -109,6 +109,149 @@ __device__ __forceinline__ void softmax_bwd_row(const T* alpha, const T* dalpha,
     }
 }
 
+// ---- a warp per row with 16-byte (fp32) / 8-byte (bf16) loads: H = 4, 8, 16 or 32.  A lane takes chunks of four
+// consecutive values; its chunks are 128 values apart, a multiple of H, so the four heads of a lane never change and
+// lanes that are equal modulo H/4 hold the same heads.  Rows of up to 512 values (64 positions at 8 heads) are read
+// once and stay in registers through all steps.
+template <typename T> __device__ __forceinline__ void ld4(const T* p, size_t i, float* v);
+template <> __device__ __forceinline__ void ld4<float>(const float* p, size_t i, float* v) {
+    const float4 q = *reinterpret_cast<const float4*>(p + i);
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+template <> __device__ __forceinline__ void ld4<__nv_bfloat16>(const __nv_bfloat16* p, size_t i, float* v) {
+    const uint2 q = *reinterpret_cast<const uint2*>(p + i);
+    v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xFFFF0000u);
+}
+template <typename T> __device__ __forceinline__ void st4(T* p, size_t i, const float* v);
+template <> __device__ __forceinline__ void st4<float>(float* p, size_t i, const float* v) {
+    *reinterpret_cast<float4*>(p + i) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ __forceinline__ void st4<__nv_bfloat16>(__nv_bfloat16* p, size_t i, const float* v) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    *reinterpret_cast<uint2*>(p + i) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+}
+template <class Op>
+__device__ __forceinline__ void reduce_heads4(float* v, int H) {
+    const int lane = threadIdx.x & 31, lo = H / 4;
+    for (int o = 16; o >= lo; o >>= 1)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[j], o);
+            v[j] = ((lane & o) == 0) ? Op::f(v[j], other) : Op::f(other, v[j]);
+        }
+}
+constexpr int V4_U = 4;  // chunks a lane keeps in registers
+
+template <typename T>
+__device__ __forceinline__ void softmax_row_vec4(const T* __restrict__ s, T* __restrict__ alpha, int64_t a, int64_t b, int H, int row,
+                                                 float* rowmax, float* rowsum) {
+    const int lane = threadIdx.x & 31;
+    const size_t lo = (size_t)a * H;
+    const int nch = (int)(((b - a) * H) >> 2);
+    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, z[4] = {0.f, 0.f, 0.f, 0.f};
+    if (nch <= 32 * V4_U) {
+        float v[V4_U][4];
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch) ld4(s, lo + 4 * (size_t)(lane + 32 * u), v[u]);
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) m[j] = fmaxf(m[j], v[u][j]);
+        reduce_heads4<MaxOp>(m, H);
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { v[u][j] = expf(v[u][j] - m[j]); z[j] += v[u][j]; }
+        reduce_heads4<SumOp>(z, H);
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[u][j] = v[u][j] / z[j];
+                st4(alpha, lo + 4 * (size_t)(lane + 32 * u), v[u]);
+            }
+    } else {
+        float v[4];
+        for (int c = lane; c < nch; c += 32) {
+            ld4(s, lo + 4 * (size_t)c, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) m[j] = fmaxf(m[j], v[j]);
+        }
+        reduce_heads4<MaxOp>(m, H);
+        for (int c = lane; c < nch; c += 32) {
+            ld4(s, lo + 4 * (size_t)c, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) z[j] += expf(v[j] - m[j]);
+        }
+        reduce_heads4<SumOp>(z, H);
+        for (int c = lane; c < nch; c += 32) {
+            ld4(s, lo + 4 * (size_t)c, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = expf(v[j] - m[j]) / z[j];
+            st4(alpha, lo + 4 * (size_t)c, v);
+        }
+    }
+    if (lane < H / 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (rowmax) rowmax[(size_t)row * H + 4 * lane + j] = m[j];
+            if (rowsum) rowsum[(size_t)row * H + 4 * lane + j] = z[j];
+        }
+    }
+}
+
+// ds = alpha * (dalpha - sum_row alpha*dalpha), same lane layout
+template <typename T>
+__device__ __forceinline__ void softmax_bwd_row_vec4(const T* __restrict__ alpha, const T* __restrict__ dalpha, T* __restrict__ ds,
+                                                     int64_t a, int64_t b, int H) {
+    const int lane = threadIdx.x & 31;
+    const size_t lo = (size_t)a * H;
+    const int nch = (int)(((b - a) * H) >> 2);
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    if (nch <= 32 * V4_U) {
+        float al[V4_U][4], da[V4_U][4];
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch) {
+                ld4(alpha, lo + 4 * (size_t)(lane + 32 * u), al[u]);
+                ld4(dalpha, lo + 4 * (size_t)(lane + 32 * u), da[u]);
+            }
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) d[j] = fmaf(al[u][j], da[u][j], d[j]);
+        reduce_heads4<SumOp>(d, H);
+#pragma unroll
+        for (int u = 0; u < V4_U; ++u)
+            if (lane + 32 * u < nch) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) da[u][j] = al[u][j] * (da[u][j] - d[j]);
+                st4(ds, lo + 4 * (size_t)(lane + 32 * u), da[u]);
+            }
+    } else {
+        float x[4], y[4];
+        for (int c = lane; c < nch; c += 32) {
+            ld4(alpha, lo + 4 * (size_t)c, x);
+            ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) d[j] = fmaf(x[j], y[j], d[j]);
+        }
+        reduce_heads4<SumOp>(d, H);
+        for (int c = lane; c < nch; c += 32) {
+            ld4(alpha, lo + 4 * (size_t)c, x);
+            ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) y[j] = x[j] * (y[j] - d[j]);
+            st4(ds, lo + 4 * (size_t)c, y);
+        }
+    }
+}
+
 static __host__ __device__ inline bool head_pow2(int H) { return H >= 1 && H <= 32 && (H & (H - 1)) == 0; }
 
 // Row loops.  LONG = false: every warp strides over the rows and takes the ones of at most
@@ -157,6 +300,8 @@ edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restri
                     T* __restrict__ alpha, float* __restrict__ rowmax, float* __restrict__ rowsum) {
     __shared__ float red[SM_BLOCK];
     __shared__ LongRows lrows;
+    // four heads per lane and 16-byte / 8-byte accesses: H = 4 .. 32, a power of two, and aligned arrays
+    const bool vec4 = H >= 4 && head_pow2(H) && ((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(alpha)) & (4 * sizeof(T) - 1)) == 0;
     for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int row, int64_t a, int64_t b) {
         if (b == a) {
             if ((threadIdx.x & 31) < H) {
@@ -165,7 +310,8 @@ edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restri
             }
             return;
         }
-        if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
+        if (!LONG && vec4) softmax_row_vec4<T>(s, alpha, a, b, H, row, rowmax, rowsum);
+        else if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
         else softmax_row_any<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
     });
 }
@@ -176,8 +322,12 @@ edge_softmax_backward_kernel(const int64_t* __restrict__ rowptr, int N, const T*
                              const T* __restrict__ dalpha, int H, T* __restrict__ ds) {
     __shared__ float red[SM_BLOCK];
     __shared__ LongRows lrows;
+    const bool vec4 = H >= 4 && head_pow2(H) &&
+                      ((reinterpret_cast<uintptr_t>(alpha) | reinterpret_cast<uintptr_t>(dalpha) | reinterpret_cast<uintptr_t>(ds)) & (4 * sizeof(T) - 1)) == 0;
     for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int, int64_t a, int64_t b) {
-        if (b > a) softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
+        if (b == a) return;
+        if (!LONG && vec4) softmax_bwd_row_vec4<T>(alpha, dalpha, ds, a, b, H);
+        else softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
     });
 }
 
