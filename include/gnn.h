@@ -458,10 +458,11 @@ gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_
 
 /* Y = X * W (the Dense layer / the weight of a conv layer in the training example): X [N,K],
  * W [K,M], Y [N,M], all row-major and of dtype, 16-byte aligned.  With K and M multiples of 16
- * (16..256) the product runs on the tensor cores with fp32 accumulation: bf16 directly, fp32 (when
- * the weight matrix is small enough to sit in shared memory three times, e.g. 128x128) by an exact
- * three-term bf16 split of every value, which keeps fp32 accuracy.  Other cases use an fp32 FFMA
- * kernel.  The first call on a device looks up the driver's tensor-map encoder; the calls
+ * (16..256) the product runs on the tensor cores with fp32 accumulation: bf16 directly, fp32 by an exact
+ * three-term bf16 split of every value, which keeps fp32 accuracy (weights that do not fit shared memory
+ * three times, e.g. 256x256, run as one launch per block of output columns).  The weight gradient of
+ * gnn_linear_backward takes the tensor cores for K and M multiples of 32 (bf16: M of 16).  Other cases use an
+ * fp32 FFMA kernel, several times slower.  The first call on a device looks up the driver's tensor-map encoder; the calls
  * themselves allocate nothing.
  * ws: gnn_linear_workspace(N, K, M) bytes; its first 4 bytes are a device status word that the
  * tensor-core path sets to GNN_ERR_TIMEOUT if one of its bounded waits expired (0 otherwise);
