@@ -903,7 +903,8 @@ linear_tma_f32_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_
 
 bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
     if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - FD_ROWS_MAX) return false;
-    if (K % 32 != 0 || K < 32 || K > 256 || M % 32 != 0 || M < 32 || M > 256) return false;
+    if (K % 32 != 0 || K < 32 || K > 512 || M % 32 != 0 || M < 32 || M > 256) return false;
+    if (M * ((K + 127) / 128) > 512) return false;  // one accumulator [128, M] per block of 128 features: 512 columns of tensor memory
     return encoder() != nullptr;
 }
 
@@ -942,14 +943,14 @@ static size_t tf_fixed_bytes(int Kc, int Mo) {
 
 // widest block of output columns (a multiple of 16) whose three weight levels fit shared memory beside two slices
 static int tf_column_block(int Kc, int Mo) {
-    int mc = Mo;
+    int mc = Mo < 256 ? Mo : 256;  // the MMA takes at most 256 columns, two accumulators of them fill tensor memory
     while (mc >= 16 && tf_fixed_bytes(Kc, mc) + 2 * TF_SLICE_BYTES > TM_SMEM_MAX) mc -= 16;
     return mc >= 16 ? mc : 0;
 }
 
 bool linear_tma_f32_supported(int64_t N, int Kc, int Mo, gnn_dtype dtype) {
     if (dtype != GNN_F32 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
-    if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
+    if (Kc % 16 != 0 || Kc < 16 || Kc > 512 || Mo % 16 != 0 || Mo < 16 || Mo > 1024) return false;
     if (tf_column_block(Kc, Mo) == 0) return false;
     return encoder() != nullptr;
 }

@@ -35,7 +35,9 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          # ... and up to 256 wide: 16-row slots, two accumulator halves, feature rows past K zero in the second half
          ("f32", 2049, 256, 256), ("f32", 900, 160, 224), ("f32", 300, 128, 256),
          # bf16 dW with K off the 128-row blocks of the MMA (boxes past column K arrive as zeros)
-         ("bf16", 5000, 192, 192), ("bf16", 1234, 96, 80), ("bf16", 777, 224, 256), ("bf16", 40, 32, 16)]
+         ("bf16", 5000, 192, 192), ("bf16", 1234, 96, 80), ("bf16", 777, 224, 256), ("bf16", 40, 32, 16),
+         # fp32 beyond 256: long contraction (16 slices per tile), many column blocks, four accumulator blocks in dW
+         ("f32", 3000, 512, 64), ("f32", 3000, 64, 512), ("f32", 700, 384, 128), ("f32", 900, 512, 512)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
