@@ -671,7 +671,8 @@ linear_tma_dw_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_cons
 
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype) {
     if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
-    if (K % 32 != 0 || K < 32 || K > 256 || M % 16 != 0 || M < 16 || M > 256) return false;
+    if (K % 32 != 0 || K < 32 || K > 512 || M % 16 != 0 || M < 16 || M > 256) return false;
+    if (M * ((K + 127) / 128) > 512) return false;  // one accumulator [128, M] per block of 128 features: 512 columns of tensor memory
     return encoder() != nullptr;
 }
 

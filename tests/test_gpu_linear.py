@@ -37,7 +37,9 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          # bf16 dW with K off the 128-row blocks of the MMA (boxes past column K arrive as zeros)
          ("bf16", 5000, 192, 192), ("bf16", 1234, 96, 80), ("bf16", 777, 224, 256), ("bf16", 40, 32, 16),
          # fp32 beyond 256: long contraction (16 slices per tile), many column blocks, four accumulator blocks in dW
-         ("f32", 3000, 512, 64), ("f32", 3000, 64, 512), ("f32", 700, 384, 128), ("f32", 900, 512, 512)]
+         ("f32", 3000, 512, 64), ("f32", 3000, 64, 512), ("f32", 700, 384, 128), ("f32", 900, 512, 512),
+         # bf16 dW with up to 512 features (four accumulator blocks)
+         ("bf16", 3000, 512, 64), ("bf16", 2000, 384, 128), ("bf16", 1000, 320, 48)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
