@@ -48,6 +48,7 @@ struct TmaParams {
     int64_t N;
     int Kc, Mo;        // contraction length, output columns
     int b_transposed;
+    int w_box_rows;    // rows of one weight box (a box has at most 256 rows: taller blocks arrive as two boxes)
     int stages;        // ring slots
     int acc_stride;    // tensor-memory columns between the two accumulators
     int tmem_cols;
@@ -99,7 +100,10 @@ linear_tma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (lane == 0) {
             const uint64_t keep = policy_evict_last(), stream = policy_evict_first();
             mbar_arrive_expect_tx(wfull, (uint32_t)wblocks * wblock_bytes);
-            for (int b = 0; b < wblocks; ++b) tma_load_2d(w0 + (uint32_t)b * wblock_bytes, &mapW, b * 64, 0, wfull, keep);
+            const int w_rows = P.b_transposed ? Mo : Kc;
+            for (int b = 0; b < wblocks; ++b)
+                for (int r0 = 0; r0 < w_rows; r0 += P.w_box_rows)  // rows are 128 bytes apart: stacked boxes lie as one taller box would
+                    tma_load_2d(w0 + (uint32_t)b * wblock_bytes + (uint32_t)r0 * 128u, &mapW, b * 64, r0, wfull, keep);
             uint32_t it = 0;
             for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x)
                 for (int j = 0; j < kblocks; ++j, ++it) {
@@ -227,11 +231,14 @@ static EncodeTiledFn encoder() {
 // row-major bf16 matrix [rows, cols]; box = 64 columns (128 bytes, swizzled) x box_rows rows; out-of-range reads give zeros
 bool tensor_map_encoder_available() { return encoder() != nullptr; }
 
-bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) {
+static bool make_map_ld(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int ld, int box_rows);
+bool make_map(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows) { return make_map_ld(m, ptr, rows, cols, cols, box_rows); }
+// a block of columns of a wider matrix: rows ld elements apart
+static bool make_map_ld(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int ld, int box_rows) {
     EncodeTiledFn enc = encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -242,38 +249,59 @@ static size_t tma_w_bytes(int Kc, int Mo, int b_transposed) {
     return b_transposed ? (size_t)((Kc + 63) / 64) * Mo * 128 : (size_t)((Mo + 63) / 64) * Kc * 128;
 }
 
+// widest block of output columns whose weights fit shared memory beside the staging blocks and two slices; the MMA
+// takes at most 256 columns and two accumulators of them fill tensor memory
+static int tma_column_block(int Kc, int Mo, int b_transposed) {
+    int mc = Mo < 256 ? Mo : 256;
+    while (mc >= 16 && tma_w_bytes(Kc, mc, b_transposed) + TM_EPI_WARPS * TM_STAGING_BYTES + 2 * TM_SLICE_BYTES + 1024 > TM_SMEM_MAX) mc -= 16;
+    return mc >= 16 ? mc : 0;
+}
+
 bool linear_tma_supported(int64_t N, int Kc, int Mo, int b_transposed, gnn_dtype dtype) {
     if (dtype != GNN_BF16 || N <= 0 || N >= ((int64_t)1 << 31) - TC_ROWS) return false;
-    if (Kc % 16 != 0 || Kc < 16 || Kc > 256 || Mo % 16 != 0 || Mo < 16 || Mo > 256) return false;
-    if (tma_w_bytes(Kc, Mo, b_transposed) + TM_EPI_WARPS * TM_STAGING_BYTES + 2 * TM_SLICE_BYTES + 1024 > TM_SMEM_MAX) return false;
+    if (Kc % 16 != 0 || Kc < 16 || Kc > 512 || Mo % 16 != 0 || Mo < 16 || Mo > 1024) return false;
+    if (Kc > 256 && Kc % 32 != 0) return false;  // a weight block taller than 256 rows arrives as two boxes of Kc / 2 rows
+    if (tma_column_block(Kc, Mo, b_transposed) == 0) return false;
     return encoder() != nullptr;
 }
 
+// More than 256 output columns, or weights too large for shared memory, run as one launch per block of output columns.
 gnn_status linear_tma_forward(const void* X, const void* W, int64_t N, int Kc, int Mo, int b_transposed, void* Y, int* d_flag,
                               cudaStream_t st, const float* bias, int relu) {
     const char* who = "gnn_linear (pipelined tensor-core path)";
     GNN_REQUIRE(aligned16(X) && aligned16(W) && aligned16(Y), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
-    CUtensorMap mapX, mapW, mapY;
-    const int w_rows = b_transposed ? Mo : Kc, w_cols = b_transposed ? Kc : Mo;
-    if (!make_map(&mapX, X, N, Kc, TC_ROWS) || !make_map(&mapW, W, w_rows, w_cols, w_rows) ||
-        !make_map(&mapY, Y, N, Mo, 32))
-        GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
-    TmaParams P;
-    P.N = N; P.Kc = Kc; P.Mo = Mo; P.b_transposed = b_transposed; P.status = d_flag; P.bias = bias; P.relu = relu;
-    const size_t wbytes = tma_w_bytes(Kc, Mo, b_transposed);
-    const size_t fixed = 1024 + wbytes + (size_t)TM_EPI_WARPS * TM_STAGING_BYTES;
-    int stages = (int)((TM_SMEM_MAX - fixed) / TM_SLICE_BYTES);
-    P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
-    P.acc_stride = (Mo + 31) & ~31;
-    int cols = 32;
-    while (cols < 2 * P.acc_stride) cols <<= 1;
-    P.tmem_cols = cols;
-    const size_t smem = fixed + (size_t)P.stages * TM_SLICE_BYTES;
+    const int block = tma_column_block(Kc, Mo, b_transposed);
+    GNN_REQUIRE(block > 0, GNN_ERR_UNSUPPORTED, "%s: weights do not fit shared memory", who);
+    CUtensorMap mapX;
+    if (!make_map(&mapX, X, N, Kc, TC_ROWS)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     gnn_status rc = allow_big_smem(who, (const void*)linear_tma_kernel, 4, TM_SMEM_MAX);
     if (rc != GNN_OK) return rc;
     const int64_t ntiles = (N + TC_ROWS - 1) / TC_ROWS;
-    linear_tma_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TM_THREADS, smem, st>>>(mapX, mapW, mapY, P);
-    GNN_CHECK_LAUNCH(who);
+    const __nv_bfloat16* Wb = (const __nv_bfloat16*)W;
+    for (int c0 = 0; c0 < Mo; c0 += block) {
+        const int mc = Mo - c0 < block ? Mo - c0 : block;
+        // stored [Kc,Mo]: a block of columns (rows Mo apart); stored [Mo,Kc]: a block of rows
+        const int w_rows = b_transposed ? mc : Kc, w_cols = b_transposed ? Kc : mc;
+        const int box_rows = w_rows > 256 ? w_rows / 2 : w_rows;
+        CUtensorMap mapW, mapY;
+        if (!make_map_ld(&mapW, b_transposed ? Wb + (size_t)c0 * Kc : Wb + c0, w_rows, w_cols, b_transposed ? Kc : Mo, box_rows) ||
+            !make_map_ld(&mapY, (const __nv_bfloat16*)Y + c0, N, mc, Mo, 32))
+            GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+        TmaParams P;
+        P.N = N; P.Kc = Kc; P.Mo = mc; P.b_transposed = b_transposed; P.w_box_rows = box_rows; P.status = d_flag;
+        P.bias = bias ? bias + c0 : nullptr; P.relu = relu;
+        const size_t wbytes = tma_w_bytes(Kc, mc, b_transposed);
+        const size_t fixed = 1024 + wbytes + (size_t)TM_EPI_WARPS * TM_STAGING_BYTES;
+        int stages = (int)((TM_SMEM_MAX - fixed) / TM_SLICE_BYTES);
+        P.stages = stages > TM_MAX_STAGES ? TM_MAX_STAGES : stages;
+        P.acc_stride = (mc + 31) & ~31;
+        int cols = 32;
+        while (cols < 2 * P.acc_stride) cols <<= 1;
+        P.tmem_cols = cols;
+        const size_t smem = fixed + (size_t)P.stages * TM_SLICE_BYTES;
+        linear_tma_kernel<<<(int)(ntiles < 148 ? ntiles : 148), TM_THREADS, smem, st>>>(mapX, mapW, mapY, P);
+        GNN_CHECK_LAUNCH(who);
+    }
     return GNN_OK;
 }
 

@@ -39,7 +39,9 @@ CASES = [("f32", 2000, 64, 64), ("f32", 1000, 100, 36), ("f32", 333, 128, 128), 
          # fp32 beyond 256: long contraction (16 slices per tile), many column blocks, four accumulator blocks in dW
          ("f32", 3000, 512, 64), ("f32", 3000, 64, 512), ("f32", 700, 384, 128), ("f32", 900, 512, 512),
          # bf16 dW with up to 512 features (four accumulator blocks)
-         ("bf16", 3000, 512, 64), ("bf16", 2000, 384, 128), ("bf16", 1000, 320, 48)]
+         ("bf16", 3000, 512, 64), ("bf16", 2000, 384, 128), ("bf16", 1000, 320, 48),
+         # bf16 forward / dX beyond 256: weight blocks of two boxes, several column blocks
+         ("bf16", 3000, 64, 512), ("bf16", 900, 512, 512), ("bf16", 500, 288, 1024)]
 
 
 @pytest.mark.parametrize("dtype,n,K,M", CASES)
