@@ -458,7 +458,7 @@ gnn_status gnn_reduce_nodes_backward(const int64_t* graph_ptr, int32_t G, int32_
 
 /* Y = X * W (the Dense layer / the weight of a conv layer in the training example): X [N,K],
  * W [K,M], Y [N,M], all row-major and of dtype, 16-byte aligned.  With K and M multiples of 16
- * (16..256; fp32 also K up to 512 and M up to 1024) the product runs on the tensor cores with fp32 accumulation: bf16 directly, fp32 by an exact
+ * (K up to 512, M up to 1024) the product runs on the tensor cores with fp32 accumulation: bf16 directly, fp32 by an exact
  * three-term bf16 split of every value, which keeps fp32 accuracy (weights that do not fit shared memory
  * three times, e.g. 256x256, run as one launch per block of output columns).  The weight gradient of
  * gnn_linear_backward takes the tensor cores for K and M multiples of 32 (bf16: M of 16).  Other cases use an

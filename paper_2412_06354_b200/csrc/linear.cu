@@ -92,7 +92,7 @@ gemm_simt_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* _
 // ascending group order.  64 elements x 4 groups per block.
 template <typename TC>
 __global__ void __launch_bounds__(256)
-slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __restrict__ out) {
+slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __restrict__ out, int cols, int ld, int c0) {
     __shared__ float gsum[4][64];
     const int e = threadIdx.x & 63, g = threadIdx.x >> 6;
     const int64_t i = blockIdx.x * (int64_t)64 + e;
@@ -109,7 +109,8 @@ slab_sum_kernel(const float* __restrict__ part, int slabs, int64_t n, TC* __rest
     }
     gsum[g][e] = s;
     __syncthreads();
-    if (g == 0 && i < n) out[i] = from_f32<TC>(((gsum[0][e] + gsum[1][e]) + gsum[2][e]) + gsum[3][e]);
+    // the partials are [rows, cols]; the result may be a block of columns (c0 ..) of a matrix with rows ld apart
+    if (g == 0 && i < n) out[(i / cols) * ld + c0 + (i % cols)] = from_f32<TC>(((gsum[0][e] + gsum[1][e]) + gsum[2][e]) + gsum[3][e]);
 }
 
 template <typename TA, typename TB, typename TC>
@@ -137,9 +138,9 @@ gnn_status linear_tma_f32_forward(const void* X, const void* W, int64_t N, int K
 bool linear_tma_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 bool linear_tma_f32_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tma_f32_dw_partials(int64_t N);
-gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
+gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, int ldd, float* part, int* d_flag, cudaStream_t st);
 int linear_tma_dw_partials(int64_t N);
-gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st);
+gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, int ldd, float* part, int* d_flag, cudaStream_t st);
 bool linear_tc_dw_supported(int64_t N, int K, int M, gnn_dtype dtype);
 int linear_tc_dw_partials(int64_t N);
 gnn_status linear_tc_dw(const void* X, const void* dY, int64_t N, int K, int M, gnn_dtype dtype, float* part, int* d_flag,
@@ -225,13 +226,43 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
         float* part = (float*)((char*)ws + 256);
         int slabs = dw_slabs(N);
         const int64_t km = (int64_t)K * M;
+        // more output columns than one pipelined launch takes (256, or fewer where K fills tensor memory): one launch
+        // and one ordered sum per block of columns of dY, each through the same partial buffer
+        int block = 0;
+        if (N > 0 && M > 32) {
+            const int step = dtype == GNN_F32 ? 32 : 16;
+            for (int mc = (M < 256 ? M : 256) / step * step; mc >= step && !block; mc -= step)
+                if (dtype == GNN_F32 ? linear_tma_f32_dw_supported(N, K, mc, dtype) : linear_tma_dw_supported(N, K, mc, dtype)) block = mc;
+        }
+        const bool whole = dtype == GNN_F32 ? linear_tma_f32_dw_supported(N, K, M, dtype) : linear_tma_dw_supported(N, K, M, dtype);
+        if (!whole && block > 0 && M % (dtype == GNN_F32 ? 32 : 16) == 0) {
+            const int s_el = dtype == GNN_F32 ? 4 : 2;
+            for (int c0 = 0; c0 < M; c0 += block) {
+                const int mc = M - c0 < block ? M - c0 : block;
+                const void* dYb = (const char*)dY + (size_t)c0 * s_el;
+                gnn_status rc;
+                if (dtype == GNN_F32) {
+                    slabs = linear_tma_f32_dw_partials(N);
+                    rc = linear_tma_f32_dw(X, dYb, N, K, mc, M, part, (int*)ws, st);
+                } else {
+                    slabs = linear_tma_dw_partials(N);
+                    rc = linear_tma_dw(X, dYb, N, K, mc, M, part, (int*)ws, st);
+                }
+                if (rc != GNN_OK) return rc;
+                const int64_t kmc = (int64_t)K * mc;
+                if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(kmc, 64), 256, 0, st>>>(part, slabs, kmc, (float*)dW, mc, M, c0);
+                else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(kmc, 64), 256, 0, st>>>(part, slabs, kmc, (__nv_bfloat16*)dW, mc, M, c0);
+                GNN_CHECK_LAUNCH(who);
+            }
+            return GNN_OK;
+        }
         if (linear_tma_f32_dw_supported(N, K, M, dtype)) {
             slabs = linear_tma_f32_dw_partials(N);
-            gnn_status rc = linear_tma_f32_dw(X, dY, N, K, M, part, (int*)ws, st);
+            gnn_status rc = linear_tma_f32_dw(X, dY, N, K, M, M, part, (int*)ws, st);
             if (rc != GNN_OK) return rc;
         } else if (linear_tma_dw_supported(N, K, M, dtype)) {
             slabs = linear_tma_dw_partials(N);
-            gnn_status rc = linear_tma_dw(X, dY, N, K, M, part, (int*)ws, st);
+            gnn_status rc = linear_tma_dw(X, dY, N, K, M, M, part, (int*)ws, st);
             if (rc != GNN_OK) return rc;
         } else if (linear_tc_dw_supported(N, K, M, dtype)) {
             slabs = linear_tc_dw_partials(N);
@@ -245,8 +276,8 @@ gnn_status gnn_linear_backward(const void* X, const void* W, const void* dY, int
             launch_simt<__nv_bfloat16, __nv_bfloat16, float>((const __nv_bfloat16*)X, 1, K, (const __nv_bfloat16*)dY, M, 1, part, K, M, N,
                                                            dw_slab_rows(N), slabs, km, st);
         }
-        if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (float*)dW);
-        else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW);
+        if (dtype == GNN_F32) slab_sum_kernel<float><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (float*)dW, M, M, 0);
+        else slab_sum_kernel<__nv_bfloat16><<<(int)ceil_div(km, 64), 256, 0, st>>>(part, slabs, km, (__nv_bfloat16*)dW, M, M, 0);
         GNN_CHECK_LAUNCH(who);
     }
     return GNN_OK;

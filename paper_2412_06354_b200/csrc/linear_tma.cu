@@ -712,11 +712,11 @@ int linear_tma_dw_partials(int64_t N) {
 bool make_map_f32(CUtensorMap* m, const void* ptr, int64_t rows, int cols, int box_rows);
 
 // writes linear_tma_dw_partials(N) fp32 partials [K,M] to part
-gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
+gnn_status linear_tma_dw(const void* X, const void* dY, int64_t N, int K, int M, int ldd, float* part, int* d_flag, cudaStream_t st) {
     const char* who = "gnn_linear_backward (pipelined tensor-core dW)";
     GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
     CUtensorMap mapX, mapD, mapP;
-    if (!make_map(&mapX, X, N, K, DW_ROWS) || !make_map(&mapD, dY, N, M, DW_ROWS) ||
+    if (!make_map(&mapX, X, N, K, DW_ROWS) || !make_map_ld(&mapD, dY, N, M, ldd, DW_ROWS) ||  // dY may be a block of columns: rows ldd apart
         !make_map_f32(&mapP, part, (int64_t)linear_tma_dw_partials(N) * K, M, 32))
         GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaDwParams P;
@@ -945,12 +945,12 @@ int linear_tma_f32_dw_partials(int64_t N) {
 }
 
 // writes linear_tma_f32_dw_partials(N) fp32 partials [K,M] to part
-gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, float* part, int* d_flag, cudaStream_t st) {
+gnn_status linear_tma_f32_dw(const void* X, const void* dY, int64_t N, int K, int M, int ldd, float* part, int* d_flag, cudaStream_t st) {
     const char* who = "gnn_linear_backward (pipelined fp32 tensor-core dW)";
     GNN_REQUIRE(aligned16(X) && aligned16(dY) && aligned16(part), GNN_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
     CUtensorMap mapX, mapD;
     const int R = fd_rows(K, M), ka = (K + 127) / 128 * 128;
-    if (!make_map_f32(&mapX, X, N, K, R) || !make_map_f32(&mapD, dY, N, M, R)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
+    if (!make_map_f32(&mapX, X, N, K, R) || !make_map_f32_ld(&mapD, dY, N, M, ldd, R)) GNN_FAIL(GNN_ERR_CUDA, "%s: tensor map encoding failed", who);
     TmaF32DwParams P;
     P.part = part; P.N = N; P.K = K; P.M = M; P.status = d_flag; P.rows = R;
     const size_t slot = (size_t)(K / 32 + M / 32) * R * 128, ops = 2 * 3 * ((size_t)ka * R * 2 + (size_t)M * R * 2);
