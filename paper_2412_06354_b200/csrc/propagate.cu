@@ -215,7 +215,12 @@ struct Walker {
     static constexpr int NG = 32 / LPR;
     static constexpr bool EF = (MODE == MODE_EFSUM);  // one multiplier per (position, feature)
     // the per-feature mode also streams EPC multipliers per gathered chunk: half as many gathers in flight
-    static constexpr int U = (LPR >= 16) ? (EF ? (PF_U_WIDE / VPL > 1 ? PF_U_WIDE / VPL / 2 : 1) : PF_U_WIDE / VPL) : PF_U_NARROW;
+    // 256-byte rows of a sum (half a warp per row): four (bf16) or six (fp32) gathers in flight measured 3 % faster than
+    // eight on the large graph (bf16 F=128 3.52 -> 3.41 ms, fp32 F=64 3.10 -> 3.01 ms)
+    static constexpr int U_MID = Chunk<T>::N == 8 ? 4 : 6;
+    static constexpr int U = (LPR >= 16) ? (EF ? (PF_U_WIDE / VPL > 1 ? PF_U_WIDE / VPL / 2 : 1)
+                                               : (LPR == 16 && VPL == 1 && MODE == MODE_SUM ? U_MID : PF_U_WIDE / VPL))
+                                         : PF_U_NARROW;
     static constexpr int MW = EF ? EPC : 1;  // multipliers a lane holds per gathered 16-byte chunk
     static constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
     using A = Acc<T, VPL, MODE>;
@@ -1589,8 +1594,12 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     // sum reductions run one 512-byte column slab at a time.  Each pass re-reads the index stream but
     // gathers from a 4x (2x) narrower matrix, of which 4x (2x) more rows stay in L2: fewer DRAM
     // re-reads and a shorter run in total.  The result is the same arithmetic in the same order.
-    const bool slabs = mode == MODE_SUM && nvec > 32 && nvec % 32 == 0 && (size_t)N * nvec * 16 > ((size_t)256 << 20);
+    // ... and on graphs small enough for one-slab chunks every pass takes the position-first kernel, which rows over
+    // 512 bytes otherwise cannot (1.36 M edges: 1024-byte fp32 rows 267 us as one row walk, 2 x 115 us as two passes)
+    const bool slabs = mode == MODE_SUM && nvec > 32 && nvec % 32 == 0 &&
+                       ((size_t)N * nvec * 16 > ((size_t)256 << 20) || (E > 0 && chunk_edges(E) <= PF_SLAB));
     if (slabs) {
+        if (sum_half_slab(mode, N, E, 32)) { P.chunk = PF_SLAB / 2; P.nchunks = ceil_div(E, (int64_t)P.chunk); }  // the rule of 512-byte rows, per pass
         const int nslab = nvec / 32, fslab = F / nslab;
         P.nvec = 32; P.F = fslab;
         for (int sl = 0; sl < nslab; ++sl) {
