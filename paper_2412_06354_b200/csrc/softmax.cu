@@ -3,15 +3,20 @@
 // Logits and coefficients are [E,H] in CSR order, so a node's incoming edges are contiguous.
 //
 // One warp per row for ordinary rows; rows longer than SM_LONG_ROW positions are left to a
-// second kernel that gives each of them a whole block.  Reductions use fixed shuffle / shared
-// memory trees, so results are bit-reproducible.  All arithmetic is fp32.
+// second kernel that gives each of them a whole block, and rows longer than SM_HUB_ROW positions
+// (4, 8, 16 or 32 heads) a cluster of eight blocks that combine their results through distributed
+// shared memory.  Reductions use fixed shuffle / shared memory trees and a fixed block order, so
+// results are bit-reproducible.  All arithmetic is fp32.
 #include <mutex>
 
 #include "common.cuh"
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
 
 namespace gnn {
 
-constexpr int SM_LONG_ROW = 2048;  // positions
+constexpr int SM_LONG_ROW = 512;  // positions (12 M-edge power-law graph, 8 heads: 2048 is 2 % / 16 % slower forward / backward)
 constexpr int SM_BLOCK = 256;
 
 template <typename T> __device__ __forceinline__ float ld_as_f32(const T* p, size_t i);
@@ -252,6 +257,188 @@ __device__ __forceinline__ void softmax_bwd_row_vec4(const T* __restrict__ alpha
     }
 }
 
+// ---- a block per row with the same 16-byte / 8-byte accesses.  Thread t takes chunks t, t + SM_BLOCK, ...: 4 * SM_BLOCK
+// values apart, a multiple of H, so its four heads never change.  A head's value is reduced over the lanes of a warp,
+// then over the warps in warp order through shared memory (red: SM_BLOCK floats); every thread gets the result.
+template <class Op>
+__device__ __forceinline__ void reduce_heads4_block(float* v, int H, float* red) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, lo = H / 4;
+    reduce_heads4<Op>(v, H);
+    __syncthreads();  // red is free again
+    if (lane < lo)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) red[w * 32 + 4 * lane + j] = v[j];
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float r = red[4 * (lane % lo) + j];
+        for (int q = 1; q < SM_BLOCK / 32; ++q) r = Op::f(r, red[q * 32 + 4 * (lane % lo) + j]);
+        v[j] = r;
+    }
+}
+
+// Chunks t, t + SM_BLOCK, ... of a row, VB_U loads in flight per thread: body(chunk index, slot) after the loads
+// of a batch were issued.
+constexpr int VB_U = 4;
+template <typename T, class Body>
+__device__ __forceinline__ void for_chunks4(const T* __restrict__ p, size_t lo, int64_t nch, Body body, int64_t first = 0) {
+    for (int64_t c0 = first + threadIdx.x; c0 < nch; c0 += VB_U * SM_BLOCK) {  // first: a multiple of SM_BLOCK
+        float v[VB_U][4];
+#pragma unroll
+        for (int u = 0; u < VB_U; ++u)
+            if (c0 + u * SM_BLOCK < nch) ld4(p, lo + 4 * (size_t)(c0 + u * SM_BLOCK), v[u]);
+#pragma unroll
+        for (int u = 0; u < VB_U; ++u)
+            if (c0 + u * SM_BLOCK < nch) body(c0 + u * SM_BLOCK, v[u]);
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void softmax_row_vec4_block(const T* __restrict__ s, T* __restrict__ alpha, int64_t a, int64_t b, int H, int row,
+                                                       float* rowmax, float* rowsum, float* red) {
+    const size_t lo = (size_t)a * H;
+    const int64_t nch = ((b - a) * H) >> 2;
+    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, z[4] = {0.f, 0.f, 0.f, 0.f};
+    for_chunks4(s, lo, nch, [&](int64_t, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m[j] = fmaxf(m[j], v[j]);
+    });
+    reduce_heads4_block<MaxOp>(m, H, red);
+    for_chunks4(s, lo, nch, [&](int64_t, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) z[j] += expf(v[j] - m[j]);
+    });
+    reduce_heads4_block<SumOp>(z, H, red);
+    for_chunks4(s, lo, nch, [&](int64_t c, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = expf(v[j] - m[j]) / z[j];
+        st4(alpha, lo + 4 * (size_t)c, v);
+    });
+    if (threadIdx.x < H / 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (rowmax) rowmax[(size_t)row * H + 4 * threadIdx.x + j] = m[j];
+            if (rowsum) rowsum[(size_t)row * H + 4 * threadIdx.x + j] = z[j];
+        }
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void softmax_bwd_row_vec4_block(const T* __restrict__ alpha, const T* __restrict__ dalpha, T* __restrict__ ds,
+                                                           int64_t a, int64_t b, int H, float* red) {
+    const size_t lo = (size_t)a * H;
+    const int64_t nch = ((b - a) * H) >> 2;
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    for_chunks4(alpha, lo, nch, [&](int64_t c, float* x) {
+        float y[4];
+        ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) d[j] = fmaf(x[j], y[j], d[j]);
+    });
+    reduce_heads4_block<SumOp>(d, H, red);
+    for_chunks4(alpha, lo, nch, [&](int64_t c, float* x) {
+        float y[4];
+        ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) y[j] = x[j] * (y[j] - d[j]);
+        st4(ds, lo + 4 * (size_t)c, y);
+    });
+}
+
+// ---- rows of more than SM_HUB_ROW positions: a cluster of SM_CLUSTER blocks per row.  Block k takes a contiguous
+// share of the chunks (a multiple of SM_BLOCK, so that a thread keeps its heads), reduces it as above, leaves the
+// per-head result in its shared memory, and after a cluster barrier every block combines the SM_CLUSTER results in
+// block order, read through distributed shared memory.  Two result buffers alternate, so a buffer is written
+// again only after a later barrier than the one its readers passed.
+constexpr int SM_HUB_ROW = 8192;  // positions (2048 and 32768: 5-14 % slower on the same graph)
+constexpr int SM_LONG_MINB = 3;   // blocks per SM the long-row kernels are compiled for: they are bound by the loads in
+                                  // flight per SM (forward, same graph: 865 / 565 / 481 / 486 us at 1 / 2 / 3 / 4)
+constexpr int SM_CLUSTER = 8;
+
+struct HubRows {
+    int list[SM_CLUSTER * SM_BLOCK];
+    int count;
+    float res[2][32];
+};
+
+template <class Op>
+__device__ __forceinline__ void reduce_heads4_cluster(float* v, int H, float* red, float* res, cg::cluster_group& cluster) {
+    const int lane = threadIdx.x & 31, lo = H / 4;
+    reduce_heads4_block<Op>(v, H, red);
+    if (threadIdx.x < lo)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) res[4 * threadIdx.x + j] = v[j];
+    cluster.sync();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float r = cluster.map_shared_rank(res, 0)[4 * (lane % lo) + j];
+        for (int q = 1; q < SM_CLUSTER; ++q) r = Op::f(r, cluster.map_shared_rank(res, q)[4 * (lane % lo) + j]);
+        v[j] = r;
+    }
+}
+
+// this block's chunks [first, last) of a row of nch chunks
+__device__ __forceinline__ void hub_share(int64_t nch, int rank, int64_t* first, int64_t* last) {
+    int64_t per = (nch + SM_CLUSTER - 1) / SM_CLUSTER;
+    per = (per + SM_BLOCK - 1) / SM_BLOCK * SM_BLOCK;
+    *first = rank * per < nch ? rank * per : nch;
+    *last = *first + per < nch ? *first + per : nch;
+}
+
+template <typename T>
+__device__ __forceinline__ void softmax_row_vec4_cluster(const T* __restrict__ s, T* __restrict__ alpha, int64_t a, int64_t b, int H, int row,
+                                                         float* rowmax, float* rowsum, float* red, HubRows& hub, cg::cluster_group& cluster) {
+    const size_t lo = (size_t)a * H;
+    int64_t first, last;
+    hub_share(((b - a) * H) >> 2, (int)cluster.block_rank(), &first, &last);
+    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, z[4] = {0.f, 0.f, 0.f, 0.f};
+    for_chunks4(s, lo, last, [&](int64_t, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m[j] = fmaxf(m[j], v[j]);
+    }, first);
+    reduce_heads4_cluster<MaxOp>(m, H, red, hub.res[0], cluster);
+    for_chunks4(s, lo, last, [&](int64_t, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) z[j] += expf(v[j] - m[j]);
+    }, first);
+    reduce_heads4_cluster<SumOp>(z, H, red, hub.res[1], cluster);
+    for_chunks4(s, lo, last, [&](int64_t c, float* v) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = expf(v[j] - m[j]) / z[j];
+        st4(alpha, lo + 4 * (size_t)c, v);
+    }, first);
+    if (cluster.block_rank() == 0 && threadIdx.x < H / 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (rowmax) rowmax[(size_t)row * H + 4 * threadIdx.x + j] = m[j];
+            if (rowsum) rowsum[(size_t)row * H + 4 * threadIdx.x + j] = z[j];
+        }
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void softmax_bwd_row_vec4_cluster(const T* __restrict__ alpha, const T* __restrict__ dalpha, T* __restrict__ ds,
+                                                             int64_t a, int64_t b, int H, float* red, float* res, cg::cluster_group& cluster) {
+    const size_t lo = (size_t)a * H;
+    int64_t first, last;
+    hub_share(((b - a) * H) >> 2, (int)cluster.block_rank(), &first, &last);
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    for_chunks4(alpha, lo, last, [&](int64_t c, float* x) {
+        float y[4];
+        ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) d[j] = fmaf(x[j], y[j], d[j]);
+    }, first);
+    reduce_heads4_cluster<SumOp>(d, H, red, res, cluster);
+    for_chunks4(alpha, lo, last, [&](int64_t c, float* x) {
+        float y[4];
+        ld4(dalpha, lo + 4 * (size_t)c, y);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) y[j] = x[j] * (y[j] - d[j]);
+        st4(ds, lo + 4 * (size_t)c, y);
+    }, first);
+}
+
 static __host__ __device__ inline bool head_pow2(int H) { return H >= 1 && H <= 32 && (H & (H - 1)) == 0; }
 
 // Row loops.  LONG = false: every warp strides over the rows and takes the ones of at most
@@ -294,6 +481,97 @@ __device__ __forceinline__ void for_each_row(const int64_t* __restrict__ rowptr,
     }
 }
 
+// Long rows for a grid of clusters, in two phases.  First every block alone: it takes a contiguous share of the rows,
+// scans it NT rows at a time and works through the rows above THRESH positions (up to SM_HUB_ROW when hubs is set).
+// Then, when hubs is set, every cluster: its blocks scan SM_CLUSTER * NT rows of the cluster's share at a time and
+// append the rows above SM_HUB_ROW positions to block 0's list (atomics on distributed shared memory), and the
+// whole cluster takes those rows one by one.  Every block of a cluster passes the same number of cluster barriers:
+// the windows depend on the cluster's share alone, and the number of hub rows is read from block 0 after a barrier.
+// The list orders vary from run to run; no row's arithmetic depends on them.
+template <int NT, int THRESH, class Body, class HubBody>
+__device__ __forceinline__ void for_each_long_row_cluster(const int64_t* __restrict__ rowptr, int N, bool hubs, LongRows& L, HubRows& Hb,
+                                                          cg::cluster_group& cluster, Body body, HubBody hub_body) {
+    {
+        const int per = (N + (int)gridDim.x - 1) / (int)gridDim.x;
+        const int r0 = (int)blockIdx.x * per < N ? (int)blockIdx.x * per : N, r1 = min(N, r0 + per);
+        for (int base = r0; base < r1; base += NT) {
+            __syncthreads();  // every thread is done with the previous list
+            if (threadIdx.x == 0) L.count = 0;
+            __syncthreads();
+            const int r = base + (int)threadIdx.x;
+            if (r < r1) {
+                const int64_t len = rowptr[r + 1] - rowptr[r];
+                if (len > THRESH && !(hubs && len > SM_HUB_ROW)) L.list[atomicAdd(&L.count, 1)] = r;
+            }
+            __syncthreads();
+            const int n = L.count;
+            for (int i = 0; i < n; ++i) {
+                const int row = L.list[i];
+                body(row, rowptr[row], rowptr[row + 1]);
+            }
+        }
+    }
+    if (!hubs) return;  // the same for every block of the grid
+    const int rank = (int)cluster.block_rank();
+    const int clusters = (int)gridDim.x / SM_CLUSTER, me = (int)blockIdx.x / SM_CLUSTER;
+    const int per = (N + clusters - 1) / clusters;
+    const int r0 = me * per < N ? me * per : N, r1 = min(N, r0 + per);
+    int* count0 = cluster.map_shared_rank(&Hb.count, 0);
+    int* list0 = cluster.map_shared_rank(Hb.list, 0);
+    for (int base = r0; base < r1; base += SM_CLUSTER * NT) {
+        if (threadIdx.x == 0) Hb.count = 0;
+        cluster.sync();  // block 0's counter is reset
+        const int r = base + rank * NT + (int)threadIdx.x;
+        if (r < r1 && rowptr[r + 1] - rowptr[r] > SM_HUB_ROW) list0[atomicAdd(count0, 1)] = r;
+        cluster.sync();  // the list is complete
+        const int nh = *count0;
+        for (int i = 0; i < nh; ++i) {
+            const int row = list0[i];
+            hub_body(row, rowptr[row], rowptr[row + 1], i);
+        }
+        cluster.sync();  // nobody reads the list or a result buffer any more
+    }
+}
+
+template <typename T>
+__global__ void __cluster_dims__(SM_CLUSTER, 1, 1) __launch_bounds__(SM_BLOCK, SM_LONG_MINB)
+edge_softmax_long_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ s, int H,
+                         T* __restrict__ alpha, float* __restrict__ rowmax, float* __restrict__ rowsum) {
+    __shared__ float red[SM_BLOCK];
+    __shared__ LongRows lrows;
+    __shared__ HubRows hub;
+    cg::cluster_group cluster = cg::this_cluster();
+    const bool vec4 = H >= 4 && head_pow2(H) && ((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(alpha)) & (4 * sizeof(T) - 1)) == 0;
+    for_each_long_row_cluster<SM_BLOCK, SM_LONG_ROW>(
+        rowptr, N, vec4, lrows, hub, cluster,
+        [&](int row, int64_t a, int64_t b) {
+            if (vec4) softmax_row_vec4_block<T>(s, alpha, a, b, H, row, rowmax, rowsum, red);
+            else if (head_pow2(H)) softmax_row_pow2<T, SM_BLOCK>(s, alpha, a, b, H, row, rowmax, rowsum, red);
+            else softmax_row_any<T, SM_BLOCK>(s, alpha, a, b, H, row, rowmax, rowsum, red);
+        },
+        [&](int row, int64_t a, int64_t b, int) { softmax_row_vec4_cluster<T>(s, alpha, a, b, H, row, rowmax, rowsum, red, hub, cluster); });
+}
+
+template <typename T>
+__global__ void __cluster_dims__(SM_CLUSTER, 1, 1) __launch_bounds__(SM_BLOCK)
+edge_softmax_backward_long_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ alpha,
+                                  const T* __restrict__ dalpha, int H, T* __restrict__ ds) {
+    __shared__ float red[SM_BLOCK];
+    __shared__ LongRows lrows;
+    __shared__ HubRows hub;
+    cg::cluster_group cluster = cg::this_cluster();
+    const bool vec4 = H >= 4 && head_pow2(H) &&
+                      ((reinterpret_cast<uintptr_t>(alpha) | reinterpret_cast<uintptr_t>(dalpha) | reinterpret_cast<uintptr_t>(ds)) & (4 * sizeof(T) - 1)) == 0;
+    for_each_long_row_cluster<SM_BLOCK, SM_LONG_ROW>(
+        rowptr, N, vec4, lrows, hub, cluster,
+        [&](int, int64_t a, int64_t b) {
+            if (vec4) softmax_bwd_row_vec4_block<T>(alpha, dalpha, ds, a, b, H, red);
+            else softmax_bwd_row<T, SM_BLOCK>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
+        },
+        // one result buffer per parity of the hub's place in the list: it is written again two barriers later
+        [&](int, int64_t a, int64_t b, int i) { softmax_bwd_row_vec4_cluster<T>(alpha, dalpha, ds, a, b, H, red, hub.res[i & 1], cluster); });
+}
+
 template <typename T, bool LONG>
 __global__ void __launch_bounds__(SM_BLOCK)
 edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restrict__ s, int H,
@@ -311,6 +589,7 @@ edge_softmax_kernel(const int64_t* __restrict__ rowptr, int N, const T* __restri
             return;
         }
         if (!LONG && vec4) softmax_row_vec4<T>(s, alpha, a, b, H, row, rowmax, rowsum);
+        else if (vec4) softmax_row_vec4_block<T>(s, alpha, a, b, H, row, rowmax, rowsum, red);
         else if (head_pow2(H)) softmax_row_pow2<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
         else softmax_row_any<T, LONG ? SM_BLOCK : 32>(s, alpha, a, b, H, row, rowmax, rowsum, red);
     });
@@ -327,6 +606,7 @@ edge_softmax_backward_kernel(const int64_t* __restrict__ rowptr, int N, const T*
     for_each_row<LONG, SM_BLOCK>(rowptr, N, lrows, [&](int, int64_t a, int64_t b) {
         if (b == a) return;
         if (!LONG && vec4) softmax_bwd_row_vec4<T>(alpha, dalpha, ds, a, b, H);
+        else if (vec4) softmax_bwd_row_vec4_block<T>(alpha, dalpha, ds, a, b, H, red);
         else softmax_bwd_row<T, LONG ? SM_BLOCK : 32>(alpha, dalpha, ds, a, b, H, head_pow2(H), red);
     });
 }
@@ -598,6 +878,12 @@ static int row_grid(int N, bool is_long) {
     return (int)(want < cap ? (want > 0 ? want : 1) : cap);
 }
 
+// grid of whole clusters for the long rows: a block per row up to eight blocks per SM
+static int row_grid_cluster(int N) {
+    const int64_t want = ceil_div((int64_t)N, SM_CLUSTER), cap = 148;
+    return SM_CLUSTER * (int)(want < cap ? (want > 0 ? want : 1) : cap);
+}
+
 // grid for a row-strided kernel: one warp per row up to a few waves; one block per row for long rows
 static int row_grid_pl(int N, bool is_long) {
     const int64_t want = is_long ? N : ceil_div((int64_t)N * 32, SM_BLOCK);
@@ -729,16 +1015,16 @@ gnn_status gnn_edge_softmax(const gnn_csr* g, const void* logits_EH, int H, gnn_
     if (g->N == 0) return GNN_OK;
     GNN_REQUIRE(g->E == 0 || (logits_EH && alpha_EH), GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
-    const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
+    const int wgrid = row_grid(g->N, false), lgrid = row_grid_cluster(g->N);
     // the two row tiers write disjoint rows: side by side (the long rows' blocks beside the warps of the short ones)
     if (dtype == GNN_F32)
         run_row_tiers(
-            st, [&](cudaStream_t q) { edge_softmax_kernel<float, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum); },
+            st, [&](cudaStream_t q) { edge_softmax_long_kernel<float><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum); },
             [&](cudaStream_t q) { edge_softmax_kernel<float, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)logits_EH, H, (float*)alpha_EH, rowmax, rowsum); },
             [&](cudaStream_t) {});
     else
         run_row_tiers(
-            st, [&](cudaStream_t q) { edge_softmax_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum); },
+            st, [&](cudaStream_t q) { edge_softmax_long_kernel<__nv_bfloat16><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum); },
             [&](cudaStream_t q) { edge_softmax_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)logits_EH, H, (__nv_bfloat16*)alpha_EH, rowmax, rowsum); },
             [&](cudaStream_t) {});
     GNN_CHECK_LAUNCH(who);
@@ -753,15 +1039,15 @@ gnn_status gnn_edge_softmax_backward(const gnn_csr* g, const void* alpha_EH, con
     if (g->N == 0 || g->E == 0) return GNN_OK;
     GNN_REQUIRE(alpha_EH && dAlpha_EH && dLogits_EH, GNN_ERR_INVALID_ARG, "%s: null argument", who);
     cudaStream_t st = as_stream(stream);
-    const int wgrid = row_grid(g->N, false), lgrid = row_grid(g->N, true);
+    const int wgrid = row_grid(g->N, false), lgrid = row_grid_cluster(g->N);
     if (dtype == GNN_F32)
         run_row_tiers(
-            st, [&](cudaStream_t q) { edge_softmax_backward_kernel<float, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH); },
+            st, [&](cudaStream_t q) { edge_softmax_backward_long_kernel<float><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH); },
             [&](cudaStream_t q) { edge_softmax_backward_kernel<float, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const float*)alpha_EH, (const float*)dAlpha_EH, H, (float*)dLogits_EH); },
             [&](cudaStream_t) {});
     else
         run_row_tiers(
-            st, [&](cudaStream_t q) { edge_softmax_backward_kernel<__nv_bfloat16, true><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH); },
+            st, [&](cudaStream_t q) { edge_softmax_backward_long_kernel<__nv_bfloat16><<<lgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH); },
             [&](cudaStream_t q) { edge_softmax_backward_kernel<__nv_bfloat16, false><<<wgrid, SM_BLOCK, 0, q>>>(g->rowptr, g->N, (const __nv_bfloat16*)alpha_EH, (const __nv_bfloat16*)dAlpha_EH, H, (__nv_bfloat16*)dLogits_EH); },
             [&](cudaStream_t) {});
     GNN_CHECK_LAUNCH(who);

@@ -98,7 +98,7 @@ def test_aggregate_matches_checker_and_fused_path(gnn, dtype, F):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("H", [1, 3, 8, 32])
+@pytest.mark.parametrize("H", [1, 3, 4, 8, 16, 32])
 def test_edge_softmax_forward_backward(gnn, dtype, H):
     n, src, dst = ragged_graph(80 + H)  # hub row of 6000 edges takes the block-per-row path
     g = build_graph(gnn, n, src, dst)
@@ -127,6 +127,50 @@ def test_edge_softmax_forward_backward(gnn, dtype, H):
     assert_close(to_host64(ds), dso[eid], S[eid], dtype, "dlogits")
     again = gnn.edge_softmax(g, to_dev(s[eid]))
     assert np.array_equal(bits(again), bits(alpha))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("H", [1, 4, 8, 32])
+def test_edge_softmax_rows_of_tens_of_thousands_of_positions(gnn, dtype, H):
+    """Three rows above 8192 positions (shared by a cluster of blocks when H is 4, 8, 16 or 32), two of them in one
+    scan window, one a single position above the threshold; a band of rows of 513 ... 3000 positions (a block each)."""
+    rng = np.random.default_rng(31 + H)
+    n, e = 3000, 120000
+    src = rng.integers(0, n, e).astype(np.int32)
+    dst = rng.integers(0, n, e).astype(np.int32)
+    dst[:20000] = 7
+    dst[20000:29000] = 9
+    dst[29000:37193] = 2990
+    at = 40000
+    for k in range(12):
+        dst[at:at + 513 + 220 * k] = 300 + 5 * k
+        at += 513 + 220 * k
+    perm = rng.permutation(e)
+    src, dst = src[perm].copy(), dst[perm].copy()
+    g = build_graph(gnn, n, src, dst)
+    eid = host_csr(n, src, dst)["eid"]
+    s = feats((e, H), dtype, 900 + H)
+    if dtype == "f32":
+        s = (s * 3).astype(np.float32)
+    alpha, rmax, rsum = gnn.edge_softmax(g, to_dev(s[eid]), want_stats=True)
+    ao = oracle.edge_softmax(n, dst, s)
+    assert_close(to_host64(alpha), ao[eid], ao[eid], dtype, "alpha")
+    deg = np.bincount(dst, minlength=n)
+    smax = np.full((n, H), -np.inf)
+    np.maximum.at(smax, dst, synth.to_f64(s))
+    assert np.array_equal(to_host64(rmax)[deg > 0], smax[deg > 0])
+    ssum = np.zeros((n, H))
+    np.add.at(ssum, dst, np.exp(synth.to_f64(s) - smax[dst]))
+    assert np.allclose(to_host64(rsum)[deg > 0], ssum[deg > 0], rtol=1e-4)
+    a_host = np.empty((e, H), np.float64)
+    a_host[eid] = to_host64(alpha)
+    R = feats((e, H), dtype, 901 + H)
+    ds = gnn.edge_softmax_backward(g, alpha, to_dev(R[eid]))
+    dso, S = oracle.edge_softmax_backward(n, dst, a_host, R)
+    assert_close(to_host64(ds), dso[eid], S[eid], dtype, "dlogits")
+    again = gnn.edge_softmax(g, to_dev(s[eid]))
+    assert np.array_equal(bits(again), bits(alpha))
+    assert np.array_equal(bits(gnn.edge_softmax_backward(g, alpha, to_dev(R[eid]))), bits(ds))
 
 
 def test_edge_softmax_degenerate(gnn):

@@ -231,3 +231,37 @@ def test_gatv2_logits_forward_backward(gnn, dtype, H, C):
     assert_close(to_host64(da), rb["da"], rb["Sda"], "f32", "GATv2 da")
     again = gnn.gatv2_logits_backward(g, to_dev(Xl), to_dev(Xr), to_dev(a), to_dev(ds[ref["eid"]]), H)
     assert all(np.array_equal(bits(x), bits(y)) for x, y in zip((dXl, dXr, da), again)), "not bit-reproducible"
+
+
+@pytest.mark.parametrize("dtype,H,C", [("f32", 4, 16), ("bf16", 8, 32), ("f32", 1, 128)])
+def test_gatv2_backward_hub_rows_of_both_orientations(gnn, dtype, H, C):
+    """Several rows of thousands of positions and a band of rows of 257 ... 2000 positions (the block tier), in the
+    target and in the source orientation, among 80000 mostly short rows."""
+    rng = np.random.default_rng(77 + H)
+    n, e = 80000, 300000
+    src = rng.integers(0, n, e).astype(np.int32)
+    dst = rng.integers(0, n, e).astype(np.int32)
+    dst[:9000] = 7
+    dst[9000:12001] = 7 + 37
+    dst[12001:14050] = 79999            # the last row
+    for k in range(30):                 # block-tier rows of 257 ... 2000 positions
+        dst[20000 + 2000 * k:20000 + 2000 * k + 257 + 60 * k] = 100 + k
+    src[90000:95000] = 79990
+    for k in range(20):
+        src[100000 + 1000 * k:100000 + 1000 * k + 300 + 30 * k] = 200 + 3 * k
+    perm = rng.permutation(e)
+    src, dst = src[perm].copy(), dst[perm].copy()
+    g = build_graph(gnn, n, src, dst)
+    ref = host_csr(n, src, dst)
+    F = H * C
+    Xl = feats((n, F), dtype, 1600 + F)
+    Xr = feats((n, F), dtype, 1601 + F, stream=1)
+    a = synth.uniform_f32((H, C), -1.0, 1.0, 28)
+    ds = synth.normal_f32((e, H), 29)
+    dXl, dXr, da = gnn.gatv2_logits_backward(g, to_dev(Xl), to_dev(Xr), to_dev(a), to_dev(ds[ref["eid"]]), H)
+    rb = oracle.gatv2_logits_backward(n, src, dst, Xl, Xr, a, H, ds)
+    assert_close(to_host64(dXl), rb["dXl"], rb["SXl"], dtype, "GATv2 dXl")
+    assert_close(to_host64(dXr), rb["dXr"], rb["SXr"], dtype, "GATv2 dXr")
+    assert_close(to_host64(da), rb["da"], rb["Sda"], "f32", "GATv2 da")
+    again = gnn.gatv2_logits_backward(g, to_dev(Xl), to_dev(Xr), to_dev(a), to_dev(ds[ref["eid"]]), H)
+    assert all(np.array_equal(bits(x), bits(y)) for x, y in zip((dXl, dXr, da), again)), "not bit-reproducible"
