@@ -9,7 +9,8 @@
 // Backward: dXr[i] sums over the positions of row i, dXl[j] over the transposed row of j, each term
 // ds * a * LeakyReLU'(z) needing both rows again.  A warp walks a row (four gathers in flight), rows over 256
 // positions get a block whose warps take contiguous shares that are added in warp order; da is the column sum
-// of per-row partials.  Every order is fixed: results are bit-reproducible.
+// of per-row partials.  Every order is fixed: results are bit-reproducible.  Gathered rows stay in registers as
+// loaded and are unpacked where they are used (bf16: 14-16 registers fewer, one more block per SM).
 #include "common.cuh"
 
 namespace gnn {
@@ -48,6 +49,11 @@ __device__ __forceinline__ void v2_load(const void* base, int64_t row, int nvec,
     }
 }
 
+// the same chunk as it lies in memory: unpacked where it is used, so that a gather in flight holds four registers
+__device__ __forceinline__ uint4 v2_load_raw(const void* base, int64_t row, int nvec, int li, bool on) {
+    return on ? __ldg(reinterpret_cast<const uint4*>(base) + (size_t)row * nvec + li) : make_uint4(0u, 0u, 0u, 0u);
+}
+
 // ------------------------------------------------------------------ forward
 template <typename T>
 __global__ void __launch_bounds__(256) gatv2_logits_kernel(const V2Params P) {
@@ -67,10 +73,10 @@ __global__ void __launch_bounds__(256) gatv2_logits_kernel(const V2Params P) {
     float xs[EPC];
     v2_load<T>(P.Xself, r, P.nvec, lane, on, xs);
     for (int64_t p0 = cs; p0 < ce; p0 += V2_U) {
-        float xo[V2_U][EPC];
+        uint4 raw[V2_U];
 #pragma unroll
         for (int u = 0; u < V2_U; ++u)
-            if (p0 + u < ce) v2_load<T>(P.Xother, P.col[p0 + u], P.nvec, lane, on, xo[u]);
+            if (p0 + u < ce) raw[u] = v2_load_raw(P.Xother, P.col[p0 + u], P.nvec, lane, on);
 #pragma unroll
         for (int u = 0; u < V2_U; ++u) {
             const int64_t p = p0 + u;
@@ -79,10 +85,12 @@ __global__ void __launch_bounds__(256) gatv2_logits_kernel(const V2Params P) {
                 do { ++r; rend = P.rowptr[r + 1]; } while (p >= rend);
                 v2_load<T>(P.Xself, r, P.nvec, lane, on, xs);
             }
+            float xo[EPC];
+            Chunk<T>::unpack(raw[u], xo);
             float t = 0.f;
 #pragma unroll
             for (int j = 0; j < EPC; ++j) {
-                const float z = xo[u][j] + xs[j];
+                const float z = xo[j] + xs[j];
                 t = fmaf(av[j], z > 0.f ? z : P.slope * z, t);
             }
             for (int o = span >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -99,21 +107,23 @@ __device__ __forceinline__ void v2_row_share(const V2Params& P, int row, int64_t
     constexpr int EPC = Chunk<T>::N;
     const int head = P.H > 1 ? lane / P.lph : 0;
     for (int64_t p0 = pa; p0 < pb; p0 += V2_U) {
-        float xo[V2_U][EPC];
+        uint4 raw[V2_U];
         float dsv[V2_U];
 #pragma unroll
         for (int u = 0; u < V2_U; ++u)
             if (p0 + u < pb) {
-                v2_load<T>(P.Xother, P.col[p0 + u], P.nvec, lane, on, xo[u]);
+                raw[u] = v2_load_raw(P.Xother, P.col[p0 + u], P.nvec, lane, on);
                 const int64_t q = P.pos_index ? (int64_t)P.pos_index[p0 + u] : p0 + u;
                 dsv[u] = on ? __ldg(P.ds + q * P.H + head) : 0.f;
             }
 #pragma unroll
         for (int u = 0; u < V2_U; ++u) {
             if (p0 + u >= pb) break;
+            float xo[EPC];
+            Chunk<T>::unpack(raw[u], xo);
 #pragma unroll
             for (int j = 0; j < EPC; ++j) {
-                const float z = xo[u][j] + xs[j];
+                const float z = xo[j] + xs[j];
                 acc[j] = fmaf(dsv[u] * av[j], z > 0.f ? 1.0f : P.slope, acc[j]);
                 if (DA) acc_a[j] = fmaf(dsv[u], z > 0.f ? z : P.slope * z, acc_a[j]);
             }
@@ -155,39 +165,53 @@ __global__ void __launch_bounds__(256) gatv2_backward_rows_kernel(const V2Params
     }
 }
 
-// longer rows: a block per row, its warps take contiguous shares, added in warp order
+// longer rows: a block per row, its warps take contiguous shares, added in warp order.  Block k owns the rows
+// k, k + blocks, ... (hub rows of a power-law graph sit at neighbouring indices, the stride spreads them); its
+// threads look at V2_BLOCK of them at once and list the long ones in shared memory, then the block works through
+// the list.  The order of the list varies from run to run; no row's arithmetic depends on it.
 template <typename T, bool DA>
-__global__ void __launch_bounds__(V2_BLOCK) gatv2_backward_long_kernel(const V2Params P) {
+__global__ void __launch_bounds__(V2_BLOCK, 2) gatv2_backward_long_kernel(const V2Params P) {
     constexpr int EPC = Chunk<T>::N, NW = V2_BLOCK / 32;
     __shared__ float part[2][NW][32 * EPC];
+    __shared__ int list[V2_BLOCK];
+    __shared__ int count;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const bool on = lane < P.nvec;
     float av[EPC];
 #pragma unroll
     for (int j = 0; j < EPC; ++j) av[j] = on ? P.a[lane * EPC + j] : 0.f;
-    for (int row = blockIdx.x; row < P.N; row += gridDim.x) {
-        const int64_t a = P.rowptr[row], b = P.rowptr[row + 1];
-        if (b - a <= V2_LONG) continue;  // uniform over the block
-        const int64_t per = (b - a + NW - 1) / NW;
-        const int64_t pa = a + w * per, pb = pa + per < b ? pa + per : b;
-        float xs[EPC], acc[EPC], acc_a[EPC];
-        v2_load<T>(P.Xself, row, P.nvec, lane, on, xs);
-#pragma unroll
-        for (int j = 0; j < EPC; ++j) { acc[j] = 0.f; acc_a[j] = 0.f; }
-        if (pa < pb) v2_row_share<T, DA>(P, row, pa, pb, lane, on, xs, av, acc, acc_a);
-#pragma unroll
-        for (int j = 0; j < EPC; ++j) { part[0][w][lane * EPC + j] = acc[j]; part[1][w][lane * EPC + j] = acc_a[j]; }
+    for (int64_t k0 = 0; (int64_t)blockIdx.x + k0 * gridDim.x < P.N; k0 += V2_BLOCK) {
+        __syncthreads();  // every thread is done with the previous list
+        if (threadIdx.x == 0) count = 0;
         __syncthreads();
-        if (w == 0) {
+        const int64_t mine = (int64_t)blockIdx.x + (k0 + threadIdx.x) * gridDim.x;
+        if (mine < P.N && P.rowptr[mine + 1] - P.rowptr[mine] > V2_LONG) list[atomicAdd(&count, 1)] = (int)mine;
+        __syncthreads();
+        const int n = count;
+        for (int i = 0; i < n; ++i) {
+            const int row = list[i];
+            const int64_t a = P.rowptr[row], b = P.rowptr[row + 1];
+            const int64_t per = (b - a + NW - 1) / NW;
+            const int64_t pa = a + w * per, pb = pa + per < b ? pa + per : b;
+            float xs[EPC], acc[EPC], acc_a[EPC];
+            v2_load<T>(P.Xself, row, P.nvec, lane, on, xs);
 #pragma unroll
-            for (int j = 0; j < EPC; ++j) {
-                float s0 = part[0][0][lane * EPC + j], s1 = part[1][0][lane * EPC + j];
-                for (int q = 1; q < NW; ++q) { s0 += part[0][q][lane * EPC + j]; s1 += part[1][q][lane * EPC + j]; }
-                acc[j] = s0; acc_a[j] = s1;
+            for (int j = 0; j < EPC; ++j) { acc[j] = 0.f; acc_a[j] = 0.f; }
+            if (pa < pb) v2_row_share<T, DA>(P, row, pa, pb, lane, on, xs, av, acc, acc_a);
+#pragma unroll
+            for (int j = 0; j < EPC; ++j) { part[0][w][lane * EPC + j] = acc[j]; part[1][w][lane * EPC + j] = acc_a[j]; }
+            __syncthreads();
+            if (w == 0) {
+#pragma unroll
+                for (int j = 0; j < EPC; ++j) {
+                    float s0 = part[0][0][lane * EPC + j], s1 = part[1][0][lane * EPC + j];
+                    for (int q = 1; q < NW; ++q) { s0 += part[0][q][lane * EPC + j]; s1 += part[1][q][lane * EPC + j]; }
+                    acc[j] = s0; acc_a[j] = s1;
+                }
+                v2_store<T>(P, row, lane, on, acc, acc_a, DA);
             }
-            v2_store<T>(P, row, lane, on, acc, acc_a, DA);
+            __syncthreads();
         }
-        __syncthreads();
     }
 }
 
