@@ -177,16 +177,59 @@ gat_da_final_kernel(const float* __restrict__ partial, int nblocks, int F,
     }
 }
 
-// dal[j,h] = sum over transposed positions q of row j of dz[t2f[q],h]  (any H; H % 4 == 0 goes
-// through the chunked kernel instead)
-__global__ void gat_dal_simple_kernel(const int64_t* __restrict__ rowptrT, const int32_t* __restrict__ t2f,
-                                      int N, int H, const float* __restrict__ dz, float* __restrict__ dal) {
-    int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (t >= (int64_t)N * H) return;
-    const int j = (int)(t / H), h = (int)(t % H);
-    float s = 0.f;
-    for (int64_t q = rowptrT[j]; q < rowptrT[j + 1]; ++q) s += dz[(size_t)t2f[q] * H + h];
-    dal[t] = s;
+// dal[j,h] = sum over transposed positions q of row j of dz[t2f[q],h]  (any H; H % 4 == 0 goes through the chunked
+// kernel instead).  LONG = false: a warp per row of at most DAL_LONG positions, lanes stride over the positions,
+// fixed shuffle tree.  LONG = true: block k owns the rows k, k + blocks, ...; its threads look at DAL_BLOCK of them
+// at once and list the longer ones in shared memory (the order of the list enters no sum), then the whole block
+// takes a listed row: threads stride over its positions, shuffle tree, the warps' sums added in warp order.
+constexpr int DAL_LONG = 1024, DAL_BLOCK = 256;
+template <bool LONG>
+__global__ void __launch_bounds__(DAL_BLOCK) gat_dal_rows_kernel(const int64_t* __restrict__ rowptrT, const int32_t* __restrict__ t2f,
+                                                                 int N, int H, const float* __restrict__ dz, float* __restrict__ dal) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (!LONG) {
+        const int stride = (int)gridDim.x * (DAL_BLOCK / 32);
+        for (int row = (int)blockIdx.x * (DAL_BLOCK / 32) + w; row < N; row += stride) {
+            const int64_t a = rowptrT[row], b = rowptrT[row + 1];
+            if (b - a > DAL_LONG) continue;  // uniform per warp
+            for (int h = 0; h < H; ++h) {
+                float s = 0.f;
+                for (int64_t q = a + lane; q < b; q += 32) s += dz[(size_t)t2f[q] * H + h];
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                if (lane == 0) dal[(size_t)row * H + h] = s;
+            }
+        }
+    } else {
+        __shared__ float red[DAL_BLOCK / 32];
+        __shared__ int list[DAL_BLOCK];
+        __shared__ int count;
+        for (int64_t k0 = 0; (int64_t)blockIdx.x + k0 * gridDim.x < N; k0 += DAL_BLOCK) {
+            __syncthreads();  // every thread is done with the previous list
+            if (threadIdx.x == 0) count = 0;
+            __syncthreads();
+            const int64_t mine = (int64_t)blockIdx.x + (k0 + threadIdx.x) * gridDim.x;
+            if (mine < N && rowptrT[mine + 1] - rowptrT[mine] > DAL_LONG) list[atomicAdd(&count, 1)] = (int)mine;
+            __syncthreads();
+            const int n = count;
+            for (int i = 0; i < n; ++i) {
+                const int row = list[i];
+                const int64_t a = rowptrT[row], b = rowptrT[row + 1];
+                for (int h = 0; h < H; ++h) {
+                    float s = 0.f;
+                    for (int64_t q = a + threadIdx.x; q < b; q += DAL_BLOCK) s += dz[(size_t)t2f[q] * H + h];
+                    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                    if (lane == 0) red[w] = s;
+                    __syncthreads();
+                    if (threadIdx.x == 0) {
+                        float t = red[0];
+                        for (int k = 1; k < DAL_BLOCK / 32; ++k) t += red[k];
+                        dal[(size_t)row * H + h] = t;
+                    }
+                    __syncthreads();
+                }
+            }
+        }
+    }
 }
 
 static bool pow2_le32(int H) { return H >= 1 && H <= 32 && (H & (H - 1)) == 0; }
@@ -322,7 +365,9 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
                          nullptr, nullptr, 0, H, GNN_F32, w.chunk_ws, w.chunk_bytes, st);
         if (rc != GNN_OK) return rc;
     } else {
-        gat_dal_simple_kernel<<<(int)ceil_div((int64_t)g->N * H, 256), 256, 0, st>>>(g->rowptrT, g->t2f, g->N, H, w.dz, w.dal);
+        const int64_t wblocks = ceil_div((int64_t)g->N, DAL_BLOCK / 32);
+        gat_dal_rows_kernel<false><<<(int)(wblocks < 148 * 8 ? wblocks : 148 * 8), DAL_BLOCK, 0, st>>>(g->rowptrT, g->t2f, g->N, H, w.dz, w.dal);
+        gat_dal_rows_kernel<true><<<g->N < 148 * 4 ? g->N : 148 * 4, DAL_BLOCK, 0, st>>>(g->rowptrT, g->t2f, g->N, H, w.dz, w.dal);
         GNN_CHECK_LAUNCH(who);
     }
     // attention-vector gradients: two small reductions that need dal and dar only, on a side branch of the stream

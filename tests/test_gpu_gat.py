@@ -76,6 +76,21 @@ def test_gat_ragged(gnn, dtype, H, C):
     run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, dtype, f"gat H={H} C={C} {dtype}")
 
 
+@pytest.mark.parametrize("H,C", [(1, 64), (2, 16)])
+def test_gat_one_and_two_heads_with_source_hubs(gnn, H, C):
+    """Sources with 5000 and 1025 outgoing edges: the per-source sum of the logit gradients takes the
+    block-per-row path (one and two heads do not go through the chunked reduction)."""
+    n, src, dst = ragged_graph(97 + H)
+    src = src.copy()
+    src[100:5100] = 11
+    src[6000:7025] = 1499
+    Wx = synth.normal((n, H * C), "f32", 960 + H, 1)
+    a = (6.0 / (C + 1)) ** 0.5
+    a_s = synth.uniform_f32((H, C), -a, a, 961, 1)
+    a_d = synth.uniform_f32((H, C), -a, a, 962, 1)
+    run_case(gnn, n, src, dst, Wx, a_s, a_d, H, C, "f32", f"gat source hubs H={H}")
+
+
 def test_gat_zero_attention_is_mean_aggregation(gnn):
     n, src, dst = ragged_graph(95)
     H, C = 4, 16
