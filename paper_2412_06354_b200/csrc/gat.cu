@@ -353,10 +353,12 @@ gnn_status gnn_gat_fused_backward(const gnn_csr* g, const void* Wx, const float*
     // softmax and LeakyReLU derivatives, dz over dalpha, dar per row
     if (!gat_rows_backward_pl(g, alpha_csr, w.dz, al, ar, slope, H, w.dar, st)) {
         const int64_t wwant = ceil_div((int64_t)g->N * 32, GB_BLOCK), cap = (int64_t)148 * 64;
-        gat_backward_rows_kernel<false><<<(int)(wwant < cap ? wwant : cap), GB_BLOCK, 0, st>>>(
-            g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+        cudaStream_t beside = side_fork(st);  // the two tiers write disjoint rows: side by side
         gat_backward_rows_kernel<true><<<(int)(g->N < cap ? g->N : cap), GB_BLOCK, 0, st>>>(
             g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+        gat_backward_rows_kernel<false><<<(int)(wwant < cap ? wwant : cap), GB_BLOCK, 0, beside>>>(
+            g->rowptr, g->col, g->N, H, alpha_csr, w.dz, al, ar, slope, w.dar);
+        side_join(st, beside);
     }
     GNN_CHECK_LAUNCH(who);
     // dal[j,h] = sum over the out-edges of j of dz

@@ -979,8 +979,10 @@ gnn_status gat_alpha(const gnn_csr* g, const float* al, const float* ar, float s
         [&](cudaStream_t q) { gat_alpha_pl_kernel<HV, false><<<wg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha); },    \
         [&](cudaStream_t q) { gat_alpha_pl_kernel<HV, false, 8><<<sg, SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, al, ar, slope, alpha); });
     if (H == 4) { GNN_GA(1) } else if (H == 8) { GNN_GA(2) } else if (H == 16) { GNN_GA(4) } else if (H == 32) { GNN_GA(8) } else {
-        gat_alpha_kernel<false><<<row_grid(g->N, false), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
-        gat_alpha_kernel<true><<<row_grid(g->N, true), SM_BLOCK, 0, st>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha);
+        run_row_tiers(  // the two tiers write disjoint rows: side by side
+            st, [&](cudaStream_t q) { gat_alpha_kernel<true><<<row_grid(g->N, true), SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha); },
+            [&](cudaStream_t q) { gat_alpha_kernel<false><<<row_grid(g->N, false), SM_BLOCK, 0, q>>>(g->rowptr, g->col, g->N, H, al, ar, slope, alpha); },
+            [&](cudaStream_t) {});
     }
 #undef GNN_GA
     GNN_CHECK_LAUNCH("gnn_gat_fused (attention coefficients)");
