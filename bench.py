@@ -48,7 +48,7 @@ TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cl
                   "full-size traffic (better L2 reuse on the reduced matrix); summary under profiles/")
 TRAFFIC_SCALE = 4.0
 TRAFFIC_KERNEL_FILES = ("propagate.cu", "propagate.cuh", "common.cuh")
-TRAFFIC_KERNEL_SHA256 = "ddedf6f68d7848898f03d17a43bc317b1fe739fdec2fcfd710c8c04dda79686e"
+TRAFFIC_KERNEL_SHA256 = "62facf4d2c659f955d3468cd3144d3ed4b685ffbeb12d73cf41affba107fcf9c"
 TRAFFIC_GB_REDUCED = {
     "32:bf16:copy_xj:fwd": 0.192,
     "32:bf16:copy_xj:bwd": 0.19,
@@ -58,38 +58,38 @@ TRAFFIC_GB_REDUCED = {
     "64:bf16:copy_xj:bwd": 0.27,
     "64:bf16:e_mul_xj:fwd": 0.395,
     "64:bf16:e_mul_xj:bwd": 0.395,
-    "128:bf16:copy_xj:fwd": 0.611,
+    "128:bf16:copy_xj:fwd": 0.61,
     "128:bf16:copy_xj:bwd": 0.61,
     "128:bf16:e_mul_xj:fwd": 0.737,
-    "128:bf16:e_mul_xj:bwd": 0.738,
-    "256:bf16:copy_xj:fwd": 2.003,
+    "128:bf16:e_mul_xj:bwd": 0.737,
+    "256:bf16:copy_xj:fwd": 2.004,
     "256:bf16:copy_xj:bwd": 2.004,
     "256:bf16:e_mul_xj:fwd": 2.133,
-    "256:bf16:e_mul_xj:bwd": 2.132,
-    "512:bf16:copy_xj:fwd": 4.017,
+    "256:bf16:e_mul_xj:bwd": 2.133,
+    "512:bf16:copy_xj:fwd": 4.018,
     "512:bf16:copy_xj:bwd": 4.021,
-    "512:bf16:e_mul_xj:fwd": 4.276,
+    "512:bf16:e_mul_xj:fwd": 4.277,
     "512:bf16:e_mul_xj:bwd": 4.281,
-    "32:f32:copy_xj:fwd": 0.256,
-    "32:f32:copy_xj:bwd": 0.256,
+    "32:f32:copy_xj:fwd": 0.257,
+    "32:f32:copy_xj:bwd": 0.258,
     "32:f32:e_mul_xj:fwd": 0.381,
     "32:f32:e_mul_xj:bwd": 0.382,
     "64:f32:copy_xj:fwd": 0.579,
-    "64:f32:copy_xj:bwd": 0.579,
+    "64:f32:copy_xj:bwd": 0.58,
     "64:f32:e_mul_xj:fwd": 0.706,
     "64:f32:e_mul_xj:bwd": 0.706,
     "128:f32:copy_xj:fwd": 1.918,
-    "128:f32:copy_xj:bwd": 1.916,
+    "128:f32:copy_xj:bwd": 1.917,
     "128:f32:e_mul_xj:fwd": 2.047,
-    "128:f32:e_mul_xj:bwd": 2.045,
+    "128:f32:e_mul_xj:bwd": 2.044,
     "256:f32:copy_xj:fwd": 3.848,
-    "256:f32:copy_xj:bwd": 3.842,
+    "256:f32:copy_xj:bwd": 3.843,
     "256:f32:e_mul_xj:fwd": 4.107,
     "256:f32:e_mul_xj:bwd": 4.103,
-    "512:f32:copy_xj:fwd": 7.683,
-    "512:f32:copy_xj:bwd": 7.678,
-    "512:f32:e_mul_xj:fwd": 8.2,
-    "512:f32:e_mul_xj:bwd": 8.197,
+    "512:f32:copy_xj:fwd": 7.685,
+    "512:f32:copy_xj:bwd": 7.68,
+    "512:f32:e_mul_xj:fwd": 8.199,
+    "512:f32:e_mul_xj:bwd": 8.198,
 }
 TRAFFIC_GB = {k: v * TRAFFIC_SCALE for k, v in TRAFFIC_GB_REDUCED.items()}
 

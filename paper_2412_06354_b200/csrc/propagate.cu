@@ -567,6 +567,7 @@ constexpr int FIXL_BLOCKS = 592;
 #define FIXL_MIN_CHUNKS_N 16384
 #endif
 constexpr int64_t FIXL_MIN_CHUNKS = FIXL_MIN_CHUNKS_N;  // below this many chunks the extra launch costs more than the walk
+constexpr int64_t FIXL_MIN_CHUNKS_ARG = 4096;           // the same for max / min
 
 // second pass: finish the rows that were cut by chunk boundaries, in ascending chunk order
 template <typename T, int MODE>
@@ -581,7 +582,7 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
     if (r < 0) return;
     const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
     const int64_t c_end = (re - 1) / P.chunk;
-    if (!ARG && P.fix_long && c_end - c > FIX_LONG) return;  // a hub row: propagate_fixup_long_kernel finishes it
+    if (P.fix_long && c_end - c > FIX_LONG) return;  // a hub row: propagate_fixup_long_kernel finishes it
     float v[EPC];
     int32_t a[EPC];
     const size_t F = P.F;
@@ -648,16 +649,19 @@ __global__ void propagate_fixup_kernel(const PropParams P) {
     }
 }
 
-// Sum modes only.  Block b looks at its share of the chunks; for every row that starts in one of them and is cut
+// Block b looks at its share of the chunks; for every row that starts in one of them and is cut
 // into more than FIX_LONG chunks, thread (k, q) adds column float4 q of the partial rows k, k + K, k + 2K, ... of
 // that row (K = 256 / (F/4) walkers per column, four loads in flight each), the K sums are added in walker order,
 // and the row is scaled, given its epilogue and stored as in the kernel above.  The order of the additions is a
-// fixed function of the row's length and F.
+// fixed function of the row's length and F.  Max / min: the walkers keep (value, position) pairs and combine them
+// with the same rule as everywhere else (ties go to the smaller position), which does not depend on the order.
 template <typename T, int MODE>
 __global__ void __launch_bounds__(FIXL_THREADS)
 propagate_fixup_long_kernel(const PropParams P) {
     constexpr int EPC = Chunk<T>::N;
+    constexpr bool ARG = (MODE == MODE_MAX || MODE == MODE_MIN);
     __shared__ float4 sums[FIXL_THREADS];
+    __shared__ int4 args[ARG ? FIXL_THREADS : 1];
     __shared__ int todo[64];
     __shared__ int ntodo;
     const int tid = threadIdx.x;
@@ -682,35 +686,59 @@ propagate_fixup_long_kernel(const PropParams P) {
             const int64_t rs = P.rowptr[r], re = P.rowptr[r + 1];
             const int64_t span = (re - 1) / P.chunk - c;  // partial rows: (c, tail), then the heads of c + 1 .. c + span
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            int4 arg = make_int4(-1, -1, -1, -1);
             if (k < K && q < F4) {
                 for (int64_t j = k; j <= span; j += 4 * (int64_t)K) {
                     float4 t[4];
+                    int4 ta[ARG ? 4 : 1];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const int64_t jj = j + (int64_t)u * K;
                         if (jj <= span) {
                             const size_t slot = jj == 0 ? (size_t)c * 2 + 1 : (size_t)(c + jj) * 2;
                             t[u] = *(reinterpret_cast<const float4*>(P.part_val + slot * (size_t)F) + q);
+                            if (ARG) ta[u] = *(reinterpret_cast<const int4*>(P.part_arg + slot * (size_t)F) + q);
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        if (j + (int64_t)u * K <= span) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+                        if (j + (int64_t)u * K <= span) {
+                            if (ARG) {
+                                if (beats<MODE>(t[u].x, ta[u].x, acc.x, arg.x)) { acc.x = t[u].x; arg.x = ta[u].x; }
+                                if (beats<MODE>(t[u].y, ta[u].y, acc.y, arg.y)) { acc.y = t[u].y; arg.y = ta[u].y; }
+                                if (beats<MODE>(t[u].z, ta[u].z, acc.z, arg.z)) { acc.z = t[u].z; arg.z = ta[u].z; }
+                                if (beats<MODE>(t[u].w, ta[u].w, acc.w, arg.w)) { acc.w = t[u].w; arg.w = ta[u].w; }
+                            } else {
+                                acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w;
+                            }
+                        }
                 }
                 sums[k * F4 + q] = acc;
+                if (ARG) args[k * F4 + q] = arg;
             }
             __syncthreads();
             if (tid < P.nvec) {
                 const int ci = tid;
                 float v[EPC];
+                int32_t av[ARG ? EPC : 1];
 #pragma unroll
                 for (int j4 = 0; j4 < EPC / 4; ++j4) {
                     float4 a = sums[ci * (EPC / 4) + j4];
+                    int4 aa = ARG ? args[ci * (EPC / 4) + j4] : make_int4(-1, -1, -1, -1);
                     for (int kk = 1; kk < K; ++kk) {
                         const float4 b = sums[kk * F4 + ci * (EPC / 4) + j4];
-                        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                        if (ARG) {
+                            const int4 ba = args[kk * F4 + ci * (EPC / 4) + j4];
+                            if (beats<MODE>(b.x, ba.x, a.x, aa.x)) { a.x = b.x; aa.x = ba.x; }
+                            if (beats<MODE>(b.y, ba.y, a.y, aa.y)) { a.y = b.y; aa.y = ba.y; }
+                            if (beats<MODE>(b.z, ba.z, a.z, aa.z)) { a.z = b.z; aa.z = ba.z; }
+                            if (beats<MODE>(b.w, ba.w, a.w, aa.w)) { a.w = b.w; aa.w = ba.w; }
+                        } else {
+                            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                        }
                     }
                     v[4 * j4] = a.x; v[4 * j4 + 1] = a.y; v[4 * j4 + 2] = a.z; v[4 * j4 + 3] = a.w;
+                    if (ARG) { av[4 * j4] = aa.x; av[4 * j4 + 1] = aa.y; av[4 * j4 + 2] = aa.z; av[4 * j4 + 3] = aa.w; }
                 }
                 if (P.mean) {
                     const float d = (float)(re - rs);
@@ -726,6 +754,11 @@ propagate_fixup_long_kernel(const PropParams P) {
                 row_epilogue<T>(P, r, ci, v);
                 char* ob = reinterpret_cast<char*>(P.out) + (size_t)r * P.out_ld + (size_t)ci * 16;
                 *reinterpret_cast<uint4*>(ob) = Chunk<T>::pack(v);
+                if (ARG && P.argmax) {
+                    int32_t* ap = P.argmax + (size_t)r * F + (size_t)ci * EPC;
+#pragma unroll
+                    for (int j = 0; j < EPC; ++j) ap[j] = av[j];
+                }
             }
             __syncthreads();
         }
@@ -1560,7 +1593,10 @@ gnn_status run_chunked(const char* who, int mode, int32_t N, int64_t E, const in
     if (flat_by_degree(mode, N, E, nvec, s)) { P.chunk = P.chunk < PF_SLAB ? P.chunk : PF_SLAB; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
     if (sum_half_slab(mode, N, E, nvec)) { P.chunk = PF_SLAB / 2; P.nchunks = ceil_div(E, (int64_t)P.chunk); }
     P.tail_row = wsv.tail_row; P.part_val = wsv.part_val; P.part_arg = wsv.part_arg;
-    P.fix_long = (!with_arg && P.nchunks >= FIXL_MIN_CHUNKS) ? 1 : 0;
+    // also where the mean row is long (pooling over a few large graphs), and from fewer chunks on for max / min, whose
+    // walk compares (value, position) pairs one partial row after the other
+    const bool long_mean = E / N > (int64_t)FIX_LONG * P.chunk && P.nchunks > FIX_LONG;
+    P.fix_long = (P.nchunks >= (with_arg ? FIXL_MIN_CHUNKS_ARG : FIXL_MIN_CHUNKS) || long_mean) ? 1 : 0;
     P.wh = nullptr; P.wh_index = nullptr; P.H = 1; P.fph = F; P.epi_l = P.epi_r = P.epi_a = P.epi_b = nullptr;
     if (hx) {
         const int epc = 16 / s;

@@ -219,6 +219,32 @@ def test_batched_pooling(gnn, dtype):
             assert_close(to_host64(dX), ref, np.abs(ref), dtype, f"reduce_nodes_backward {op}")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_pooling_over_graphs_of_a_million_nodes(gnn, dtype):
+    """Two graphs of 700000 and 499980 nodes around one of 20: a graph spans thousands of chunks of the reduction,
+    so its partial results are combined by the block-per-row pass, for max / min with the winning positions."""
+    import torch
+    sizes = [700_000, 20, 499_980]
+    gp = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n, F = int(gp[-1]), 32
+    X = feats((n, F), dtype, 1234)
+    p0 = int(oracle.reduce_nodes("max", gp, X)[2][0, 0])  # the winner of column 0 in the first graph ...
+    X[(p0 + 350_000) % 700_000] = X[p0]                   # ... now has a twin far away: the smaller position wins
+    gptr = to_dev(gp)
+    R = feats((3, F), dtype, 1235)
+    for op in ("mean", "max", "min"):
+        got = gnn.reduce_nodes(gptr, to_dev(X), op)
+        o, S, a = oracle.reduce_nodes(op, gp, X)
+        if op in ("max", "min"):
+            out, arg = got
+            assert np.array_equal(bits(out), f64_to_dtype_bits(o, dtype))
+            assert np.array_equal(arg.cpu().numpy(), a)
+            again = gnn.reduce_nodes(gptr, to_dev(X), op)
+            assert torch.equal(again[1], arg)
+        else:
+            assert_close(to_host64(got), o, S, dtype, f"reduce_nodes {op}")
+
+
 def test_pooling_edge_cases(gnn):
     import torch
     # an empty graph in the middle of the batch, and unsorted ids
