@@ -371,19 +371,44 @@ __global__ void degree_unit_kernel(int32_t N, const int64_t* __restrict__ rowptr
     if (i < N) deg[i] = (float)(rowptr[i + 1] - rowptr[i]);
 }
 
-__global__ void gcn_coef_kernel(int32_t N, const int64_t* __restrict__ rowptr,
-                                const int32_t* __restrict__ col, const float* __restrict__ w,
-                                const float* __restrict__ deg, float* __restrict__ coef) {
-    int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    int lane = threadIdx.x & 31;
-    if (row >= N) return;
-    int64_t a = rowptr[row], b = rowptr[row + 1];
-    float di = deg[row];
-    for (int64_t p = a + lane; p < b; p += 32) {
-        float dj = deg[col[p]];
-        float wp = w ? w[p] : 1.0f;
-        // IEEE sqrt and division (no approximate rsqrt): ~1e-7 relative
-        coef[p] = (di > 0.f && dj > 0.f) ? __fdiv_rn(wp, __fsqrt_rn(di * dj)) : 0.f;
+// coef[p] = w[p] / sqrt(deg[row(p)] * deg[col[p]]).  LONG = false: a warp per row of at most GC_LONG positions.
+// LONG = true: block k owns the rows k, k + blocks, ...; its threads look at 256 of them at once, list the longer ones
+// in shared memory, and the whole block takes a listed row (a single warp would walk a hub of 10^5 positions alone).
+constexpr int GC_LONG = 1024;
+__device__ __forceinline__ float gcn_coef(float wp, float di, float dj) {
+    // IEEE sqrt and division (no approximate rsqrt): ~1e-7 relative
+    return (di > 0.f && dj > 0.f) ? __fdiv_rn(wp, __fsqrt_rn(di * dj)) : 0.f;
+}
+template <bool LONG>
+__global__ void __launch_bounds__(256) gcn_coef_kernel(int32_t N, const int64_t* __restrict__ rowptr,
+                                                       const int32_t* __restrict__ col, const float* __restrict__ w,
+                                                       const float* __restrict__ deg, float* __restrict__ coef) {
+    if (!LONG) {
+        int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+        int lane = threadIdx.x & 31;
+        if (row >= N) return;
+        int64_t a = rowptr[row], b = rowptr[row + 1];
+        if (b - a > GC_LONG) return;
+        float di = deg[row];
+        for (int64_t p = a + lane; p < b; p += 32) coef[p] = gcn_coef(w ? w[p] : 1.0f, di, deg[col[p]]);
+    } else {
+        __shared__ int list[256];
+        __shared__ int count;
+        for (int64_t k0 = 0; (int64_t)blockIdx.x + k0 * gridDim.x < N; k0 += 256) {
+            __syncthreads();  // every thread is done with the previous list
+            if (threadIdx.x == 0) count = 0;
+            __syncthreads();
+            const int64_t mine = (int64_t)blockIdx.x + (k0 + threadIdx.x) * gridDim.x;
+            if (mine < N && rowptr[mine + 1] - rowptr[mine] > GC_LONG) list[atomicAdd(&count, 1)] = (int)mine;
+            __syncthreads();
+            const int n = count;
+            for (int i = 0; i < n; ++i) {  // the order of the list does not matter: every position is written once
+                const int row = list[i];
+                const int64_t a = rowptr[row], b = rowptr[row + 1];
+                const float di = deg[row];
+                for (int64_t p = a + threadIdx.x; p < b; p += 256) coef[p] = gcn_coef(w ? w[p] : 1.0f, di, deg[col[p]]);
+            }
+        }
     }
 }
 
@@ -568,7 +593,8 @@ gnn_status gnn_gcn_norm(const gnn_csr* g, const float* w_csr, float* deg_out, fl
         degree_unit_kernel<<<(int)ceil_div(g->N, 256), 256, 0, st>>>(g->N, g->rowptr, deg_out);
     if (coef_csr && g->E > 0) {
         GNN_REQUIRE(g->col, GNN_ERR_INVALID_ARG, "gnn_gcn_norm: null col");
-        gcn_coef_kernel<<<(int)ceil_div((int64_t)g->N * 32, 256), 256, 0, st>>>(g->N, g->rowptr, g->col, w_csr, deg_out, coef_csr);
+        gcn_coef_kernel<false><<<(int)ceil_div((int64_t)g->N * 32, 256), 256, 0, st>>>(g->N, g->rowptr, g->col, w_csr, deg_out, coef_csr);
+        gcn_coef_kernel<true><<<g->N < 148 * 8 ? g->N : 148 * 8, 256, 0, st>>>(g->N, g->rowptr, g->col, w_csr, deg_out, coef_csr);
         if (coef_csrT) {
             GNN_REQUIRE(g->t2f, GNN_ERR_INVALID_ARG, "gnn_gcn_norm: null t2f");
             permute_f32_kernel<<<grid_for(g->E, 256), 256, 0, st>>>(g->E, g->t2f, coef_csr, coef_csrT);
